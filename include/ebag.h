@@ -1,0 +1,157 @@
+/*
+ * ebag.h -- C ABI of libebag.so: jagged, pooled embedding-bag forward over one or many tables
+ * ("TBE", table-batched embedding) on one NVIDIA B200 (sm_100a).
+ *
+ * The operator.  Recommendation models keep categorical features as embedding tables whose
+ * lookups are memory-bound and irregular ("embedding lookup and aggregation kernels optimized
+ * for irregular memory access patterns", paper Sec. 1.1, paragraph "Model Diversity Across
+ * Ranking Stages"; "sparse feature embeddings", Sec. 2.1, paragraph "DLRM Architecture").
+ * The ids arrive as jagged lists of int64 and, for weighted features, as (int64 id, float32
+ * score) pairs (Sec. 2.2, paragraph "Feature Types and Memory Layout").  For T tables and B
+ * bags per table this library computes, with bag id g = t*B + b,
+ *
+ *     out[b, Doff[t] + d] = pool_{i = offsets[g] .. offsets[g+1]-1} w_i * value(t, indices[i], d)
+ *
+ * where pool is a sum or (EBAG_MEAN) the sum divided by the bag length L = offsets[g+1] -
+ * offsets[g] (an empty bag gives +0.0f in every mode), w_i = per_sample_weights[i] or 1, and
+ * value() widens the stored element to fp32 (fp16 and bf16 exactly; rowwise int8 as
+ * scale[row]*q + bias[row]).  Accumulation and output are fp32.  Doff is the running sum of D.
+ * Batching every table behind one launch follows the flattened-array-plus-offsets idea the
+ * paper uses for its own jagged preprocessing kernels (Sec. 5.4, "Data Preprocessing Kernels on
+ * MTIA", MBDT; Sec. 5.5, "Batch Event Truncate").
+ *
+ * Conventions.  "device" pointers are CUDA global-memory pointers on the handle's device;
+ * "host" pointers are ordinary process memory.  Nothing here takes ownership of a caller's
+ * buffer.  ebag_stream is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ * Unless stated otherwise a call only enqueues work on the stream and returns; the caller keeps
+ * every buffer alive until the stream has passed that work.  One forward per handle may be in
+ * flight at a time (the handle's work-queue counters and status words are shared).
+ * There is no CPU fallback: without a usable CUDA device every call fails with EBAG_ERR_CUDA.
+ */
+#ifndef EBAG_H_
+#define EBAG_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct ebag_tbe ebag_tbe; /* opaque, library-owned */
+typedef void* ebag_stream;        /* a cudaStream_t */
+
+typedef enum {
+    EBAG_OK = 0,
+    EBAG_ERR_INVALID_ARG = 1, /* NULL where a pointer is required, T<=0, B<0, bad D, ... */
+    EBAG_ERR_UNSUPPORTED = 2, /* mean pooling with weights; sizes beyond the stated limits */
+    EBAG_ERR_CUDA = 3,        /* a CUDA runtime call failed (see ebag_last_cuda_error) */
+    EBAG_ERR_INDEX_OOB = 4,   /* reported by ebag_last_status: ids outside [0, rows) were skipped */
+    EBAG_ERR_BAD_OFFSETS = 5  /* reported by ebag_last_status: malformed bags were treated as empty */
+} ebag_status;
+
+typedef enum { EBAG_F32 = 0, EBAG_F16 = 1, EBAG_BF16 = 2, EBAG_INT8_ROWWISE = 3 } ebag_dtype;
+
+/* weighted sum = EBAG_SUM with per_sample_weights != NULL */
+typedef enum { EBAG_SUM = 0, EBAG_MEAN = 1 } ebag_mode;
+
+#define EBAG_MAX_TABLES 2048
+
+/*
+ * Bytes from one stored row to the next.  F32/F16/BF16: D * element size.  INT8_ROWWISE: the
+ * packed row [D int8 codes][fp32 scale][fp32 bias][8 bytes pad] = D + 16 (one gather fetches
+ * codes and dequantisation constants together).  Returns -1 if D is not allowed for the dtype:
+ * D > 0 and D * element size must be a multiple of 16 bytes (D%4==0 for F32, D%8==0 for
+ * F16/BF16, D%16==0 for INT8_ROWWISE), so that rows can be gathered with 128-bit loads.
+ */
+int64_t ebag_row_stride(ebag_dtype dtype, int32_t D);
+
+/*
+ * Create a handle for T tables of `dtype` with rows[t] rows (0 <= rows[t] < 2^31) of D[t]
+ * elements on CUDA device `device`.  rows and D are host arrays [T], copied.  1 <= T <=
+ * EBAG_MAX_TABLES.  Allocates a few KB of device memory (per-table metadata, work-queue
+ * counters, status words) that the handle owns until ebag_destroy.  Synchronous.
+ * Errors: INVALID_ARG, UNSUPPORTED (T or rows too large), CUDA.
+ */
+ebag_status ebag_create_tbe(int32_t T, const int64_t* rows, const int32_t* D, ebag_dtype dtype,
+                            int device, ebag_tbe** out);
+
+/*
+ * Pooled forward for all T tables in ONE kernel launch on `stream` (the operator defined at
+ * the top of this file).
+ *   tables   host array [T] of DEVICE pointers; table t is row-major with row pitch
+ *            ebag_row_stride(dtype, D[t]) bytes, 16-byte aligned.  The array is read before the
+ *            call returns.
+ *   D        host [T]; must equal the create-time D (checked).
+ *   indices  device int64 [n_indices]: the concatenated id lists, table-major.
+ *   n_indices  length of indices (and of per_sample_weights); bags reaching past it are malformed.
+ *   offsets  device int64 [T*B + 1], non-decreasing, offsets[0] == 0: bag g = t*B + b owns
+ *            indices[offsets[g] .. offsets[g+1]).
+ *   per_sample_weights  device fp32 [n_indices] or NULL (must be NULL for EBAG_MEAN).
+ *   B        bags per table, B >= 0, T*B < 2^31.
+ *   out      device fp32 [B, sum(D)] row-major, 16-byte aligned; every element is overwritten
+ *            exactly once; must not alias an input.
+ * No allocation, no host-device synchronisation.  Host-detectable problems return an error and
+ * launch nothing.  Problems only the device can see never fault: an id outside [0, rows[t]) is
+ * skipped (it adds nothing but still counts in the mean's divisor) and a bag with
+ * offsets[g+1] < offsets[g], or reaching outside [0, n_indices], is treated as empty; both are
+ * counted and reported by ebag_last_status.  B == 0 or n_indices == 0 is fine.
+ */
+ebag_status ebag_forward(ebag_tbe* h, const void* const* tables, const int32_t* D,
+                         const int64_t* indices, int64_t n_indices, const int64_t* offsets,
+                         const float* per_sample_weights, int64_t B, ebag_mode mode, float* out,
+                         ebag_stream stream);
+
+/*
+ * The same forward for callers whose per-step data lives in HOST memory: indices, offsets,
+ * per_sample_weights and out are host pointers (pinned memory makes the copies asynchronous);
+ * tables stay device pointers (they are model state, loaded once).  The call copies the inputs
+ * to device staging buffers owned by the handle, runs the forward, and copies the result back,
+ * all on `stream`; the caller synchronises the stream before reading `out`.  The staging
+ * buffers are (re)allocated inside this call whenever n_indices or B exceed what they hold, so
+ * the first call, and any call with larger inputs, allocates and synchronises.
+ */
+ebag_status ebag_forward_host(ebag_tbe* h, const void* const* tables, const int32_t* D,
+                              const int64_t* indices, int64_t n_indices, const int64_t* offsets,
+                              const float* per_sample_weights, int64_t B, ebag_mode mode,
+                              float* out, ebag_stream stream);
+
+/*
+ * Wait for `stream`, then report and clear what the device counted since the last call:
+ * *n_oob = ids skipped as out of range, *n_bad_offsets = malformed bags (either pointer may be
+ * NULL).  Returns EBAG_ERR_BAD_OFFSETS, else EBAG_ERR_INDEX_OOB, else EBAG_OK.  The only call
+ * that synchronises besides create/destroy.
+ */
+ebag_status ebag_last_status(ebag_tbe* h, ebag_stream stream, int64_t* n_oob,
+                             int64_t* n_bad_offsets);
+
+/*
+ * Load-time helper: build the packed INT8_ROWWISE table (see ebag_row_stride) from separate
+ * device arrays q [rows, D] int8, scale [rows] fp32, bias [rows] fp32 into device buffer dst
+ * (rows * ebag_row_stride bytes, 16-byte aligned).  Enqueued on `stream`.
+ */
+ebag_status ebag_pack_int8_rowwise(const int8_t* q, const float* scale, const float* bias,
+                                   int64_t rows, int32_t D, void* dst, ebag_stream stream);
+
+/*
+ * Tuning knobs, for experiments; defaults are chosen at create.  Names:
+ *   "item_bytes"   target bytes of gathered rows per work item (default 32768)
+ *   "ctas_per_sm"  resident CTAs per SM of the persistent grid (default: occupancy limit)
+ * Returns INVALID_ARG for an unknown name or a value out of range.
+ */
+ebag_status ebag_set_param(ebag_tbe* h, const char* name, int64_t value);
+
+/* Number of kernels this handle has launched so far (forward and host-forward). */
+int64_t ebag_launch_count(const ebag_tbe* h);
+
+/* Text of the last CUDA error seen by this handle ("" if none). */
+const char* ebag_last_cuda_error(const ebag_tbe* h);
+
+/* Frees the handle and its device memory.  Synchronises the device.  NULL is allowed. */
+void ebag_destroy(ebag_tbe* h);
+
+const char* ebag_status_string(ebag_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* EBAG_H_ */

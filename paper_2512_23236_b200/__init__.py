@@ -1,0 +1,203 @@
+"""Python binding of libebag.so: the pooled embedding-bag forward on one B200.
+
+Argument marshalling only.  Every step of the operator runs in the library's CUDA kernels;
+torch is used to hold device memory and to name the stream.  The functions carry the names of
+the C entry points declared in ``include/ebag.h``; ``TBE`` is a small convenience wrapper around
+a handle.  There is no CPU fallback: if ``libebag.so`` has not been built (``python -m
+paper_2512_23236_b200.build``) or no CUDA device is usable, calls raise.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import List, Optional, Sequence
+
+EBAG_F32, EBAG_F16, EBAG_BF16, EBAG_INT8_ROWWISE = 0, 1, 2, 3
+EBAG_SUM, EBAG_MEAN = 0, 1
+EBAG_OK, EBAG_ERR_INVALID_ARG, EBAG_ERR_UNSUPPORTED, EBAG_ERR_CUDA = 0, 1, 2, 3
+EBAG_ERR_INDEX_OOB, EBAG_ERR_BAD_OFFSETS = 4, 5
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libebag.so")
+
+# name -> (restype, argtypes); kept in step with include/ebag.h (a test parses the header)
+_vp, _i32, _i64, _int = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_int
+SIGNATURES = {
+    "ebag_row_stride": (_i64, [_int, _i32]),
+    "ebag_create_tbe": (_int, [_i32, _vp, _vp, _int, _int, _vp]),
+    "ebag_forward": (_int, [_vp, _vp, _vp, _vp, _i64, _vp, _vp, _i64, _int, _vp, _vp]),
+    "ebag_forward_host": (_int, [_vp, _vp, _vp, _vp, _i64, _vp, _vp, _i64, _int, _vp, _vp]),
+    "ebag_last_status": (_int, [_vp, _vp, _vp, _vp]),
+    "ebag_pack_int8_rowwise": (_int, [_vp, _vp, _vp, _i64, _i32, _vp, _vp]),
+    "ebag_set_param": (_int, [_vp, ctypes.c_char_p, _i64]),
+    "ebag_launch_count": (_i64, [_vp]),
+    "ebag_last_cuda_error": (ctypes.c_char_p, [_vp]),
+    "ebag_destroy": (None, [_vp]),
+    "ebag_status_string": (ctypes.c_char_p, [_int]),
+}
+
+_lib = None
+
+
+class EbagError(RuntimeError):
+    def __init__(self, status: int, what: str = ""):
+        self.status = status
+        msg = lib().ebag_status_string(status).decode()
+        super().__init__(f"{what}: {msg}" if what else msg)
+
+
+def lib():
+    """The loaded library (loads it on first use; raises if it is missing)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(f"{LIB_PATH} not found: build it with "
+                              "`python -m paper_2512_23236_b200.build` (there is no fallback path)")
+        L = ctypes.CDLL(LIB_PATH)
+        for name, (res, args) in SIGNATURES.items():
+            fn = getattr(L, name)
+            fn.restype = res
+            fn.argtypes = args
+        _lib = L
+    return _lib
+
+
+def _check(status: int, what: str):
+    if status != EBAG_OK:
+        raise EbagError(status, what)
+
+
+def _stream_ptr(stream) -> int:
+    import torch
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return int(stream.cuda_stream) if hasattr(stream, "cuda_stream") else int(stream)
+
+
+def _ptr(t) -> Optional[int]:
+    return None if t is None else int(t.data_ptr())
+
+
+# ---------------------------------------------------------------- functions named as the C ABI
+def ebag_row_stride(dtype: int, D: int) -> int:
+    return int(lib().ebag_row_stride(dtype, D))
+
+
+def ebag_create_tbe(rows: Sequence[int], D: Sequence[int], dtype: int, device: int = 0) -> int:
+    """Returns the handle as an integer address."""
+    T = len(rows)
+    r = (ctypes.c_int64 * T)(*[int(x) for x in rows])
+    d = (ctypes.c_int32 * T)(*[int(x) for x in D])
+    h = ctypes.c_void_p(0)
+    st = lib().ebag_create_tbe(T, ctypes.cast(r, _vp), ctypes.cast(d, _vp), dtype, device,
+                               ctypes.addressof(h))
+    _check(st, "ebag_create_tbe")
+    return int(h.value)
+
+
+def ebag_forward(h: int, table_ptrs: Sequence[int], D: Sequence[int], indices_ptr, n_indices: int,
+                 offsets_ptr, weights_ptr, B: int, mode: int, out_ptr, stream_ptr,
+                 host: bool = False) -> None:
+    T = len(table_ptrs)
+    tp = (ctypes.c_void_p * T)(*[int(p) if p else None for p in table_ptrs])
+    d = (ctypes.c_int32 * T)(*[int(x) for x in D])
+    fn = lib().ebag_forward_host if host else lib().ebag_forward
+    st = fn(h, ctypes.cast(tp, _vp), ctypes.cast(d, _vp), indices_ptr, n_indices, offsets_ptr,
+            weights_ptr, B, mode, out_ptr, stream_ptr)
+    _check(st, "ebag_forward_host" if host else "ebag_forward")
+
+
+def ebag_last_status(h: int, stream_ptr) -> tuple:
+    """(status, n_oob, n_bad_offsets); synchronises the stream."""
+    a, b = ctypes.c_int64(0), ctypes.c_int64(0)
+    st = lib().ebag_last_status(h, stream_ptr, ctypes.addressof(a), ctypes.addressof(b))
+    if st == EBAG_ERR_CUDA or st == EBAG_ERR_INVALID_ARG:
+        raise EbagError(st, "ebag_last_status")
+    return int(st), int(a.value), int(b.value)
+
+
+def ebag_destroy(h: int) -> None:
+    lib().ebag_destroy(h)
+
+
+def ebag_pack_int8_rowwise(q, scale, bias, stream=None):
+    """torch int8 [rows, D], fp32 [rows], fp32 [rows] (device) -> packed uint8 [rows, D+16]."""
+    import torch
+    rows, D = q.shape
+    stride = ebag_row_stride(EBAG_INT8_ROWWISE, D)
+    if stride < 0:
+        raise EbagError(EBAG_ERR_INVALID_ARG, "ebag_pack_int8_rowwise")
+    q = q.contiguous()
+    scale = scale.contiguous().float()
+    bias = bias.contiguous().float()
+    dst = torch.empty((rows, stride), dtype=torch.uint8, device=q.device)
+    with torch.cuda.device(q.device):
+        st = lib().ebag_pack_int8_rowwise(_ptr(q), _ptr(scale), _ptr(bias), rows, D, _ptr(dst),
+                                          _stream_ptr(stream))
+    _check(st, "ebag_pack_int8_rowwise")
+    return dst
+
+
+# ---------------------------------------------------------------- convenience wrapper
+class TBE:
+    """A handle for T tables.  ``tables`` passed to forward() are torch device tensors laid out
+    as the library expects: [rows, D] of float32 / float16 / bfloat16, or for rowwise int8 the
+    packed uint8 [rows, D+16] tensor from ebag_pack_int8_rowwise()."""
+
+    def __init__(self, rows: Sequence[int], D: Sequence[int], dtype: int, device: int = 0):
+        self.rows = [int(r) for r in rows]
+        self.D = [int(d) for d in D]
+        self.dtype = dtype
+        self.device = device
+        self.sumD = sum(self.D)
+        self._h = ebag_create_tbe(self.rows, self.D, dtype, device)
+
+    @property
+    def T(self) -> int:
+        return len(self.rows)
+
+    def close(self):
+        if self._h:
+            ebag_destroy(self._h)
+            self._h = 0
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def set_param(self, name: str, value: int):
+        _check(lib().ebag_set_param(self._h, name.encode(), int(value)), "ebag_set_param")
+
+    def launch_count(self) -> int:
+        return int(lib().ebag_launch_count(self._h))
+
+    def last_cuda_error(self) -> str:
+        return lib().ebag_last_cuda_error(self._h).decode()
+
+    def forward(self, tables: List, indices, offsets, B: int, mode: int = EBAG_SUM,
+                per_sample_weights=None, out=None, stream=None):
+        """Device tensors in, device tensor out ([B, sum D] float32).  Enqueues only."""
+        import torch
+        if out is None:
+            out = torch.empty((B, self.sumD), dtype=torch.float32, device=indices.device)
+        ebag_forward(self._h, [t.data_ptr() for t in tables], self.D, _ptr(indices),
+                     int(indices.numel()), _ptr(offsets), _ptr(per_sample_weights), B, mode,
+                     _ptr(out), _stream_ptr(stream))
+        return out
+
+    def forward_host(self, tables: List, indices, offsets, B: int, mode: int = EBAG_SUM,
+                     per_sample_weights=None, out=None, stream=None):
+        """Host (ideally pinned) tensors for indices/offsets/weights/out, device tables.
+        The caller synchronises the stream before reading ``out``."""
+        import torch
+        if out is None:
+            out = torch.empty((B, self.sumD), dtype=torch.float32).pin_memory()
+        ebag_forward(self._h, [t.data_ptr() for t in tables], self.D, _ptr(indices),
+                     int(indices.numel()), _ptr(offsets), _ptr(per_sample_weights), B, mode,
+                     _ptr(out), _stream_ptr(stream), host=True)
+        return out
+
+    def last_status(self, stream=None) -> tuple:
+        return ebag_last_status(self._h, _stream_ptr(stream))

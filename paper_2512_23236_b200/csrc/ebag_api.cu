@@ -1,0 +1,420 @@
+// Host side of libebag.so: argument checks, the handle and its few KB of device state, and the
+// kernel launches.  Declarations and the contract of every entry point are in include/ebag.h.
+#include <cuda_runtime.h>
+
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "ebag.h"
+#include "ebag_fwd.cuh"
+
+using namespace ebag;
+
+namespace {
+
+constexpr int kTableSlots = 4;   // device copies of the table-pointer array that may be in flight
+
+struct DeviceGuard {             // make the handle's device current for the duration of a call
+    int prev = -1;
+    bool ok = false;
+    explicit DeviceGuard(int dev) {
+        if (cudaGetDevice(&prev) != cudaSuccess) return;
+        ok = (prev == dev) || cudaSetDevice(dev) == cudaSuccess;
+        if (prev == dev) prev = -1;
+    }
+    ~DeviceGuard() {
+        if (prev >= 0) cudaSetDevice(prev);
+    }
+};
+
+int elem_bytes(int dtype) { return dtype == EBAG_F32 ? 4 : (dtype == EBAG_INT8_ROWWISE ? 1 : 2); }
+
+}  // namespace
+
+struct ebag_tbe {
+    int T = 0, dtype = 0, device = 0, sumD = 0, num_sms = 0;
+    std::vector<int64_t> rows;
+    std::vector<int32_t> D;
+    TableMeta* d_meta = nullptr;
+    Queue* d_queue = nullptr;
+    Status* d_status = nullptr;
+    // table pointers: cached on the device, re-sent only when the caller's array changes
+    const void** d_tables[kTableSlots] = {};
+    const void** h_tables[kTableSlots] = {};       // pinned
+    cudaEvent_t slot_event[kTableSlots] = {};
+    bool slot_busy[kTableSlots] = {};
+    int slot = -1;
+    int occupancy[2] = {0, 0};                     // CTAs per SM, [unweighted, weighted]
+    uint32_t item_bytes = 32768;
+    int ctas_per_sm = 0;                           // 0: occupancy limit
+    int64_t launches = 0;
+    std::string cuda_error;
+    // staging for ebag_forward_host
+    int64_t* s_indices = nullptr;
+    int64_t* s_offsets = nullptr;
+    float* s_weights = nullptr;
+    float* s_out = nullptr;
+    int64_t cap_indices = 0, cap_offsets = 0, cap_weights = 0, cap_out = 0;
+};
+
+namespace {
+
+ebag_status cuda_fail(ebag_tbe* h, cudaError_t e) {
+    if (h) h->cuda_error = cudaGetErrorString(e);
+    cudaGetLastError();   // clear the sticky-less error state
+    return EBAG_ERR_CUDA;
+}
+
+#define EBAG_CUDA(h, call)                                 \
+    do {                                                   \
+        cudaError_t e__ = (call);                          \
+        if (e__ != cudaSuccess) return cuda_fail(h, e__);  \
+    } while (0)
+
+void free_handle(ebag_tbe* h) {
+    if (!h) return;
+    cudaFree(h->d_meta);
+    cudaFree(h->d_queue);
+    cudaFree(h->d_status);
+    for (int i = 0; i < kTableSlots; ++i) {
+        cudaFree(h->d_tables[i]);
+        if (h->h_tables[i]) cudaFreeHost(h->h_tables[i]);
+        if (h->slot_event[i]) cudaEventDestroy(h->slot_event[i]);
+    }
+    cudaFree(h->s_indices);
+    cudaFree(h->s_offsets);
+    cudaFree(h->s_weights);
+    cudaFree(h->s_out);
+    delete h;
+}
+
+size_t fwd_smem_bytes(int T) { return (size_t)(2 * T + 1) * sizeof(int); }
+
+cudaError_t launch_fwd(int dtype, const FwdParams& p, bool w, int grid, size_t smem, cudaStream_t s) {
+    switch (dtype) {
+        case EBAG_F32: return launch_fwd_f32(p, w, grid, smem, s);
+        case EBAG_F16: return launch_fwd_f16(p, w, grid, smem, s);
+        case EBAG_BF16: return launch_fwd_bf16(p, w, grid, smem, s);
+        default: return launch_fwd_int8(p, w, grid, smem, s);
+    }
+}
+
+cudaError_t occupancy_fwd(int dtype, bool w, size_t smem, int* n) {
+    switch (dtype) {
+        case EBAG_F32: return occupancy_fwd_f32(w, smem, n);
+        case EBAG_F16: return occupancy_fwd_f16(w, smem, n);
+        case EBAG_BF16: return occupancy_fwd_bf16(w, smem, n);
+        default: return occupancy_fwd_int8(w, smem, n);
+    }
+}
+
+// Checks shared by ebag_forward and ebag_forward_host (pointers may be host or device).
+ebag_status check_forward_args(ebag_tbe* h, const void* const* tables, const int32_t* D,
+                               const int64_t* indices, int64_t n_indices, const int64_t* offsets,
+                               const float* weights, int64_t B, ebag_mode mode, float* out) {
+    if (!h || !tables || !D || !offsets || B < 0 || n_indices < 0) return EBAG_ERR_INVALID_ARG;
+    if (mode != EBAG_SUM && mode != EBAG_MEAN) return EBAG_ERR_INVALID_ARG;
+    if (mode == EBAG_MEAN && weights) return EBAG_ERR_UNSUPPORTED;
+    if (n_indices > 0 && !indices) return EBAG_ERR_INVALID_ARG;
+    if (B > 0 && !out) return EBAG_ERR_INVALID_ARG;
+    if ((int64_t)h->T * B >= (1ll << 31)) return EBAG_ERR_UNSUPPORTED;
+    for (int t = 0; t < h->T; ++t) {
+        if (D[t] != h->D[t]) return EBAG_ERR_INVALID_ARG;
+        if (!tables[t] && h->rows[t] > 0) return EBAG_ERR_INVALID_ARG;
+        if ((uintptr_t)tables[t] & 15u) return EBAG_ERR_INVALID_ARG;
+    }
+    return EBAG_OK;
+}
+
+// Device copy of the caller's table-pointer array; re-sent only when it changed.
+ebag_status stage_tables(ebag_tbe* h, const void* const* tables, cudaStream_t stream,
+                         const void* const** d_out) {
+    const size_t bytes = (size_t)h->T * sizeof(void*);
+    if (h->slot >= 0 && std::memcmp(h->h_tables[h->slot], tables, bytes) == 0) {
+        *d_out = h->d_tables[h->slot];
+        return EBAG_OK;
+    }
+    const int s = (h->slot + 1) % kTableSlots;
+    if (h->slot_busy[s]) {   // an older launch may still read this slot's staging memory
+        EBAG_CUDA(h, cudaEventSynchronize(h->slot_event[s]));
+        h->slot_busy[s] = false;
+    }
+    std::memcpy(h->h_tables[s], tables, bytes);
+    EBAG_CUDA(h, cudaMemcpyAsync(h->d_tables[s], h->h_tables[s], bytes, cudaMemcpyHostToDevice, stream));
+    EBAG_CUDA(h, cudaEventRecord(h->slot_event[s], stream));
+    h->slot_busy[s] = true;
+    h->slot = s;
+    *d_out = h->d_tables[s];
+    return EBAG_OK;
+}
+
+// Launch on device pointers; arguments already checked.
+ebag_status forward_device(ebag_tbe* h, const void* const* tables, const int64_t* indices,
+                           int64_t n_indices, const int64_t* offsets, const float* weights,
+                           int64_t B, ebag_mode mode, float* out, cudaStream_t stream) {
+    if (B == 0) return EBAG_OK;
+    if (((uintptr_t)out & 15u) || ((uintptr_t)indices & 7u) || ((uintptr_t)offsets & 7u) ||
+        ((uintptr_t)weights & 3u))
+        return EBAG_ERR_INVALID_ARG;
+    const void* const* d_tables = nullptr;
+    ebag_status st = stage_tables(h, tables, stream, &d_tables);
+    if (st != EBAG_OK) return st;
+
+    FwdParams p;
+    p.tables = d_tables;
+    p.meta = h->d_meta;
+    p.indices = indices;
+    p.offsets = offsets;
+    p.weights = weights;
+    p.out = out;
+    p.queue = h->d_queue;
+    p.status = h->d_status;
+    p.n_indices = n_indices;
+    p.B = B;
+    p.T = h->T;
+    p.sumD = h->sumD;
+    p.mean = mode == EBAG_MEAN ? 1 : 0;
+    p.item_bytes = h->item_bytes;
+    const bool w = weights != nullptr;
+    int per_sm = h->occupancy[w ? 1 : 0];
+    if (h->ctas_per_sm > 0 && h->ctas_per_sm < per_sm) per_sm = h->ctas_per_sm;
+    const int grid = h->num_sms * per_sm;
+    EBAG_CUDA(h, launch_fwd(h->dtype, p, w, grid, fwd_smem_bytes(h->T), stream));
+    ++h->launches;
+    return EBAG_OK;
+}
+
+template <typename T>
+ebag_status grow(ebag_tbe* h, T** buf, int64_t* cap, int64_t need) {
+    if (need <= *cap) return EBAG_OK;
+    EBAG_CUDA(h, cudaDeviceSynchronize());
+    cudaFree(*buf);
+    *buf = nullptr;
+    *cap = 0;
+    EBAG_CUDA(h, cudaMalloc((void**)buf, (size_t)need * sizeof(T)));
+    *cap = need;
+    return EBAG_OK;
+}
+
+__global__ void pack_int8_rowwise_kernel(const int8_t* __restrict__ q, const float* __restrict__ scale,
+                                         const float* __restrict__ bias, int64_t rows, int D,
+                                         uint4* __restrict__ dst) {
+    // one thread per 16-byte vector of the packed row: D/16 vectors of codes, then one vector
+    // holding scale, bias and 8 bytes of zero padding
+    const int vecs = D / 16 + 1;
+    const int64_t total = rows * vecs;
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total;
+         i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t r = i / vecs;
+        const int v = (int)(i - r * vecs);
+        uint4 x;
+        if (v < vecs - 1) {
+            x = *reinterpret_cast<const uint4*>(q + r * D + v * 16);
+        } else {
+            x = make_uint4(__float_as_uint(scale[r]), __float_as_uint(bias[r]), 0u, 0u);
+        }
+        dst[i] = x;
+    }
+}
+
+}  // namespace
+
+extern "C" {
+
+int64_t ebag_row_stride(ebag_dtype dtype, int32_t D) {
+    if (D <= 0 || dtype < EBAG_F32 || dtype > EBAG_INT8_ROWWISE) return -1;
+    const int64_t payload = (int64_t)D * elem_bytes(dtype);
+    if (payload % 16 != 0) return -1;
+    return dtype == EBAG_INT8_ROWWISE ? payload + 16 : payload;
+}
+
+ebag_status ebag_create_tbe(int32_t T, const int64_t* rows, const int32_t* D, ebag_dtype dtype,
+                            int device, ebag_tbe** out) {
+    if (!out) return EBAG_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (T <= 0 || !rows || !D || dtype < EBAG_F32 || dtype > EBAG_INT8_ROWWISE)
+        return EBAG_ERR_INVALID_ARG;
+    if (T > EBAG_MAX_TABLES) return EBAG_ERR_UNSUPPORTED;
+    std::vector<TableMeta> meta(T);
+    int64_t d_off = 0;
+    for (int t = 0; t < T; ++t) {
+        const int64_t stride = ebag_row_stride(dtype, D[t]);
+        if (stride < 0 || rows[t] < 0) return EBAG_ERR_INVALID_ARG;
+        if (rows[t] >= (1ll << 31) || stride >= (1ll << 31)) return EBAG_ERR_UNSUPPORTED;
+        TableMeta& m = meta[t];
+        m.rows = rows[t];
+        m.D = D[t];
+        m.D_off = (int32_t)d_off;
+        m.stride = (int32_t)stride;
+        m.nvec = (int32_t)((int64_t)D[t] * elem_bytes(dtype) / 16);
+        int g_log2 = 2;
+        while ((1 << g_log2) < m.nvec && g_log2 < 5) ++g_log2;
+        m.g_log2 = g_log2;
+        const int per_lane = (m.nvec + 31) / 32;
+        m.V = per_lane <= 1 ? 1 : (per_lane == 2 ? 2 : 4);
+        d_off += D[t];
+        if (d_off >= (1ll << 31)) return EBAG_ERR_UNSUPPORTED;
+    }
+    int ndev = 0;
+    if (cudaGetDeviceCount(&ndev) != cudaSuccess || device < 0 || device >= ndev) {
+        cudaGetLastError();
+        return EBAG_ERR_CUDA;
+    }
+    DeviceGuard guard(device);
+    if (!guard.ok) return EBAG_ERR_CUDA;
+    ebag_tbe* h = new (std::nothrow) ebag_tbe;
+    if (!h) return EBAG_ERR_INVALID_ARG;
+    h->T = T;
+    h->dtype = dtype;
+    h->device = device;
+    h->sumD = (int)d_off;
+    h->rows.assign(rows, rows + T);
+    h->D.assign(D, D + T);
+    ebag_status st = EBAG_OK;
+    auto body = [&]() -> ebag_status {
+        cudaDeviceProp prop;
+        EBAG_CUDA(h, cudaGetDeviceProperties(&prop, device));
+        h->num_sms = prop.multiProcessorCount;
+        EBAG_CUDA(h, cudaMalloc((void**)&h->d_meta, sizeof(TableMeta) * T));
+        EBAG_CUDA(h, cudaMemcpy(h->d_meta, meta.data(), sizeof(TableMeta) * T, cudaMemcpyHostToDevice));
+        EBAG_CUDA(h, cudaMalloc((void**)&h->d_queue, sizeof(Queue)));
+        EBAG_CUDA(h, cudaMemset(h->d_queue, 0, sizeof(Queue)));
+        EBAG_CUDA(h, cudaMalloc((void**)&h->d_status, sizeof(Status)));
+        EBAG_CUDA(h, cudaMemset(h->d_status, 0, sizeof(Status)));
+        for (int i = 0; i < kTableSlots; ++i) {
+            EBAG_CUDA(h, cudaMalloc((void**)&h->d_tables[i], sizeof(void*) * T));
+            EBAG_CUDA(h, cudaMallocHost((void**)&h->h_tables[i], sizeof(void*) * T));
+            EBAG_CUDA(h, cudaEventCreateWithFlags(&h->slot_event[i], cudaEventDisableTiming));
+        }
+        for (int w = 0; w < 2; ++w) {
+            EBAG_CUDA(h, occupancy_fwd(dtype, w != 0, fwd_smem_bytes(T), &h->occupancy[w]));
+            if (h->occupancy[w] < 1) h->occupancy[w] = 1;
+        }
+        return EBAG_OK;
+    };
+    st = body();
+    if (st != EBAG_OK) {
+        free_handle(h);
+        return st;
+    }
+    *out = h;
+    return EBAG_OK;
+}
+
+ebag_status ebag_forward(ebag_tbe* h, const void* const* tables, const int32_t* D,
+                         const int64_t* indices, int64_t n_indices, const int64_t* offsets,
+                         const float* per_sample_weights, int64_t B, ebag_mode mode, float* out,
+                         ebag_stream stream) {
+    ebag_status st = check_forward_args(h, tables, D, indices, n_indices, offsets,
+                                        per_sample_weights, B, mode, out);
+    if (st != EBAG_OK) return st;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) return EBAG_ERR_CUDA;
+    return forward_device(h, tables, indices, n_indices, offsets, per_sample_weights, B, mode, out,
+                          (cudaStream_t)stream);
+}
+
+ebag_status ebag_forward_host(ebag_tbe* h, const void* const* tables, const int32_t* D,
+                              const int64_t* indices, int64_t n_indices, const int64_t* offsets,
+                              const float* per_sample_weights, int64_t B, ebag_mode mode,
+                              float* out, ebag_stream stream) {
+    ebag_status st = check_forward_args(h, tables, D, indices, n_indices, offsets,
+                                        per_sample_weights, B, mode, out);
+    if (st != EBAG_OK) return st;
+    if (B == 0) return EBAG_OK;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) return EBAG_ERR_CUDA;
+    cudaStream_t s = (cudaStream_t)stream;
+    const int64_t n_off = (int64_t)h->T * B + 1;
+    const int64_t n_out = B * (int64_t)h->sumD;
+    if ((st = grow(h, &h->s_indices, &h->cap_indices, n_indices > 0 ? n_indices : 1)) != EBAG_OK) return st;
+    if ((st = grow(h, &h->s_offsets, &h->cap_offsets, n_off)) != EBAG_OK) return st;
+    if (per_sample_weights &&
+        (st = grow(h, &h->s_weights, &h->cap_weights, n_indices > 0 ? n_indices : 1)) != EBAG_OK)
+        return st;
+    if ((st = grow(h, &h->s_out, &h->cap_out, n_out)) != EBAG_OK) return st;
+    if (n_indices > 0)
+        EBAG_CUDA(h, cudaMemcpyAsync(h->s_indices, indices, sizeof(int64_t) * n_indices, cudaMemcpyHostToDevice, s));
+    EBAG_CUDA(h, cudaMemcpyAsync(h->s_offsets, offsets, sizeof(int64_t) * n_off, cudaMemcpyHostToDevice, s));
+    if (per_sample_weights && n_indices > 0)
+        EBAG_CUDA(h, cudaMemcpyAsync(h->s_weights, per_sample_weights, sizeof(float) * n_indices, cudaMemcpyHostToDevice, s));
+    st = forward_device(h, tables, h->s_indices, n_indices, h->s_offsets,
+                        per_sample_weights ? h->s_weights : nullptr, B, mode, h->s_out, s);
+    if (st != EBAG_OK) return st;
+    EBAG_CUDA(h, cudaMemcpyAsync(out, h->s_out, sizeof(float) * n_out, cudaMemcpyDeviceToHost, s));
+    return EBAG_OK;
+}
+
+ebag_status ebag_last_status(ebag_tbe* h, ebag_stream stream, int64_t* n_oob, int64_t* n_bad_offsets) {
+    if (!h) return EBAG_ERR_INVALID_ARG;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) return EBAG_ERR_CUDA;
+    cudaStream_t s = (cudaStream_t)stream;
+    Status host;
+    EBAG_CUDA(h, cudaMemcpyAsync(&host, h->d_status, sizeof host, cudaMemcpyDeviceToHost, s));
+    EBAG_CUDA(h, cudaMemsetAsync(h->d_status, 0, sizeof(Status), s));
+    EBAG_CUDA(h, cudaStreamSynchronize(s));
+    if (n_oob) *n_oob = (int64_t)host.n_oob;
+    if (n_bad_offsets) *n_bad_offsets = (int64_t)host.n_bad_offsets;
+    if (host.n_bad_offsets) return EBAG_ERR_BAD_OFFSETS;
+    if (host.n_oob) return EBAG_ERR_INDEX_OOB;
+    return EBAG_OK;
+}
+
+ebag_status ebag_pack_int8_rowwise(const int8_t* q, const float* scale, const float* bias,
+                                   int64_t rows, int32_t D, void* dst, ebag_stream stream) {
+    if (rows < 0 || ebag_row_stride(EBAG_INT8_ROWWISE, D) < 0) return EBAG_ERR_INVALID_ARG;
+    if (rows == 0) return EBAG_OK;
+    if (!q || !scale || !bias || !dst) return EBAG_ERR_INVALID_ARG;
+    if (((uintptr_t)q & 15u) || ((uintptr_t)dst & 15u)) return EBAG_ERR_INVALID_ARG;
+    const int64_t total = rows * (D / 16 + 1);
+    int64_t blocks = (total + 255) / 256;
+    if (blocks > 148 * 32) blocks = 148 * 32;
+    pack_int8_rowwise_kernel<<<(int)blocks, 256, 0, (cudaStream_t)stream>>>(
+        q, scale, bias, rows, D, static_cast<uint4*>(dst));
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(nullptr, e);
+    return EBAG_OK;
+}
+
+ebag_status ebag_set_param(ebag_tbe* h, const char* name, int64_t value) {
+    if (!h || !name) return EBAG_ERR_INVALID_ARG;
+    if (std::strcmp(name, "item_bytes") == 0) {
+        if (value < 256 || value > (1ll << 30)) return EBAG_ERR_INVALID_ARG;
+        h->item_bytes = (uint32_t)value;
+        return EBAG_OK;
+    }
+    if (std::strcmp(name, "ctas_per_sm") == 0) {
+        if (value < 0 || value > 32) return EBAG_ERR_INVALID_ARG;
+        h->ctas_per_sm = (int)value;
+        return EBAG_OK;
+    }
+    return EBAG_ERR_INVALID_ARG;
+}
+
+int64_t ebag_launch_count(const ebag_tbe* h) { return h ? h->launches : 0; }
+
+const char* ebag_last_cuda_error(const ebag_tbe* h) { return h ? h->cuda_error.c_str() : ""; }
+
+void ebag_destroy(ebag_tbe* h) {
+    if (!h) return;
+    DeviceGuard guard(h->device);
+    cudaDeviceSynchronize();
+    free_handle(h);
+}
+
+const char* ebag_status_string(ebag_status s) {
+    switch (s) {
+        case EBAG_OK: return "ok";
+        case EBAG_ERR_INVALID_ARG: return "invalid argument";
+        case EBAG_ERR_UNSUPPORTED: return "unsupported";
+        case EBAG_ERR_CUDA: return "CUDA error";
+        case EBAG_ERR_INDEX_OOB: return "out-of-range ids were skipped";
+        case EBAG_ERR_BAD_OFFSETS: return "malformed bags were treated as empty";
+        default: return "unknown status";
+    }
+}
+
+}  // extern "C"

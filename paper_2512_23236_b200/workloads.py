@@ -11,9 +11,10 @@ data matched to production statistics (Appendix "1D Convolution", input generati
 the precedent for doing the same here.
 
 Recipe (identical for every workload; seed 0, one numpy PCG64 stream per workload keyed by
-SeedSequence([seed, workload number]); draw order: rows, D, per-table mean length, bag lengths,
-Zipf ranks / uniform ids, row permutation, weights; table values come from a torch generator
-keyed by (seed, workload number, table)):
+SeedSequence([seed, workload number, 0]) for the table shapes (rows, D, per-table mean length)
+and one per table keyed by [seed, workload number, 1, table] for its bag lengths, Zipf ranks /
+uniform ids, row permutation and weights, in that order; table values come from a torch
+generator keyed by (seed, workload number, table)):
 
   1  1 table 10,000 x 64 fp32 N(0,1); B=512; lengths integer-uniform on 0..20; uniform ids; sum
   2  1 table 1,000,000 x 128 fp16 N(0,1); B=16,384; Poisson(30); Zipf(1.05) ranks through a
@@ -147,16 +148,27 @@ def _draw_ids(rng, w: Workload, t: int, n: int) -> np.ndarray:
     return perm[ranks].astype(np.int64, copy=False)
 
 
+def _gen_table_jagged(w: Workload, t: int):
+    rng = np.random.default_rng(np.random.SeedSequence([w.seed, w.number, 1, t]))
+    lengths = _draw_lengths(rng, w, t)
+    n = int(lengths.sum())
+    ids = _draw_ids(rng, w, t, n)
+    weights = rng.random(n, dtype=np.float32) if w.weighted else None
+    return lengths, ids, weights
+
+
 def gen_jagged(w: Workload) -> Jagged:
-    """Bag lengths, offsets, ids and weights for all T tables (host, numpy, seeded)."""
-    rng = np.random.default_rng(np.random.SeedSequence([w.seed, w.number, 1]))
-    lengths = np.concatenate([_draw_lengths(rng, w, t) for t in range(w.T)])
+    """Bag lengths, offsets, ids and weights for all T tables (host, numpy, seeded; one
+    independent stream per table, drawn on a thread pool)."""
+    import concurrent.futures
+    import os
+    with concurrent.futures.ThreadPoolExecutor(max_workers=min(w.T, os.cpu_count() or 1)) as ex:
+        parts = list(ex.map(lambda t: _gen_table_jagged(w, t), range(w.T)))
+    lengths = np.concatenate([p[0] for p in parts])
     offsets = np.zeros(w.T * w.B + 1, dtype=np.int64)
     np.cumsum(lengths, out=offsets[1:])
-    n_t = [int(offsets[(t + 1) * w.B] - offsets[t * w.B]) for t in range(w.T)]
-    indices = np.concatenate([_draw_ids(rng, w, t, n_t[t]) for t in range(w.T)]) \
-        if sum(n_t) else np.zeros(0, dtype=np.int64)
-    weights = rng.random(indices.shape[0], dtype=np.float32) if w.weighted else None
+    indices = np.concatenate([p[1] for p in parts])
+    weights = np.concatenate([p[2] for p in parts]) if w.weighted else None
     return Jagged(indices, offsets, weights, lengths)
 
 

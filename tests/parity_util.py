@@ -1,0 +1,157 @@
+"""Shared helpers of the GPU parity tests: feed the same seeded inputs to the CUDA library (through
+its C ABI binding) and to the CPU oracle, and compare element by element.
+
+Tolerances (per element, S = sum |w*x| of that element's bag, divided by the bag length in mean
+mode; S comes from the oracle's fp64 side):
+    fp32 tables            |gpu - oracle| <= 1e-5 * S
+    fp16/bf16/int8 tables  |gpu - oracle| <= 2e-3 * S
+Elements with S == 0 (empty bags, all-zero terms) must be equal, and empty bags must be +0.0f
+bit for bit.
+"""
+import numpy as np
+import torch
+
+import paper_2512_23236_b200 as eb
+from oracle import ebag_oracle as orc
+from paper_2512_23236_b200 import workloads as wl
+
+TOL = {wl.F32: 1e-5, wl.F16: 2e-3, wl.BF16: 2e-3, wl.INT8_ROWWISE: 2e-3}
+
+
+def device_tables(dtype, tables):
+    """torch tables (any device) -> list of CUDA tensors in the library's layout."""
+    out = []
+    for t in tables:
+        if dtype == wl.INT8_ROWWISE:
+            q, s, b = (x.cuda() for x in t)
+            out.append(eb.ebag_pack_int8_rowwise(q, s, b))
+        else:
+            out.append(t.cuda().contiguous())
+    return out
+
+
+def oracle_tables(dtype, tables):
+    if dtype == wl.INT8_ROWWISE:
+        return ([wl.raw_numpy(t[0]) for t in tables], [wl.raw_numpy(t[1]) for t in tables],
+                [wl.raw_numpy(t[2]) for t in tables])
+    return [wl.raw_numpy(t) for t in tables], None, None
+
+
+def run_gpu(dtype, rows, D, dev_tables, indices, offsets, B, mode, weights=None, params=None,
+            host_path=False):
+    """Returns (out numpy [B, sumD], status tuple)."""
+    tbe = eb.TBE(rows, D, dtype, device=torch.cuda.current_device())
+    try:
+        for k, v in (params or {}).items():
+            tbe.set_param(k, v)
+        sumD = sum(D)
+        if host_path:
+            idx = torch.from_numpy(np.ascontiguousarray(indices)).pin_memory()
+            off = torch.from_numpy(np.ascontiguousarray(offsets)).pin_memory()
+            w = None if weights is None else torch.from_numpy(np.ascontiguousarray(weights)).pin_memory()
+            out = torch.full((B, sumD), float("nan"), dtype=torch.float32).pin_memory()
+            tbe.forward_host(dev_tables, idx, off, B, mode, w, out=out)
+            status = tbe.last_status()
+            return out.numpy().copy(), status
+        idx = torch.from_numpy(np.ascontiguousarray(indices)).cuda()
+        off = torch.from_numpy(np.ascontiguousarray(offsets)).cuda()
+        w = None if weights is None else torch.from_numpy(np.ascontiguousarray(weights)).cuda()
+        out = torch.full((B, sumD), float("nan"), dtype=torch.float32, device="cuda")
+        tbe.forward(dev_tables, idx, off, B, mode, w, out=out)
+        status = tbe.last_status()
+        return out.cpu().numpy(), status
+    finally:
+        tbe.close()
+
+
+def compare(gpu, ref, dtype, lengths=None, T=None, B=None, D=None):
+    """Assert the parity bar; returns max(|gpu - out32| / S) over elements with S > 0."""
+    out32, S = ref["out32"], ref["S"]
+    assert gpu.shape == out32.shape
+    assert not np.isnan(gpu).any(), "an output element was never written"
+    tol = TOL[dtype]
+    err = np.abs(gpu.astype(np.float64) - out32.astype(np.float64))
+    bad = err > tol * S
+    if bad.any():
+        i = np.argwhere(bad)[0]
+        raise AssertionError(f"{bad.sum()} elements beyond {tol}*S; first at {tuple(i)}: "
+                             f"gpu={gpu[tuple(i)]} oracle={out32[tuple(i)]} S={S[tuple(i)]}")
+    if lengths is not None:
+        col = 0
+        for t in range(T):
+            empty = lengths[t * B:(t + 1) * B] == 0
+            blk = np.ascontiguousarray(gpu[:, col:col + D[t]][empty])
+            assert np.all(blk.view(np.uint32) == 0), "an empty bag is not +0.0f"
+            col += D[t]
+    pos = S > 0
+    return float((err[pos] / S[pos]).max()) if pos.any() else 0.0
+
+
+def check_workload(w, jag=None, tables=None, params=None, host_path=False):
+    """Element-by-element parity of a (small enough) workload.  Returns the max relative error."""
+    jag = jag or wl.gen_jagged(w)
+    tables = tables or wl.gen_tables(w, "cpu")
+    dev = device_tables(w.dtype, tables)
+    gpu, status = run_gpu(w.dtype, w.rows, w.D, dev, jag.indices, jag.offsets, w.B, w.mode,
+                          jag.weights, params, host_path)
+    tabs, sc, bi = oracle_tables(w.dtype, tables)
+    ref = orc.forward(tabs, w.dtype, jag.indices, jag.offsets, w.B, w.mode, weights=jag.weights,
+                      scales=sc, biases=bi)
+    assert status == (eb.EBAG_OK, ref["n_oob"], ref["n_bad_offsets"]) == (0, 0, 0)
+    return compare(gpu, ref, w.dtype, jag.lengths, w.T, w.B, w.D)
+
+
+def sampled_check(w, jag, dev_tables_raw, gpu_out, bags_per_table, seed=0):
+    """Parity at full size on sampled bags: for every table pick ``bags_per_table`` bags (the
+    longest, an empty one if there is one, the first, the last, the rest at random), copy only the
+    rows they reference to the host, renumber, and run the oracle on that compact problem.
+
+    dev_tables_raw: per table the UNPACKED device tensors (for int8 the (q, scale, bias) tuple).
+    gpu_out: device tensor [B, sumD] produced by the library for the full workload."""
+    rng = np.random.default_rng(seed)
+    K = bags_per_table
+    sel_bags, c_tables, c_sc, c_bi = [], [], [], []
+    c_idx, c_w = [], []
+    c_len = []
+    for t in range(w.T):
+        lens = jag.lengths[t * w.B:(t + 1) * w.B]
+        picks = {0, w.B - 1, int(np.argmax(lens))}
+        if (lens == 0).any():
+            picks.add(int(np.argmax(lens == 0)))
+        while len(picks) < min(K, w.B):
+            picks.add(int(rng.integers(0, w.B)))
+        picks = np.array(sorted(picks))[:K]
+        sel_bags.append(picks)
+        segs = [jag.indices[jag.offsets[t * w.B + b]:jag.offsets[t * w.B + b + 1]] for b in picks]
+        flat = np.concatenate(segs) if segs else np.zeros(0, np.int64)
+        uniq, inv = np.unique(flat, return_inverse=True)
+        if uniq.size == 0:
+            uniq = np.zeros(1, np.int64)
+        sel = torch.from_numpy(uniq).cuda()
+        tab = dev_tables_raw[t]
+        if w.dtype == wl.INT8_ROWWISE:
+            c_tables.append(wl.raw_numpy(tab[0].index_select(0, sel)))
+            c_sc.append(wl.raw_numpy(tab[1].index_select(0, sel)))
+            c_bi.append(wl.raw_numpy(tab[2].index_select(0, sel)))
+        else:
+            c_tables.append(wl.raw_numpy(tab.index_select(0, sel)))
+        c_idx.append(inv.astype(np.int64))
+        c_len.append(np.array([s.size for s in segs], dtype=np.int64))
+        if jag.weights is not None:
+            c_w.append(np.concatenate(
+                [jag.weights[jag.offsets[t * w.B + b]:jag.offsets[t * w.B + b + 1]] for b in picks]))
+    Ks = len(sel_bags[0])
+    lengths = np.concatenate(c_len)
+    offsets = np.zeros(w.T * Ks + 1, dtype=np.int64)
+    np.cumsum(lengths, out=offsets[1:])
+    ref = orc.forward(c_tables, w.dtype, np.concatenate(c_idx), offsets, Ks, w.mode,
+                      weights=np.concatenate(c_w) if c_w else None,
+                      scales=c_sc or None, biases=c_bi or None)
+    assert ref["n_oob"] == 0 and ref["n_bad_offsets"] == 0
+    gpu = np.empty((Ks, w.sumD), dtype=np.float32)
+    col = 0
+    for t in range(w.T):
+        rows_sel = torch.from_numpy(sel_bags[t]).cuda()
+        gpu[:, col:col + w.D[t]] = gpu_out.index_select(0, rows_sel)[:, col:col + w.D[t]].cpu().numpy()
+        col += w.D[t]
+    return compare(gpu, ref, w.dtype, lengths, w.T, Ks, w.D)

@@ -1,0 +1,258 @@
+"""GPU parity: the CUDA library (through its C ABI) against the CPU oracle on the same seeded
+inputs.  All tests here need a B200."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2512_23236_b200 as eb
+from oracle import ebag_oracle as orc
+from paper_2512_23236_b200 import workloads as wl
+
+import parity_util as pu
+
+pytestmark = pytest.mark.gpu
+
+
+def _jagged_from_lengths(rng, lengths_per_table, rows):
+    T = len(lengths_per_table)
+    B = len(lengths_per_table[0])
+    lengths = np.concatenate([np.asarray(l, dtype=np.int64) for l in lengths_per_table])
+    offsets = np.zeros(T * B + 1, dtype=np.int64)
+    np.cumsum(lengths, out=offsets[1:])
+    idx = np.concatenate([rng.integers(0, rows[t], size=int(np.sum(lengths_per_table[t])))
+                          for t in range(T)]).astype(np.int64)
+    return idx, offsets, lengths
+
+
+def _rand_tables(rng, dtype, rows, D, small_ints=False):
+    tabs = []
+    for r, d in zip(rows, D):
+        if dtype == wl.INT8_ROWWISE:
+            q = torch.from_numpy(rng.integers(-128, 128, size=(r, d)).astype(np.int8))
+            if small_ints:
+                s, b = torch.ones(r), torch.zeros(r)
+            else:
+                s = torch.from_numpy(rng.uniform(0.01, 0.03, r).astype(np.float32))
+                b = torch.from_numpy(rng.normal(0, 0.1, r).astype(np.float32))
+            tabs.append((q, s, b))
+        else:
+            x = rng.integers(-8, 9, size=(r, d)).astype(np.float32) if small_ints \
+                else rng.standard_normal((r, d)).astype(np.float32)
+            tabs.append(torch.from_numpy(x).to({wl.F32: torch.float32, wl.F16: torch.float16,
+                                                wl.BF16: torch.bfloat16}[dtype]))
+    return tabs
+
+
+def _both(dtype, rows, D, tabs, idx, off, B, mode, w=None, params=None, host_path=False):
+    dev = pu.device_tables(dtype, tabs)
+    gpu, status = pu.run_gpu(dtype, rows, D, dev, idx, off, B, mode, w, params, host_path)
+    ot, sc, bi = pu.oracle_tables(dtype, tabs)
+    ref = orc.forward(ot, dtype, idx, off, B, mode, weights=w, scales=sc, biases=bi)
+    return gpu, status, ref
+
+
+# ------------------------------------------------------------------ the five published workloads
+def test_cfg1_full_size():
+    pu.check_workload(wl.make_workload(1))
+
+
+def test_cfg2_full_size():
+    pu.check_workload(wl.make_workload(2))
+
+
+@pytest.mark.parametrize("number,kw", [
+    (3, dict(scale_rows=0.01, scale_B=1 / 64)),
+    (4, dict(scale_rows=0.01, scale_B=1 / 32)),
+    (5, dict(scale_rows=0.01, scale_B=1 / 64)),
+])
+def test_cfg345_scaled_down_elementwise(number, kw):
+    pu.check_workload(wl.make_workload(number, **kw))
+
+
+@pytest.mark.parametrize("item_bytes,ctas", [(256, 1), (4096, 0), (1 << 20, 2)])
+def test_work_partition_settings_do_not_change_results(item_bytes, ctas):
+    w = wl.make_workload(3, scale_rows=0.005, scale_B=1 / 128, max_tables=8)
+    pu.check_workload(w, params=dict(item_bytes=item_bytes, ctas_per_sm=ctas))
+
+
+def test_host_buffer_entry_point():
+    pu.check_workload(wl.make_workload(4, scale_rows=0.002, scale_B=1 / 64, max_tables=3),
+                      host_path=True)
+    pu.check_workload(wl.make_workload(2, scale_rows=0.05, scale_B=1 / 8), host_path=True)
+
+
+# ------------------------------------------------------------------ shapes: every row-group path
+@pytest.mark.parametrize("dtype,Ds", [
+    (wl.F32, [4, 8, 12, 36, 64, 100, 132, 256, 260, 520, 1028]),
+    (wl.F16, [8, 24, 64, 128, 264, 520, 1032]),
+    (wl.BF16, [8, 16, 72, 256, 512, 1032, 2056]),
+    (wl.INT8_ROWWISE, [16, 48, 128, 512, 528, 1040, 2064]),
+])
+@pytest.mark.parametrize("mode,weighted", [(wl.SUM, False), (wl.MEAN, False), (wl.SUM, True)])
+def test_all_row_widths(dtype, Ds, mode, weighted):
+    rng = np.random.default_rng(42 + dtype)
+    T, B = len(Ds), 77                      # ragged tail: 77 is not a multiple of any item size
+    rows = [int(rng.integers(5, 400)) for _ in Ds]
+    lens = [rng.integers(0, 40, size=B) for _ in Ds]
+    for l in lens:
+        l[rng.random(B) < 0.15] = 0
+    idx, off, lengths = _jagged_from_lengths(rng, lens, rows)
+    w = (rng.random(idx.shape[0]).astype(np.float32) - 0.25) if weighted else None
+    tabs = _rand_tables(rng, dtype, rows, Ds)
+    gpu, status, ref = _both(dtype, rows, Ds, tabs, idx, off, B, mode, w)
+    assert status == (0, 0, 0)
+    pu.compare(gpu, ref, dtype, lengths, T, B, Ds)
+
+
+# ------------------------------------------------------------------ degenerate and extreme bags
+@pytest.mark.parametrize("dtype,D", [(wl.F32, 256), (wl.BF16, 64), (wl.INT8_ROWWISE, 128)])
+def test_planted_bag_lengths(dtype, D):
+    rng = np.random.default_rng(5)
+    lens = [[0, 1, 1023, 1024, 0, 0, 7, 5000, 31, 32, 33, 255, 256, 257, 1, 0, 8, 9, 15, 16, 17]]
+    rows = [3000]
+    idx, off, lengths = _jagged_from_lengths(rng, lens, rows)
+    B = len(lens[0])
+    w = rng.random(idx.shape[0]).astype(np.float32)
+    tabs = _rand_tables(rng, dtype, rows, [D])
+    for mode, ww in ((wl.SUM, None), (wl.MEAN, None), (wl.SUM, w)):
+        gpu, status, ref = _both(dtype, rows, [D], tabs, idx, off, B, mode, ww)
+        assert status == (0, 0, 0)
+        pu.compare(gpu, ref, dtype, lengths, 1, B, [D])
+
+
+def test_empty_inputs():
+    rng = np.random.default_rng(6)
+    rows, D = [50, 60], [16, 32]
+    tabs = _rand_tables(rng, wl.F32, rows, D)
+    dev = pu.device_tables(wl.F32, tabs)
+    # B == 0: nothing to do, nothing launched
+    gpu, status = pu.run_gpu(wl.F32, rows, D, dev, np.zeros(0, np.int64), np.zeros(1, np.int64), 0, wl.SUM)
+    assert gpu.shape == (0, 48) and status == (0, 0, 0)
+    # all bags empty, no lookups at all
+    B = 100
+    gpu, status = pu.run_gpu(wl.F32, rows, D, dev, np.zeros(0, np.int64),
+                             np.zeros(2 * B + 1, np.int64), B, wl.MEAN)
+    assert status == (0, 0, 0) and np.all(gpu.view(np.uint32) == 0)
+    # a table with zero lookups next to one with some
+    lens = [np.zeros(B, np.int64), rng.integers(0, 5, size=B)]
+    idx, off, lengths = _jagged_from_lengths(rng, lens, rows)
+    gpu, status, ref = _both(wl.F32, rows, D, tabs, idx, off, B, wl.SUM)
+    pu.compare(gpu, ref, wl.F32, lengths, 2, B, D)
+
+
+def test_single_bag_single_lookup():
+    tabs = [torch.arange(32, dtype=torch.float32).reshape(4, 8)]
+    gpu, status, ref = _both(wl.F32, [4], [8], tabs, np.array([2], np.int64),
+                             np.array([0, 1], np.int64), 1, wl.SUM)
+    assert np.array_equal(gpu, np.arange(16, 24, dtype=np.float32)[None, :])
+
+
+# ------------------------------------------------------------------ integer-exact cases, bit for bit
+@pytest.mark.parametrize("dtype", [wl.F32, wl.F16, wl.BF16, wl.INT8_ROWWISE])
+def test_integer_valued_tables_match_bit_for_bit(dtype):
+    """Products and partial sums are integers below 2^24, so every summation order gives the same
+    fp32 result: the GPU must equal the oracle exactly."""
+    rng = np.random.default_rng(7)
+    rows, D = [300, 40, 1000], [16, 64, 128]
+    B = 200
+    lens = [rng.integers(0, 60, size=B) for _ in rows]
+    idx, off, lengths = _jagged_from_lengths(rng, lens, rows)
+    tabs = _rand_tables(rng, dtype, rows, D, small_ints=True)
+    w = rng.integers(-3, 4, size=idx.shape[0]).astype(np.float32)
+    for ww in (None, w):
+        gpu, status, ref = _both(dtype, rows, D, tabs, idx, off, B, wl.SUM, ww)
+        assert status == (0, 0, 0)
+        assert np.array_equal(gpu.view(np.uint32), ref["out32"].view(np.uint32))
+
+
+def test_one_hot_table_counts():
+    rng = np.random.default_rng(8)
+    rows, B = 64, 300
+    lens = [rng.integers(0, 50, size=B)]
+    idx, off, lengths = _jagged_from_lengths(rng, lens, [rows])
+    tabs = [torch.eye(rows, dtype=torch.float32)]
+    gpu, status, ref = _both(wl.F32, [rows], [rows], tabs, idx, off, B, wl.SUM)
+    want = np.zeros((B, rows), np.float32)
+    for b in range(B):
+        np.add.at(want[b], idx[off[b]:off[b + 1]], 1.0)
+    assert np.array_equal(gpu, want) and np.array_equal(ref["out32"], want)
+
+
+# ------------------------------------------------------------------ malformed inputs never fault
+def test_out_of_range_ids_skipped_and_counted():
+    rng = np.random.default_rng(9)
+    rows, D, B = [100, 30], [32, 8], 64
+    lens = [rng.integers(1, 20, size=B) for _ in rows]
+    idx, off, lengths = _jagged_from_lengths(rng, lens, rows)
+    bad = idx.copy()
+    planted = rng.choice(idx.shape[0], size=25, replace=False)
+    bad[planted[:8]] = -1
+    bad[planted[8:16]] = 2 ** 40
+    bad[planted[16:]] = 100          # == rows[0]; in range for nothing, out of range for both tables
+    tabs = _rand_tables(rng, wl.F32, rows, D)
+    for mode in (wl.SUM, wl.MEAN):
+        gpu, status, ref = _both(wl.F32, rows, D, tabs, bad, off, B, mode)
+        assert ref["n_oob"] == 25
+        assert status == (eb.EBAG_ERR_INDEX_OOB, 25, 0)
+        pu.compare(gpu, ref, wl.F32, lengths, 2, B, D)
+
+
+def test_bad_offsets_treated_as_empty_and_counted():
+    rng = np.random.default_rng(10)
+    rows, D, B = [100], [16], 40
+    lens = [rng.integers(1, 10, size=B)]
+    idx, off, lengths = _jagged_from_lengths(rng, lens, rows)
+    bad = off.copy()
+    bad[10] = bad[9] - 1 if bad[9] > 0 else 0       # bag 9 runs backwards, bag 10 grows
+    bad[-1] = idx.shape[0] + 5                      # last bag reaches past the id list
+    tabs = _rand_tables(rng, wl.F32, rows, D)
+    gpu, status, ref = _both(wl.F32, rows, D, tabs, idx, bad, B, wl.SUM)
+    assert ref["n_bad_offsets"] >= 2
+    assert status == (eb.EBAG_ERR_BAD_OFFSETS, ref["n_oob"], ref["n_bad_offsets"])
+    pu.compare(gpu, ref, wl.F32)
+
+
+def test_host_side_argument_errors():
+    tbe = eb.TBE([10], [16], eb.EBAG_F32, device=torch.cuda.current_device())
+    tab = torch.zeros(10, 16, device="cuda")
+    idx = torch.zeros(4, dtype=torch.int64, device="cuda")
+    off = torch.tensor([0, 4], dtype=torch.int64, device="cuda")
+    w = torch.ones(4, device="cuda")
+    with pytest.raises(eb.EbagError) as e:
+        tbe.forward([tab], idx, off, 1, eb.EBAG_MEAN, w)
+    assert e.value.status == eb.EBAG_ERR_UNSUPPORTED
+    with pytest.raises(eb.EbagError) as e:
+        eb.ebag_forward(tbe._h, [tab.data_ptr()], [32], idx.data_ptr(), 4, off.data_ptr(), None, 1, 0,
+                        tab.data_ptr(), 0)
+    assert e.value.status == eb.EBAG_ERR_INVALID_ARG          # D differs from create time
+    with pytest.raises(eb.EbagError):
+        eb.ebag_forward(tbe._h, [tab.data_ptr() + 4], [16], idx.data_ptr(), 4, off.data_ptr(), None,
+                        1, 0, tab.data_ptr(), 0)              # misaligned table
+    assert tbe.launch_count() == 0
+    out = tbe.forward([tab], idx, off, 1)
+    assert tbe.launch_count() == 1 and tbe.last_status() == (0, 0, 0)
+    tbe.close()
+    with pytest.raises(eb.EbagError):
+        eb.TBE([10], [6], eb.EBAG_F32)                        # 24-byte rows
+
+
+def test_repeated_calls_and_changing_table_pointers():
+    """The work queue re-arms itself after every launch, and a new table-pointer array is picked
+    up even when many different arrays are in flight."""
+    rng = np.random.default_rng(11)
+    rows, D, B = [200, 300], [64, 32], 128
+    lens = [rng.integers(0, 30, size=B) for _ in rows]
+    idx, off, lengths = _jagged_from_lengths(rng, lens, rows)
+    tbe = eb.TBE(rows, D, eb.EBAG_F32, device=torch.cuda.current_device())
+    didx, doff = torch.from_numpy(idx).cuda(), torch.from_numpy(off).cuda()
+    outs, refs = [], []
+    for k in range(10):
+        tabs = _rand_tables(rng, wl.F32, rows, D)
+        dev = pu.device_tables(wl.F32, tabs)
+        outs.append((tbe.forward(dev, didx, doff, B), dev))
+        ot, _, _ = pu.oracle_tables(wl.F32, tabs)
+        refs.append(orc.forward(ot, wl.F32, idx, off, B, wl.SUM))
+    assert tbe.last_status() == (0, 0, 0) and tbe.launch_count() == 10
+    for (o, _), r in zip(outs, refs):
+        pu.compare(o.cpu().numpy(), r, wl.F32, lengths, 2, B, D)
+    tbe.close()
