@@ -1,0 +1,293 @@
+#!/usr/bin/env python
+"""Benchmark of the pooled embedding-bag forward on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 1..5] [--impl reference]
+
+One step = one pass of the whole hot path (one ebag_forward launch over all tables of the
+workload).  Default workload: 3, the batched 32-table bf16 TBE (the largest batched-table
+configuration the metric is quoted on).  Prints ONE JSON line:
+
+  value     pooled lookups/s, whole job, inputs resident in HBM, CUDA-event time of K steps
+  e2e       the same through ebag_forward_host: pinned host ids/offsets/weights in, pinned host
+            output back, copies inside the timed region
+  roofline  the forward kernel against the measured HBM copy bandwidth (algorithmic bytes)
+  cpu_baseline  the CPU oracle, as it stands, on a bounded sample of the same workload
+
+With N > 1 (launched by torchrun) every rank owns its own tables and batch (independent units,
+no exchange step): weak scaling, value = lookups of all ranks / slowest rank's time.
+
+--impl reference times the CPU oracle on the machine's host cores (rank 0 only); each step is the
+bounded sample.
+"""
+import argparse
+import json
+import os
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+import torch  # noqa: E402
+
+from paper_2512_23236_b200 import benchlib as bl  # noqa: E402
+from paper_2512_23236_b200 import workloads as wl  # noqa: E402
+
+METRIC = "pooled_lookups_per_sec"
+UNIT = "lookups/s"
+L2_FLUSH_BYTES = 256 << 20
+
+# DRAM bytes per forward launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu
+# capture summarised under profiles/; None where no capture of that workload exists.
+NCU_DRAM_BYTES_PER_LAUNCH = {}
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--e2e-steps", type=int, default=0, help="0: min(steps, 10)")
+    ap.add_argument("--cpu-seconds", type=float, default=15.0)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--item-bytes", type=int, default=0)
+    ap.add_argument("--ctas-per-sm", type=int, default=0)
+    # shrunk variants of a workload, for profiler captures and quick checks (not bench lines)
+    ap.add_argument("--max-tables", type=int, default=0)
+    ap.add_argument("--scale-rows", type=float, default=1.0)
+    ap.add_argument("--scale-b", type=float, default=1.0)
+    return ap.parse_args()
+
+
+def make_workload(args, seed):
+    return wl.make_workload(args.workload, scale_rows=args.scale_rows, scale_B=args.scale_b,
+                            max_tables=args.max_tables or None, seed=seed)
+
+
+def workload_config(w, ab, args=None):
+    shrunk = args is not None and (args.max_tables or args.scale_rows != 1.0 or args.scale_b != 1.0)
+    return {"workload": w.name + ("_SHRUNK" if shrunk else ""), "tables": w.T, "bags_per_table": w.B, "sum_D": w.sumD,
+            "table_dtype": wl.DTYPE_NAMES[w.dtype],
+            "pooling": "mean" if w.mode == wl.MEAN else ("weighted_sum" if w.weighted else "sum"),
+            "lookups_per_step": ab["lookups"], "algorithmic_bytes_per_step": ab["total"],
+            "index_dtype": "int64", "seed": w.seed,
+            "l2": f"{L2_FLUSH_BYTES >> 20} MiB written between timed steps (L2 flush)"}
+
+
+def oracle_inputs(w, jag, host_table, max_lookups):
+    """Host arrays of the bounded CPU sample.  host_table(t) returns table t as host tensors."""
+    k, idx, off, wts, nb, n = bl.cpu_sample(w, jag, max_lookups)
+    tabs, sc, bi = [], [], []
+    for t in range(k):
+        tab = host_table(t)
+        if w.dtype == wl.INT8_ROWWISE:
+            tabs.append(wl.raw_numpy(tab[0]))
+            sc.append(wl.raw_numpy(tab[1]))
+            bi.append(wl.raw_numpy(tab[2]))
+        else:
+            tabs.append(wl.raw_numpy(tab))
+    return dict(tables=tabs, scales=sc or None, biases=bi or None, indices=idx, offsets=off,
+                weights=wts, B=nb, lookups=n, n_tables=k, rows=w.rows[:k], D=w.D[:k])
+
+
+def time_oracle(w, inp):
+    from oracle import ebag_oracle as orc
+    t0 = time.perf_counter()
+    orc.forward(inp["tables"], w.dtype, inp["indices"], inp["offsets"], inp["B"], w.mode,
+                weights=inp["weights"], scales=inp["scales"], biases=inp["biases"], want64=True)
+    return time.perf_counter() - t0
+
+
+def sized_cpu_sample(w, jag, host_table, seconds):
+    """Pick the sample size from a short probe so that one oracle pass takes about `seconds`
+    (the whole workload if that is less work)."""
+    from oracle import ebag_oracle as orc
+    probe = oracle_inputs(w, jag, host_table, 200_000)
+    t = max(time_oracle(w, probe), 1e-4)
+    rate = probe["lookups"] / t
+    inp = oracle_inputs(w, jag, host_table, int(rate * seconds))
+    whole = inp["lookups"] == int(jag.indices.shape[0])
+    desc = (("the whole workload: " if whole else "") +
+            f"the first {inp['n_tables']} of {w.T} tables, {inp['B']} bags each, "
+            f"{inp['lookups']} of {int(jag.indices.shape[0])} lookups, "
+            f"all {orc.max_threads()} host threads")
+    return inp, desc, orc.max_threads()
+
+
+def run_reference(args, rank):
+    """The CPU oracle as the reference arm (rank 0 only)."""
+    if rank != 0:
+        return
+    w = make_workload(args, 0)
+    jag = wl.gen_jagged(w)
+    ab = wl.algorithmic_bytes(w, jag.lengths)
+    cache = {}
+
+    def host_table(t):
+        if t not in cache:
+            cache[t] = wl.gen_table(w, t, "cpu")
+        return cache[t]
+
+    # a step must stay short enough for warmup + steps to end within a few minutes
+    per_step = max(0.5, min(args.cpu_seconds, 120.0 / max(1, args.steps + args.warmup)))
+    inp, desc, cores = sized_cpu_sample(w, jag, host_table, per_step)
+    for _ in range(args.warmup):
+        time_oracle(w, inp)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        time_oracle(w, inp)
+    dt = time.perf_counter() - t0
+    value = inp["lookups"] * args.steps / dt
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32", "data": "synthetic", "config": workload_config(w, ab, args),
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+                             "sample": desc},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    args = parse_args()
+    rank, local_rank, world = bl.rank_info()
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    import paper_2512_23236_b200 as eb
+    eb.lib()                                   # fail loudly if the CUDA library is missing
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    dist = bl.init_process_group("nccl")
+    warmup = max(3, args.warmup)
+
+    # ---------------- inputs: seeded, synthetic; every rank owns its own tables and batch
+    w = make_workload(args, bl.rank_seed(0, rank))
+    jag = wl.gen_jagged(w)
+    ab = wl.algorithmic_bytes(w, jag.lengths)
+    raw_tables = [wl.gen_table(w, t, dev) for t in range(w.T)]
+    if w.dtype == wl.INT8_ROWWISE:
+        tables = [eb.ebag_pack_int8_rowwise(q, s, b) for q, s, b in raw_tables]
+    else:
+        tables = raw_tables
+
+    def host_table(t):
+        x = raw_tables[t]
+        return tuple(y.cpu() for y in x) if isinstance(x, tuple) else x.cpu()
+
+    h_idx = torch.from_numpy(jag.indices).pin_memory()
+    h_off = torch.from_numpy(jag.offsets).pin_memory()
+    h_w = None if jag.weights is None else torch.from_numpy(jag.weights).pin_memory()
+    d_idx, d_off = h_idx.to(dev), h_off.to(dev)
+    d_w = None if h_w is None else h_w.to(dev)
+    d_out = torch.empty((w.B, w.sumD), dtype=torch.float32, device=dev)
+    h_out = torch.empty((w.B, w.sumD), dtype=torch.float32).pin_memory()
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
+
+    tbe = eb.TBE(w.rows, w.D, w.dtype, device=local_rank)
+    if args.item_bytes:
+        tbe.set_param("item_bytes", args.item_bytes)
+    if args.ctas_per_sm:
+        tbe.set_param("ctas_per_sm", args.ctas_per_sm)
+    stream = torch.cuda.Stream(device=dev)
+
+    def step():
+        tbe.forward(tables, d_idx, d_off, w.B, w.mode, d_w, out=d_out, stream=stream)
+
+    def step_host():
+        tbe.forward_host(tables, h_idx, h_off, w.B, w.mode, h_w, out=h_out, stream=stream)
+
+    torch.cuda.synchronize()
+    sampler = bl.ClockSampler(f"GPU-{torch.cuda.get_device_properties(dev).uuid}").start()
+    with torch.cuda.stream(stream):
+        for _ in range(warmup):
+            flush.fill_(1)
+            step()
+        stream.synchronize()
+        assert tbe.last_status(stream) == (0, 0, 0)
+
+        # ---------------- device-resident timing: K steps, CUDA events on the launching stream
+        bl.barrier()
+        torch.cuda.synchronize()
+        launches0 = tbe.launch_count()
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+              for _ in range(args.steps)]
+        for a, b in ev:
+            flush.fill_(1)                     # outside the event pair
+            a.record(stream)
+            step()
+            b.record(stream)
+        torch.cuda.synchronize()
+        bl.barrier()
+        launches = tbe.launch_count() - launches0
+        step_ms = [a.elapsed_time(b) for a, b in ev]
+        elapsed_ms = float(sum(step_ms))
+
+        # ---------------- end to end: host buffers in, host result out, copies timed
+        e2e_steps = args.e2e_steps or min(args.steps, 10)
+        for _ in range(2):
+            step_host()
+        stream.synchronize()
+        bl.barrier()
+        torch.cuda.synchronize()
+        ev2 = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+               for _ in range(e2e_steps)]
+        for a, b in ev2:
+            a.record(stream)
+            step_host()
+            b.record(stream)
+        torch.cuda.synchronize()
+        bl.barrier()
+        e2e_ms = float(sum(a.elapsed_time(b) for a, b in ev2))
+    clocks = sampler.stop()
+    assert tbe.last_status(stream) == (0, 0, 0)
+    assert torch.equal(h_out, d_out.cpu()), "host-buffer path and device path disagree"
+
+    total_lookups, max_ms = bl.reduce_job(ab["lookups"] * args.steps, elapsed_ms, dev)
+    e2e_lookups, e2e_max_ms = bl.reduce_job(ab["lookups"] * e2e_steps, e2e_ms, dev)
+    if rank != 0:
+        tbe.close()
+        return
+
+    peaks = bl.measured_peaks(ROOT)
+    ms_per_launch = elapsed_ms / max(1, launches)
+    achieved = ab["total"] / (ms_per_launch * 1e-3) / 1e9
+    line = {
+        "metric": METRIC, "value": total_lookups / (max_ms * 1e-3), "unit": UNIT, "n_gpus": world,
+        "steps": args.steps, "warmup": warmup, "ms_per_step": max_ms / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic", "config": workload_config(w, ab, args),
+        "clocks": clocks, "gpu_launches": launches,
+        "e2e": {"value": e2e_lookups / (e2e_max_ms * 1e-3), "unit": UNIT,
+                "h2d_bytes_per_step": ab["indices"] + ab["offsets"] + ab["weights"],
+                "d2h_bytes_per_step": ab["out"], "steps": e2e_steps,
+                "ms_per_step": e2e_max_ms / e2e_steps},
+        "roofline": {"bound": "hbm", "kernel": "ebag_fwd_kernel", "achieved": achieved,
+                     "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
+                     "peak_source": f"{peaks['source']} HBM copy bandwidth (burst)",
+                     "frac_of_nominal_8TBs": achieved / 8000.0,
+                     "algorithmic_bytes_per_launch": ab["total"],
+                     "ms_per_launch": ms_per_launch, "ms_per_launch_min": min(step_ms),
+                     "traffic": NCU_DRAM_BYTES_PER_LAUNCH.get(w.number)},
+        "bags_per_sec": w.T * w.B * world * args.steps / (max_ms * 1e-3),
+    }
+    if world == 1 and not args.no_cpu_baseline:
+        inp, desc, cores = sized_cpu_sample(w, jag, host_table, args.cpu_seconds)
+        dt = time_oracle(w, inp)
+        line["cpu_baseline"] = {"value": inp["lookups"] / dt, "unit": UNIT, "cores": cores,
+                                "kind": "oracle", "sample": desc, "seconds": dt}
+    else:
+        line["cpu_baseline"] = None
+    tbe.close()
+    print(json.dumps(line), flush=True)
+
+
+if __name__ == "__main__":
+    main()
