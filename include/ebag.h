@@ -58,8 +58,9 @@ typedef enum { EBAG_SUM = 0, EBAG_MEAN = 1 } ebag_mode;
 
 /*
  * Bytes from one stored row to the next.  F32/F16/BF16: D * element size.  INT8_ROWWISE: the
- * packed row [D int8 codes][fp32 scale][fp32 bias][8 bytes pad] = D + 16 (one gather fetches
- * codes and dequantisation constants together).  Returns -1 if D is not allowed for the dtype:
+ * packed row [D codes, each stored as q + 128 in one byte][fp32 scale][fp32 bias][8 bytes pad]
+ * = D + 16 (one gather fetches codes and dequantisation constants together; build it with
+ * ebag_pack_int8_rowwise).  Returns -1 if D is not allowed for the dtype:
  * D > 0 and D * element size must be a multiple of 16 bytes (D%4==0 for F32, D%8==0 for
  * F16/BF16, D%16==0 for INT8_ROWWISE), so that rows can be gathered with 128-bit loads.
  */

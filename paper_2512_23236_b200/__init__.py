@@ -18,7 +18,8 @@ EBAG_OK, EBAG_ERR_INVALID_ARG, EBAG_ERR_UNSUPPORTED, EBAG_ERR_CUDA = 0, 1, 2, 3
 EBAG_ERR_INDEX_OOB, EBAG_ERR_BAD_OFFSETS = 4, 5
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_PKG, "libebag.so")
+# EBAG_LIB points the binding at another build of the same library (kernel-tuning experiments)
+LIB_PATH = os.environ.get("EBAG_LIB") or os.path.join(_PKG, "libebag.so")
 
 # name -> (restype, argtypes); kept in step with include/ebag.h (a test parses the header)
 _vp, _i32, _i64, _int = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_int

@@ -201,8 +201,9 @@ ebag_status grow(ebag_tbe* h, T** buf, int64_t* cap, int64_t need) {
 __global__ void pack_int8_rowwise_kernel(const int8_t* __restrict__ q, const float* __restrict__ scale,
                                          const float* __restrict__ bias, int64_t rows, int D,
                                          uint4* __restrict__ dst) {
-    // one thread per 16-byte vector of the packed row: D/16 vectors of codes, then one vector
-    // holding scale, bias and 8 bytes of zero padding
+    // one thread per 16-byte vector of the packed row: D/16 vectors of codes, stored biased by
+    // +128 (sign bit flipped) so that the forward kernel widens them without a sign fix-up, then
+    // one vector holding scale, bias and 8 bytes of zero padding
     const int vecs = D / 16 + 1;
     const int64_t total = rows * vecs;
     for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total;
@@ -212,6 +213,10 @@ __global__ void pack_int8_rowwise_kernel(const int8_t* __restrict__ q, const flo
         uint4 x;
         if (v < vecs - 1) {
             x = *reinterpret_cast<const uint4*>(q + r * D + v * 16);
+            x.x ^= 0x80808080u;
+            x.y ^= 0x80808080u;
+            x.z ^= 0x80808080u;
+            x.w ^= 0x80808080u;
         } else {
             x = make_uint4(__float_as_uint(scale[r]), __float_as_uint(bias[r]), 0u, 0u);
         }
@@ -252,8 +257,7 @@ ebag_status ebag_create_tbe(int32_t T, const int64_t* rows, const int32_t* D, eb
         int g_log2 = 2;
         while ((1 << g_log2) < m.nvec && g_log2 < 5) ++g_log2;
         m.g_log2 = g_log2;
-        const int per_lane = (m.nvec + 31) / 32;
-        m.V = per_lane <= 1 ? 1 : (per_lane == 2 ? 2 : 4);
+        m.V = m.nvec <= 32 ? 1 : 2;
         d_off += D[t];
         if (d_off >= (1ll << 31)) return EBAG_ERR_UNSUPPORTED;
     }

@@ -1,19 +1,21 @@
 // Device code of the pooled embedding-bag forward (sm_100a).
 //
-// One persistent kernel serves all T tables of a call.  Work is cut into ITEMS: runs of
+// One persistent kernel serves all T tables of a call.  Work is cut into ITEMS: runs of up to 32
 // consecutive bags of one table, sized on the device from the offsets array (which is the prefix
 // sum of the bag lengths) so that every item gathers about `item_bytes` of rows whatever the
-// table's row size and mean bag length.  Warps pull items from a global counter in table-major
-// order, so a table's hot rows stay in L2 while that table is being processed and bags of very
-// unequal length are balanced dynamically.
+// table's row size and mean bag length (less when the whole call is small, so that every warp
+// still gets work).  Warps pull items from a global counter in table-major order, so a table's
+// hot rows stay in L2 while that table is being processed and bags of very unequal length are
+// balanced dynamically.
 //
 // Inside an item a warp is split into row groups of G lanes (G*16 bytes cover one row, G in
-// {4,8,16,32}; rows above 512 bytes take V = 2 or 4 vectors per lane).  Each group owns one bag
-// at a time.  The lanes of a group read G ids (and weights) of their bag with one coalesced load,
-// one chunk ahead of use; each id is then broadcast inside the group with a shuffle and up to
-// ROWS_IN_FLIGHT rows are requested with 128-bit loads before the first is consumed.  Widening
-// (bf16/fp16), rowwise-int8 dequantisation and the per-sample weight are fused into the fp32
-// accumulation; the result is written once with 128-bit streaming stores.
+// {4,8,16,32}; rows above 512 bytes take 2 vectors per lane, in column tiles of 1 KB).  Each group owns one bag
+// at a time; the 32/G bags that run side by side are picked after sorting the item's bags by
+// length, so the groups finish together.  The lanes of a group read G ids (and weights) of their
+// bag with one coalesced load, one chunk ahead of use; each id is then broadcast inside the
+// group with a shuffle and up to U rows are requested with 128-bit loads before the first is
+// consumed.  Widening (bf16/fp16), rowwise-int8 dequantisation and the per-sample weight are
+// fused into the fp32 accumulation; the result is written once with 128-bit streaming stores.
 //
 // Ids outside the table and malformed bags never fault: they are skipped, counted and reported
 // through the handle's status words.
@@ -23,6 +25,13 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#ifndef EBAG_ROWS_IN_FLIGHT
+#define EBAG_ROWS_IN_FLIGHT 4
+#endif
+#ifndef EBAG_MIN_BLOCKS
+#define EBAG_MIN_BLOCKS 4
+#endif
+
 namespace ebag {
 
 enum : int { DT_F32 = 0, DT_F16 = 1, DT_BF16 = 2, DT_INT8 = 3 };
@@ -30,6 +39,7 @@ enum : int { DT_F32 = 0, DT_F16 = 1, DT_BF16 = 2, DT_INT8 = 3 };
 constexpr int kThreads = 256;            // 8 warps per CTA
 constexpr int kWarps = kThreads / 32;
 constexpr int kMaxItemBags = 32;         // an item's offsets live in one register per lane
+constexpr int kItemsPerWarp = 4;         // small calls: aim for at least this many items per warp
 constexpr uint32_t kInvalidRow = 0xFFFFFFFFu;
 
 struct TableMeta {       // per table, built at create, lives in device memory
@@ -39,7 +49,7 @@ struct TableMeta {       // per table, built at create, lives in device memory
     int32_t stride;      // bytes between stored rows
     int32_t nvec;        // 16-byte vectors of payload per row (int8: of codes)
     int32_t g_log2;      // log2 of lanes per row group
-    int32_t V;           // vectors per lane (1, 2 or 4); nvec > 32*4 is walked in column tiles
+    int32_t V;           // vectors per lane (1 or 2); nvec > 64 is walked in 1 KB column tiles
 };
 
 struct Queue {           // handle-owned scratch; both zero between launches
@@ -89,6 +99,15 @@ __device__ __forceinline__ int64_t shfl64(int64_t v, int src) {
     return ((int64_t)hi << 32) | (uint32_t)lo;
 }
 
+// acc += widen(h) for a 16-bit float held in the low half of `h` (mixed-precision add, one
+// instruction on sm_100a)
+__device__ __forceinline__ void add_bf16(float& acc, uint32_t h) {
+    asm("add.rn.f32.bf16 %0, %1, %0;" : "+f"(acc) : "h"((unsigned short)h));
+}
+__device__ __forceinline__ void add_f16(float& acc, uint32_t h) {
+    asm("add.rn.f32.f16 %0, %1, %0;" : "+f"(acc) : "h"((unsigned short)h));
+}
+
 // ------------------------------------------------------------------ per-dtype accumulation
 template <int DT> struct Elem;
 template <> struct Elem<DT_F32>  { static constexpr int kAcc = 4; };
@@ -109,82 +128,124 @@ __device__ __forceinline__ void accumulate(float* acc, const uint4& d, float w) 
     } else if constexpr (DT == DT_BF16) {
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-            const float lo = __uint_as_float(r[i] << 16);
-            const float hi = __uint_as_float(r[i] & 0xffff0000u);
-            acc[2 * i] = WEIGHTED ? fmaf(w, lo, acc[2 * i]) : acc[2 * i] + lo;
-            acc[2 * i + 1] = WEIGHTED ? fmaf(w, hi, acc[2 * i + 1]) : acc[2 * i + 1] + hi;
+            if constexpr (WEIGHTED) {
+                acc[2 * i] = fmaf(w, __uint_as_float(r[i] << 16), acc[2 * i]);
+                acc[2 * i + 1] = fmaf(w, __uint_as_float(r[i] & 0xffff0000u), acc[2 * i + 1]);
+            } else {
+                add_bf16(acc[2 * i], r[i]);
+                add_bf16(acc[2 * i + 1], r[i] >> 16);
+            }
         }
     } else if constexpr (DT == DT_F16) {
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-            const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&r[i]));
-            acc[2 * i] = WEIGHTED ? fmaf(w, f.x, acc[2 * i]) : acc[2 * i] + f.x;
-            acc[2 * i + 1] = WEIGHTED ? fmaf(w, f.y, acc[2 * i + 1]) : acc[2 * i + 1] + f.y;
+            if constexpr (WEIGHTED) {
+                const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&r[i]));
+                acc[2 * i] = fmaf(w, f.x, acc[2 * i]);
+                acc[2 * i + 1] = fmaf(w, f.y, acc[2 * i + 1]);
+            } else {
+                add_f16(acc[2 * i], r[i]);
+                add_f16(acc[2 * i + 1], r[i] >> 16);
+            }
         }
     } else {
-        // int8 code q -> float without the conversion pipe: flip the sign bit (u = q + 128),
-        // drop the byte into the mantissa of 2^23, subtract 2^23 + 128.  Exact.
+        // Stored code u = q + 128 (0..255).  Dropping the byte into the mantissa of 2^23 gives the
+        // float 2^23 + u; subtracting 2^23 + 128 leaves q, exactly, without the conversion pipe.
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-            const uint32_t u = r[i] ^ 0x80808080u;
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
-                const float f = __uint_as_float(__byte_perm(u, 0x4B000000u, 0x7440 + k));
-                const float q = f - 8388736.0f;                     // 2^23 + 128
-                acc[4 * i + k] = fmaf(w, q, acc[4 * i + k]);
+                const float f = __uint_as_float(__byte_perm(r[i], 0x4B000000u, 0x7440 + k));
+                acc[4 * i + k] = fmaf(w, f - 8388736.0f, acc[4 * i + k]);
             }
         }
     }
 }
 
+// Sort 32 keys, one per lane, in descending order (bitonic network, 15 exchange steps).
+__device__ __forceinline__ uint32_t warp_sort_desc(uint32_t v, int lane) {
+#pragma unroll
+    for (int k = 2; k <= 32; k <<= 1) {
+#pragma unroll
+        for (int j = k >> 1; j > 0; j >>= 1) {
+            const uint32_t o = __shfl_xor_sync(0xffffffffu, v, j);
+            const bool lower = (lane & j) == 0;
+            const bool desc = (lane & k) == 0;
+            v = (lower == desc) ? max(v, o) : min(v, o);
+        }
+    }
+    return v;
+}
+
 // ------------------------------------------------------------------ one item
-// Bags [bag0, bag0 + cnt) of table t; cnt <= 32.  G lanes per row, V vectors per lane.
+// Bags [bag0, bag0 + cnt) of table t; cnt <= 32.  V vectors per lane; the lanes per row (G) are
+// a run-time property of the table so that one instance of this code serves every row width.
 // vec0: first 16-byte vector of the column tile this call covers (0 unless the row is wider
 // than 32*4 vectors).
-template <int DT, bool WEIGHTED, int G, int V>
+template <int DT, bool WEIGHTED, int V>
 __device__ __forceinline__ void process_item(const FwdParams& p, const TableMeta& m,
                                              const char* __restrict__ tbase, int t, int64_t bag0,
                                              int cnt, int vec0, int lane, unsigned& n_oob,
                                              unsigned& n_bad) {
-    constexpr int NG = 32 / G;                       // row groups (bags in progress) per warp
     constexpr int NACC = Elem<DT>::kAcc;
-    constexpr int U = (8 / V) < G ? (8 / V) : G;     // rows requested before the first is used
+    constexpr int U = EBAG_ROWS_IN_FLIGHT / V;       // rows requested before the first is used
+    const int G = 1 << m.g_log2;                     // lanes per row (runtime: 4, 8, 16 or 32)
+    const int NG = 32 >> m.g_log2;                   // row groups (bags in progress) per warp
     const int lig = lane & (G - 1);
-    const int grp = lane / G;
+    const int grp = lane >> m.g_log2;
     const int64_t g0 = (int64_t)t * p.B + bag0;
 
-    // the item's offsets: lane i holds the bounds of bag i
-    int64_t off_lo = 0, off_hi = 0;
+    // The item's offsets: lane i holds the bounds of bag i, as 32-bit distances from the item's
+    // first offset (an item's bags are consecutive, so its ids are one contiguous run).
+    const int64_t base_raw = ld_stream_i64(p.offsets + g0);               // same address in all lanes
+    const int64_t base = base_raw < 0 ? 0 : (base_raw > p.n_indices ? p.n_indices : base_raw);
+    const int64_t room = p.n_indices - base;                              // ids left after base
+    uint32_t off_lo = 0, off_hi = 0;
+    uint32_t key = (uint32_t)lane;                   // lanes without a bag sort last
     if (lane < cnt) {
-        off_lo = ld_stream_i64(p.offsets + g0 + lane);
-        off_hi = ld_stream_i64(p.offsets + g0 + lane + 1);
-        if (off_hi < off_lo || off_lo < 0 || off_hi > p.n_indices) {
+        const int64_t lo = ld_stream_i64(p.offsets + g0 + lane) - base;
+        const int64_t hi = ld_stream_i64(p.offsets + g0 + lane + 1) - base;
+        // malformed (backwards, outside the id list) or longer than 2^31-1: treated as empty
+        if (base_raw != base || lo < 0 || hi < lo || hi > room || hi > 0x7fffffffll) {
             if (vec0 == 0) ++n_bad;
-            off_lo = off_hi = 0;
+        } else {
+            off_lo = (uint32_t)lo;
+            off_hi = (uint32_t)hi;
         }
+        const uint32_t len = off_hi - off_lo;
+        key = (((len > 0x3FFFFFEu ? 0x3FFFFFEu : len) + 1u) << 5) | (uint32_t)lane;
     }
+    // bags that share a slot run in lockstep: pair bags of similar length
+    if (NG > 1 && cnt > NG) key = warp_sort_desc(key, lane);
+    const int64_t* __restrict__ idx_base = p.indices + base;
+    const float* __restrict__ w_base = WEIGHTED ? p.weights + base : nullptr;
 
     bool col_on[V];
-    int col_byte[V];
+    const char* lane_base[V];
 #pragma unroll
     for (int v = 0; v < V; ++v) {
         const int vec = vec0 + v * G + lig;
         col_on[v] = vec < m.nvec;
-        col_byte[v] = vec * 16;
+        lane_base[v] = tbase + vec * 16;
     }
+    bool my_cols = true;
+#pragma unroll
+    for (int v = 0; v < V; ++v) my_cols = my_cols && col_on[v];
+    const bool cols_full = __all_sync(0xffffffffu, my_cols);   // every lane owns V vectors
     const uint32_t stride = (uint32_t)m.stride;
     const uint64_t rows = (uint64_t)m.rows;
+    const char* sb_base = tbase + m.D;               // int8: scale and bias follow the codes
 
     // ids (validated, narrowed to 32 bits) and weights of one chunk: lane `lig` of a group
     // holds entry pos + lig of the group's bag
-    auto load_chunk = [&](int64_t pos, int64_t end, uint32_t& ridx, float& w) {
+    auto load_chunk = [&](uint32_t pos, uint32_t end, uint32_t& ridx, float& w) {
         ridx = kInvalidRow;
         w = 0.0f;
-        const int64_t i = pos + lig;
+        const uint32_t i = pos + lig;
         if (i < end) {
-            const int64_t r = ld_stream_i64(p.indices + i);
+            const int64_t r = ld_stream_i64(idx_base + i);
             float wl = 1.0f;
-            if (WEIGHTED) wl = ld_stream_f32(p.weights + i);
+            if (WEIGHTED) wl = ld_stream_f32(w_base + i);
             if ((uint64_t)r < rows) {
                 ridx = (uint32_t)r;
                 w = wl;
@@ -193,17 +254,21 @@ __device__ __forceinline__ void process_item(const FwdParams& p, const TableMeta
             }
         }
     };
+    // bounds and output row of the bag that sorted position `pos_in_item` holds
+    auto slot_bag = [&](int pos_in_item, uint32_t& s, uint32_t& e, int& orig) {
+        const uint32_t k = __shfl_sync(0xffffffffu, key, pos_in_item & 31);
+        orig = (int)(k & 31u);
+        s = __shfl_sync(0xffffffffu, off_lo, orig);
+        e = __shfl_sync(0xffffffffu, off_hi, orig);
+        if (pos_in_item >= cnt) s = e = 0;
+    };
 
-    const int nslots = (cnt + NG - 1) / NG;
+    const int nslots = (cnt + NG - 1) >> (5 - m.g_log2);
     int slot = 0;
-    int64_t s, e;
-    {
-        const int j = grp;                            // slot 0
-        s = shfl64(off_lo, j < cnt ? j : 0);
-        e = shfl64(off_hi, j < cnt ? j : 0);
-        if (j >= cnt) s = e = 0;
-    }
-    int64_t pos = s;
+    uint32_t s, e;
+    int orig;
+    slot_bag(grp, s, e, orig);
+    uint32_t pos = s;
     uint32_t cur_r, nxt_r = kInvalidRow;
     float cur_w, nxt_w = 0.0f;
     load_chunk(pos, e, cur_r, cur_w);
@@ -217,64 +282,89 @@ __device__ __forceinline__ void process_item(const FwdParams& p, const TableMeta
 
     while (true) {
         // ---- prefetch the ids of the next chunk (same bag, or first chunk of the next slot)
-        const int64_t pos_next = pos + G;
+        // (pos <= e < 2^31 and G <= 32, so pos + G cannot wrap)
+        const uint32_t pos_next = pos + G;
         const bool more = __any_sync(0xffffffffu, pos_next < e);
-        int64_t s2 = 0, e2 = 0;
+        uint32_t s2 = 0, e2 = 0;
+        int orig2 = 0;
         if (more) {
             load_chunk(pos_next, e, nxt_r, nxt_w);
         } else if (slot + 1 < nslots) {
-            const int j = (slot + 1) * NG + grp;
-            s2 = shfl64(off_lo, j < cnt ? j : 0);
-            e2 = shfl64(off_hi, j < cnt ? j : 0);
-            if (j >= cnt) s2 = e2 = 0;
+            slot_bag((slot + 1) * NG + grp, s2, e2, orig2);
             load_chunk(s2, e2, nxt_r, nxt_w);
         }
 
         // ---- gather and accumulate the rows of the current chunk
-        int64_t left = e - pos;
-        const int nval = left <= 0 ? 0 : (left > G ? G : (int)left);
+        const uint32_t left = e - pos;               // pos <= e always
+        const int nval = left > (uint32_t)G ? G : (int)left;      // rows of my group's bag in this chunk
         const int nmax = __reduce_max_sync(0xffffffffu, nval);
-#pragma unroll
-        for (int j0 = 0; j0 < G; j0 += U) {
-            if (j0 < nmax) {
-                uint32_t r[U];
+        const int nmin = __reduce_min_sync(0xffffffffu, nval);
+        // no id of this chunk was rejected: full batches need no per-row checks
+        // (wide rows, V == 2, are bound by DRAM latency, not by instruction issue, and measured
+        // faster through the checked loop alone, which needs fewer registers)
+        const bool clean = V == 1 && cols_full &&
+                           __all_sync(0xffffffffu, lig >= nval || cur_r != kInvalidRow);
+        int j0 = 0;
+        if (clean) {
+#pragma unroll 1
+            for (; j0 + U <= nmin; j0 += U) {        // every group has U more valid rows
                 float w[U];
                 uint4 d[U][V];
-                float sb[U][2];
+                float2 sb[U];
 #pragma unroll
                 for (int u = 0; u < U; ++u) {
-                    r[u] = __shfl_sync(0xffffffffu, cur_r, j0 + u, G);
-                    w[u] = WEIGHTED ? __shfl_sync(0xffffffffu, cur_w, j0 + u, G) : 1.0f;
+                    const uint32_t r = __shfl_sync(0xffffffffu, cur_r, j0 + u, G);
+                    if (WEIGHTED) w[u] = __shfl_sync(0xffffffffu, cur_w, j0 + u, G);
+                    const uint64_t roff = (uint64_t)r * stride;
+#pragma unroll
+                    for (int v = 0; v < V; ++v) d[u][v] = ld_row16(lane_base[v] + roff);
+                    if (DT == DT_INT8) sb[u] = __ldg(reinterpret_cast<const float2*>(sb_base + roff));
                 }
 #pragma unroll
                 for (int u = 0; u < U; ++u) {
-                    const char* row = tbase + (uint64_t)r[u] * stride;
-                    const bool ok = r[u] != kInvalidRow;
-#pragma unroll
-                    for (int v = 0; v < V; ++v) {
-                        d[u][v] = make_uint4(0u, 0u, 0u, 0u);
-                        if (ok && col_on[v]) d[u][v] = ld_row16(row + col_byte[v]);
-                    }
+                    float wu = WEIGHTED ? w[u] : 1.0f;
                     if (DT == DT_INT8) {
-                        sb[u][0] = 0.0f;
-                        sb[u][1] = 0.0f;
-                        if (ok) {
-                            const float2 c = __ldg(reinterpret_cast<const float2*>(row + m.D));
-                            sb[u][0] = c.x;
-                            sb[u][1] = c.y;
-                        }
+                        acc_bias = fmaf(wu, sb[u].y, acc_bias);
+                        wu *= sb[u].x;
                     }
-                }
 #pragma unroll
-                for (int u = 0; u < U; ++u) {
+                    for (int v = 0; v < V; ++v)
+                        accumulate<DT, WEIGHTED || DT == DT_INT8>(acc[v], d[u][v], wu);
+                }
+            }
+        }
+#pragma unroll 1
+        for (; j0 < nmax; j0 += U) {                 // ragged tail, rejected ids, partial columns
+            uint32_t okmask = 0;
+            float w[U];
+            uint4 d[U][V];
+            float2 sb[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const uint32_t r = __shfl_sync(0xffffffffu, cur_r, j0 + u, G);
+                w[u] = WEIGHTED ? __shfl_sync(0xffffffffu, cur_w, j0 + u, G) : 1.0f;
+                if (j0 + u < nval && r != kInvalidRow) {
+                    okmask |= 1u << u;
+                    const uint64_t roff = (uint64_t)r * stride;
+#pragma unroll
+                    for (int v = 0; v < V; ++v)
+                        if (col_on[v]) d[u][v] = ld_row16(lane_base[v] + roff);
+                    if (DT == DT_INT8)
+                        sb[u] = __ldg(reinterpret_cast<const float2*>(sb_base + roff));
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                if (okmask & (1u << u)) {
                     float wu = w[u];
-                    if (!WEIGHTED && r[u] == kInvalidRow) wu = 0.0f;
                     if (DT == DT_INT8) {
-                        acc_bias = fmaf(wu, sb[u][1], acc_bias);
-                        wu *= sb[u][0];
+                        acc_bias = fmaf(wu, sb[u].y, acc_bias);
+                        wu *= sb[u].x;
                     }
 #pragma unroll
-                    for (int v = 0; v < V; ++v) accumulate<DT, WEIGHTED || DT == DT_INT8>(acc[v], d[u][v], wu);
+                    for (int v = 0; v < V; ++v)
+                        if (col_on[v])
+                            accumulate<DT, WEIGHTED || DT == DT_INT8>(acc[v], d[u][v], wu);
                 }
             }
         }
@@ -283,10 +373,9 @@ __device__ __forceinline__ void process_item(const FwdParams& p, const TableMeta
             pos = pos_next;
         } else {
             // ---- the bags of this slot are complete: finalise and store
-            const int j = slot * NG + grp;
-            if (j < cnt) {
-                const int64_t L = e - s;
-                float* orow = p.out + (bag0 + j) * (int64_t)p.sumD + m.D_off;
+            if (slot * NG + grp < cnt) {
+                const uint32_t L = e - s;
+                float* orow = p.out + (bag0 + orig) * (int64_t)p.sumD + m.D_off;
 #pragma unroll
                 for (int v = 0; v < V; ++v) {
                     if (!col_on[v]) continue;
@@ -307,6 +396,7 @@ __device__ __forceinline__ void process_item(const FwdParams& p, const TableMeta
             if (slot >= nslots) break;
             s = s2;
             e = e2;
+            orig = orig2;
             pos = s;
             acc_bias = 0.0f;
 #pragma unroll
@@ -321,25 +411,37 @@ __device__ __forceinline__ void process_item(const FwdParams& p, const TableMeta
 
 // ------------------------------------------------------------------ the kernel
 template <int DT, bool WEIGHTED>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, EBAG_MIN_BLOCKS)
 ebag_fwd_kernel(const FwdParams p) {
     extern __shared__ int smem_i[];
-    int* item_base = smem_i;                 // [T+1] first item of each table
-    int* item_bags = smem_i + p.T + 1;       // [T]   bags per item of each table
+    int* item_base = smem_i;                                   // [T+1] first item of each table
+    int* item_bags = smem_i + p.T + 1;                         // [T]   bags per item of each table
+    float* bag_bytes = reinterpret_cast<float*>(item_bags);    // [T]   (first pass) bytes per bag
+    __shared__ float total_bytes;
     const int tid = threadIdx.x;
     const int lane = tid & 31;
 
     // ---- size the items of every table from its share of the offsets prefix sum
+    if (tid == 0) total_bytes = 0.0f;
+    __syncthreads();
     for (int t = tid; t < p.T; t += kThreads) {
-        const TableMeta m = p.meta[t];
         const int64_t n0 = p.offsets[(int64_t)t * p.B];
         const int64_t n1 = p.offsets[(int64_t)(t + 1) * p.B];
         int64_t nt = n1 - n0;
         if (nt < 0) nt = 0;
         if (nt > p.n_indices) nt = p.n_indices;
-        const int ng = 32 >> m.g_log2;
-        const float mean_len = (float)nt / (float)p.B;
-        const float want = (float)p.item_bytes / ((float)m.stride * fmaxf(mean_len, 1e-6f));
+        const float bytes = (float)nt * (float)p.meta[t].stride;
+        bag_bytes[t] = fmaxf(bytes / (float)p.B, 1.0f);
+        atomicAdd(&total_bytes, bytes);
+    }
+    __syncthreads();
+    // small calls: shrink the items so that every warp of the grid gets a few of them
+    const float spread = total_bytes / (float)(gridDim.x * kWarps * kItemsPerWarp);
+    const float item_bytes = fminf((float)p.item_bytes, spread);
+    __syncthreads();
+    for (int t = tid; t < p.T; t += kThreads) {
+        const int ng = 32 >> p.meta[t].g_log2;
+        const float want = item_bytes / bag_bytes[t];
         int ib = want >= (float)kMaxItemBags ? kMaxItemBags : (int)want;
         ib = (ib / ng) * ng;
         if (ib < ng) ib = ng;
@@ -366,11 +468,14 @@ ebag_fwd_kernel(const FwdParams p) {
     const unsigned total = (unsigned)item_base[p.T];
 
     unsigned n_oob = 0, n_bad = 0;
-    while (true) {
-        unsigned q = 0;
-        if (lane == 0) q = atomicAdd(&p.queue->next, 1u);
-        q = __shfl_sync(0xffffffffu, q, 0);
-        if (q >= total) break;
+    unsigned q = 0;
+    if (lane == 0) q = atomicAdd(&p.queue->next, 1u);
+    q = __shfl_sync(0xffffffffu, q, 0);
+    while (q < total) {
+        // ask for the next item now; the answer is needed only after this one is done
+        unsigned q_next = 0;
+        if (lane == 0) q_next = atomicAdd(&p.queue->next, 1u);
+
         // table of item q: last t with item_base[t] <= q
         int lo = 0, hi = p.T;
         while (hi - lo > 1) {
@@ -386,23 +491,13 @@ ebag_fwd_kernel(const FwdParams p) {
         const char* tbase = static_cast<const char*>(p.tables[t]);
 
         if (m.V == 1) {
-            switch (m.g_log2) {
-                case 2: process_item<DT, WEIGHTED, 4, 1>(p, m, tbase, t, bag0, cnt, 0, lane, n_oob, n_bad); break;
-                case 3: process_item<DT, WEIGHTED, 8, 1>(p, m, tbase, t, bag0, cnt, 0, lane, n_oob, n_bad); break;
-                case 4: process_item<DT, WEIGHTED, 16, 1>(p, m, tbase, t, bag0, cnt, 0, lane, n_oob, n_bad); break;
-                default: process_item<DT, WEIGHTED, 32, 1>(p, m, tbase, t, bag0, cnt, 0, lane, n_oob, n_bad); break;
-            }
-        } else if (m.V == 2) {
-            process_item<DT, WEIGHTED, 32, 2>(p, m, tbase, t, bag0, cnt, 0, lane, n_oob, n_bad);
+            process_item<DT, WEIGHTED, 1>(p, m, tbase, t, bag0, cnt, 0, lane, n_oob, n_bad);
         } else {
-            if constexpr (DT == DT_INT8) {
-                for (int vec0 = 0; vec0 < m.nvec; vec0 += 64)
-                    process_item<DT, WEIGHTED, 32, 2>(p, m, tbase, t, bag0, cnt, vec0, lane, n_oob, n_bad);
-            } else {
-                for (int vec0 = 0; vec0 < m.nvec; vec0 += 128)
-                    process_item<DT, WEIGHTED, 32, 4>(p, m, tbase, t, bag0, cnt, vec0, lane, n_oob, n_bad);
-            }
+            // rows above 512 bytes: two vectors per lane, 1 KB column tiles
+            for (int vec0 = 0; vec0 < m.nvec; vec0 += 64)
+                process_item<DT, WEIGHTED, 2>(p, m, tbase, t, bag0, cnt, vec0, lane, n_oob, n_bad);
         }
+        q = __shfl_sync(0xffffffffu, q_next, 0);
     }
 
     // ---- report what was skipped; the last CTA out re-arms the queue for the next launch
