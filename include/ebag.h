@@ -134,6 +134,39 @@ ebag_status ebag_pack_int8_rowwise(const int8_t* q, const float* scale, const fl
                                    int64_t rows, int32_t D, void* dst, ebag_stream stream);
 
 /*
+ * The same forward without a handle and without any allocation (the paper has no counterpart;
+ * this exists for deployment).  Some callers cannot allocate device memory when they need a
+ * forward: code that runs inside a memory pool whose owner forbids side allocations, a plugin in
+ * a host application that has already given all device memory to its own allocator, a serving
+ * thread that may not pay for an allocation and the synchronisation it can imply.
+ * ebag_create_tbe allocates, so such callers cannot use a handle.  Here the few KB of device
+ * scratch the forward kernel needs (work-queue counters, status words, the table-pointer array
+ * and per-table metadata) live in a static device array of EBAG_NOALLOC_SCRATCH_BYTES that the
+ * loaded library holds on every GPU until the process exits.
+ *   T, rows, D, dtype   as for ebag_create_tbe, host arrays, read before the call returns;
+ *                       T <= EBAG_NOALLOC_MAX_TABLES (more: EBAG_ERR_UNSUPPORTED, nothing runs)
+ *   tables ... out      as for ebag_forward (device pointers; tables is a host array)
+ *   status_counts       device unsigned long long [2] or NULL.  If given, the kernel ADDS the
+ *                       number of skipped out-of-range ids to [0] and of malformed bags to [1]
+ *                       (the caller zeroes and reads it); if NULL those counts are dropped.
+ * Runs on the CURRENT device of the calling thread, on `stream`: one small set-up kernel and the
+ * forward kernel.  It calls no cudaMalloc/cudaFree and no allocating library routine.  The
+ * first call on each device also looks up the device address of the static array; make that
+ * first call before any stream capture.  All calls on one device share the array, which keeps
+ * the previous call's contents (each call rewrites what it uses and clears the counters that
+ * must start at zero): two calls that overlap on the GPU -- different streams, or the handle-free
+ * path from two threads -- race on it; run them one after another.
+ */
+#define EBAG_NOALLOC_MAX_TABLES 64
+#define EBAG_NOALLOC_SCRATCH_BYTES 4096
+ebag_status ebag_forward_noalloc(int32_t T, const int64_t* rows, const int32_t* D,
+                                 ebag_dtype dtype, const void* const* tables,
+                                 const int64_t* indices, int64_t n_indices, const int64_t* offsets,
+                                 const float* per_sample_weights, int64_t B, ebag_mode mode,
+                                 float* out, unsigned long long* status_counts,
+                                 ebag_stream stream);
+
+/*
  * Tuning knobs, for experiments; defaults are chosen at create.  Names:
  *   "item_bytes"   target bytes of gathered rows per work item (default 32768)
  *   "ctas_per_sm"  resident CTAs per SM of the persistent grid (default: occupancy limit)

@@ -16,6 +16,7 @@ EBAG_F32, EBAG_F16, EBAG_BF16, EBAG_INT8_ROWWISE = 0, 1, 2, 3
 EBAG_SUM, EBAG_MEAN = 0, 1
 EBAG_OK, EBAG_ERR_INVALID_ARG, EBAG_ERR_UNSUPPORTED, EBAG_ERR_CUDA = 0, 1, 2, 3
 EBAG_ERR_INDEX_OOB, EBAG_ERR_BAD_OFFSETS = 4, 5
+EBAG_NOALLOC_MAX_TABLES = 64
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
 # EBAG_LIB points the binding at another build of the same library (kernel-tuning experiments)
@@ -28,6 +29,8 @@ SIGNATURES = {
     "ebag_create_tbe": (_int, [_i32, _vp, _vp, _int, _int, _vp]),
     "ebag_forward": (_int, [_vp, _vp, _vp, _vp, _i64, _vp, _vp, _i64, _int, _vp, _vp]),
     "ebag_forward_host": (_int, [_vp, _vp, _vp, _vp, _i64, _vp, _vp, _i64, _int, _vp, _vp]),
+    "ebag_forward_noalloc": (_int, [_i32, _vp, _vp, _int, _vp, _vp, _i64, _vp, _vp, _i64, _int, _vp,
+                                    _vp, _vp]),
     "ebag_last_status": (_int, [_vp, _vp, _vp, _vp]),
     "ebag_pack_int8_rowwise": (_int, [_vp, _vp, _vp, _i64, _i32, _vp, _vp]),
     "ebag_set_param": (_int, [_vp, ctypes.c_char_p, _i64]),
@@ -106,6 +109,24 @@ def ebag_forward(h: int, table_ptrs: Sequence[int], D: Sequence[int], indices_pt
     st = fn(h, ctypes.cast(tp, _vp), ctypes.cast(d, _vp), indices_ptr, n_indices, offsets_ptr,
             weights_ptr, B, mode, out_ptr, stream_ptr)
     _check(st, "ebag_forward_host" if host else "ebag_forward")
+
+
+def ebag_forward_noalloc(rows: Sequence[int], D: Sequence[int], dtype: int,
+                         table_ptrs: Sequence[int], indices_ptr, n_indices: int, offsets_ptr,
+                         weights_ptr, B: int, mode: int, out_ptr, status_counts_ptr,
+                         stream_ptr) -> None:
+    """Handle-free forward for callers that must not allocate device memory (a plugin inside a
+    host that owns all of it, code under a strict memory pool, a latency-critical thread): the
+    kernel's scratch is a static device array inside the library.  Runs on the current device.
+    Calls that overlap on the GPU race on that array; issue them one after another."""
+    T = len(rows)
+    r = (ctypes.c_int64 * T)(*[int(x) for x in rows])
+    d = (ctypes.c_int32 * T)(*[int(x) for x in D])
+    tp = (ctypes.c_void_p * T)(*[int(p) if p else None for p in table_ptrs])
+    st = lib().ebag_forward_noalloc(T, ctypes.cast(r, _vp), ctypes.cast(d, _vp), dtype,
+                                    ctypes.cast(tp, _vp), indices_ptr, n_indices, offsets_ptr,
+                                    weights_ptr, B, mode, out_ptr, status_counts_ptr, stream_ptr)
+    _check(st, "ebag_forward_noalloc")
 
 
 def ebag_last_status(h: int, stream_ptr) -> tuple:
