@@ -106,10 +106,16 @@ ebag_status ebag_forward(ebag_tbe* h, const void* const* tables, const int32_t* 
  * The same forward for callers whose per-step data lives in HOST memory: indices, offsets,
  * per_sample_weights and out are host pointers (pinned memory makes the copies asynchronous);
  * tables stay device pointers (they are model state, loaded once).  The call copies the inputs
- * to device staging buffers owned by the handle, runs the forward, and copies the result back,
- * all on `stream`; the caller synchronises the stream before reading `out`.  The staging
- * buffers are (re)allocated inside this call whenever n_indices or B exceed what they hold, so
- * the first call, and any call with larger inputs, allocates and synchronises.
+ * to device staging buffers owned by the handle, runs the forward, and copies the result back;
+ * when it returns, everything is enqueued and `stream` is ordered after the last copy: the
+ * caller synchronises `stream` before reading `out`.  Large calls are cut into a few ranges (up to 16)
+ * of bags so that the inputs of one range, the kernel of the previous and the result of the one
+ * before travel at the same time (two copy streams owned by the handle; kernels stay on
+ * `stream`, one launch per range).  offsets is read on the host during the call; if it is not
+ * non-decreasing within [0, n_indices] the call falls back to one piece and the device reports
+ * the malformed bags as usual.  The staging buffers are (re)allocated inside this call whenever
+ * n_indices or B exceed what they hold, so the first call, and any call with larger inputs,
+ * allocates and synchronises.
  */
 ebag_status ebag_forward_host(ebag_tbe* h, const void* const* tables, const int32_t* D,
                               const int64_t* indices, int64_t n_indices, const int64_t* offsets,
@@ -170,6 +176,7 @@ ebag_status ebag_forward_noalloc(int32_t T, const int64_t* rows, const int32_t* 
  * Tuning knobs, for experiments; defaults are chosen at create.  Names:
  *   "item_bytes"   target bytes of gathered rows per work item (default 32768)
  *   "ctas_per_sm"  resident CTAs per SM of the persistent grid (default: occupancy limit)
+ *   "host_chunks"  bag ranges per ebag_forward_host call, 1..16 (default 0: from the size)
  * Returns INVALID_ARG for an unknown name or a value out of range.
  */
 ebag_status ebag_set_param(ebag_tbe* h, const char* name, int64_t value);

@@ -15,6 +15,9 @@ using namespace ebag;
 namespace {
 
 constexpr int kTableSlots = 4;   // device copies of the table-pointer array that may be in flight
+constexpr int kMaxHostChunks = 16;                 // bag ranges per ebag_forward_host call
+constexpr int64_t kHostChunkBytes = 64ll << 20;    // transfer size one range aims for
+constexpr int kAutoHostChunks = 6;                 // more ranges cost more in small copies than they hide
 
 struct DeviceGuard {             // make the handle's device current for the duration of a call
     int prev = -1;
@@ -57,6 +60,11 @@ struct ebag_tbe {
     float* s_weights = nullptr;
     float* s_out = nullptr;
     int64_t cap_indices = 0, cap_offsets = 0, cap_weights = 0, cap_out = 0;
+    // ebag_forward_host pipelines copies and kernels over ranges of bags
+    cudaStream_t s_h2d = nullptr, s_d2h = nullptr;
+    cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
+    cudaEvent_t ev_in[kMaxHostChunks] = {}, ev_done[kMaxHostChunks] = {};
+    int host_chunks = 0;                           // 0: pick from the transfer size
 };
 
 namespace {
@@ -82,6 +90,14 @@ void free_handle(ebag_tbe* h) {
         cudaFree(h->d_tables[i]);
         if (h->h_tables[i]) cudaFreeHost(h->h_tables[i]);
         if (h->slot_event[i]) cudaEventDestroy(h->slot_event[i]);
+    }
+    if (h->s_h2d) cudaStreamDestroy(h->s_h2d);
+    if (h->s_d2h) cudaStreamDestroy(h->s_d2h);
+    if (h->ev_fork) cudaEventDestroy(h->ev_fork);
+    if (h->ev_join) cudaEventDestroy(h->ev_join);
+    for (int i = 0; i < kMaxHostChunks; ++i) {
+        if (h->ev_in[i]) cudaEventDestroy(h->ev_in[i]);
+        if (h->ev_done[i]) cudaEventDestroy(h->ev_done[i]);
     }
     cudaFree(h->s_indices);
     cudaFree(h->s_offsets);
@@ -150,11 +166,13 @@ ebag_status stage_tables(ebag_tbe* h, const void* const* tables, cudaStream_t st
     return EBAG_OK;
 }
 
-// Launch on device pointers; arguments already checked.
+// Launch on device pointers for bags [b0, b1) of every table; arguments already checked.
+// offsets and out are the buffers of the WHOLE call (B bags per table).
 ebag_status forward_device(ebag_tbe* h, const void* const* tables, const int64_t* indices,
                            int64_t n_indices, const int64_t* offsets, const float* weights,
-                           int64_t B, ebag_mode mode, float* out, cudaStream_t stream) {
-    if (B == 0) return EBAG_OK;
+                           int64_t B, int64_t b0, int64_t b1, ebag_mode mode, float* out,
+                           cudaStream_t stream) {
+    if (b1 <= b0) return EBAG_OK;
     if (((uintptr_t)out & 15u) || ((uintptr_t)indices & 7u) || ((uintptr_t)offsets & 7u) ||
         ((uintptr_t)weights & 3u))
         return EBAG_ERR_INVALID_ARG;
@@ -166,13 +184,14 @@ ebag_status forward_device(ebag_tbe* h, const void* const* tables, const int64_t
     p.tables = d_tables;
     p.meta = h->d_meta;
     p.indices = indices;
-    p.offsets = offsets;
+    p.offsets = offsets + b0;
     p.weights = weights;
-    p.out = out;
+    p.out = out + b0 * (int64_t)h->sumD;
     p.queue = h->d_queue;
     p.status = h->d_status;
     p.n_indices = n_indices;
-    p.B = B;
+    p.B = b1 - b0;
+    p.off_stride = B;
     p.T = h->T;
     p.sumD = h->sumD;
     p.mean = mode == EBAG_MEAN ? 1 : 0;
@@ -292,6 +311,14 @@ ebag_status ebag_create_tbe(int32_t T, const int64_t* rows, const int32_t* D, eb
             EBAG_CUDA(h, cudaMallocHost((void**)&h->h_tables[i], sizeof(void*) * T));
             EBAG_CUDA(h, cudaEventCreateWithFlags(&h->slot_event[i], cudaEventDisableTiming));
         }
+        EBAG_CUDA(h, cudaStreamCreateWithFlags(&h->s_h2d, cudaStreamNonBlocking));
+        EBAG_CUDA(h, cudaStreamCreateWithFlags(&h->s_d2h, cudaStreamNonBlocking));
+        EBAG_CUDA(h, cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming));
+        EBAG_CUDA(h, cudaEventCreateWithFlags(&h->ev_join, cudaEventDisableTiming));
+        for (int i = 0; i < kMaxHostChunks; ++i) {
+            EBAG_CUDA(h, cudaEventCreateWithFlags(&h->ev_in[i], cudaEventDisableTiming));
+            EBAG_CUDA(h, cudaEventCreateWithFlags(&h->ev_done[i], cudaEventDisableTiming));
+        }
         for (int w = 0; w < 2; ++w) {
             EBAG_CUDA(h, occupancy_fwd(dtype, w != 0, fwd_smem_bytes(T), &h->occupancy[w]));
             if (h->occupancy[w] < 1) h->occupancy[w] = 1;
@@ -316,8 +343,8 @@ ebag_status ebag_forward(ebag_tbe* h, const void* const* tables, const int32_t* 
     if (st != EBAG_OK) return st;
     DeviceGuard guard(h->device);
     if (!guard.ok) return EBAG_ERR_CUDA;
-    return forward_device(h, tables, indices, n_indices, offsets, per_sample_weights, B, mode, out,
-                          (cudaStream_t)stream);
+    return forward_device(h, tables, indices, n_indices, offsets, per_sample_weights, B, 0, B, mode,
+                          out, (cudaStream_t)stream);
 }
 
 ebag_status ebag_forward_host(ebag_tbe* h, const void* const* tables, const int32_t* D,
@@ -339,15 +366,73 @@ ebag_status ebag_forward_host(ebag_tbe* h, const void* const* tables, const int3
         (st = grow(h, &h->s_weights, &h->cap_weights, n_indices > 0 ? n_indices : 1)) != EBAG_OK)
         return st;
     if ((st = grow(h, &h->s_out, &h->cap_out, n_out)) != EBAG_OK) return st;
-    if (n_indices > 0)
-        EBAG_CUDA(h, cudaMemcpyAsync(h->s_indices, indices, sizeof(int64_t) * n_indices, cudaMemcpyHostToDevice, s));
-    EBAG_CUDA(h, cudaMemcpyAsync(h->s_offsets, offsets, sizeof(int64_t) * n_off, cudaMemcpyHostToDevice, s));
-    if (per_sample_weights && n_indices > 0)
-        EBAG_CUDA(h, cudaMemcpyAsync(h->s_weights, per_sample_weights, sizeof(float) * n_indices, cudaMemcpyHostToDevice, s));
-    st = forward_device(h, tables, h->s_indices, n_indices, h->s_offsets,
-                        per_sample_weights ? h->s_weights : nullptr, B, mode, h->s_out, s);
-    if (st != EBAG_OK) return st;
-    EBAG_CUDA(h, cudaMemcpyAsync(out, h->s_out, sizeof(float) * n_out, cudaMemcpyDeviceToHost, s));
+    // How many bag ranges: enough for copies and kernels to overlap, few enough that a range
+    // still moves tens of MB.  The ranges need sane offsets at their borders (read here, on the
+    // host); otherwise everything goes in one piece and the device sorts it out.
+    const int64_t bytes = sizeof(int64_t) * (n_indices + n_off) + sizeof(float) * n_out +
+                          (per_sample_weights ? sizeof(float) * n_indices : 0);
+    int64_t chunks = h->host_chunks;
+    if (chunks <= 0) {
+        chunks = bytes / kHostChunkBytes;
+        if (chunks > kAutoHostChunks) chunks = kAutoHostChunks;
+    }
+    if (chunks > kMaxHostChunks) chunks = kMaxHostChunks;
+    if (chunks > B) chunks = B;
+    if (chunks < 1) chunks = 1;
+    if (chunks > 1) {                      // a full scan costs far less than the copies it guards
+        int64_t prev = 0;
+        for (int64_t i = 0; i < n_off && chunks > 1; ++i) {
+            const int64_t v = offsets[i];
+            if (v < prev || v > n_indices) chunks = 1;
+            prev = v;
+        }
+    }
+    if (chunks == 1) {
+        if (n_indices > 0)
+            EBAG_CUDA(h, cudaMemcpyAsync(h->s_indices, indices, sizeof(int64_t) * n_indices, cudaMemcpyHostToDevice, s));
+        EBAG_CUDA(h, cudaMemcpyAsync(h->s_offsets, offsets, sizeof(int64_t) * n_off, cudaMemcpyHostToDevice, s));
+        if (per_sample_weights && n_indices > 0)
+            EBAG_CUDA(h, cudaMemcpyAsync(h->s_weights, per_sample_weights, sizeof(float) * n_indices, cudaMemcpyHostToDevice, s));
+        st = forward_device(h, tables, h->s_indices, n_indices, h->s_offsets,
+                            per_sample_weights ? h->s_weights : nullptr, B, 0, B, mode, h->s_out, s);
+        if (st != EBAG_OK) return st;
+        EBAG_CUDA(h, cudaMemcpyAsync(out, h->s_out, sizeof(float) * n_out, cudaMemcpyDeviceToHost, s));
+        return EBAG_OK;
+    }
+    // Pipeline: inputs of range k+1 travel while the kernel works on range k and the result of
+    // range k-1 travels back.  Kernels stay on the caller's stream.
+    EBAG_CUDA(h, cudaEventRecord(h->ev_fork, s));
+    EBAG_CUDA(h, cudaStreamWaitEvent(h->s_h2d, h->ev_fork, 0));
+    EBAG_CUDA(h, cudaStreamWaitEvent(h->s_d2h, h->ev_fork, 0));
+    for (int64_t c = 0; c < chunks; ++c) {
+        const int64_t b0 = c * B / chunks, b1 = (c + 1) * B / chunks;
+        for (int t = 0; t < h->T; ++t) {
+            const int64_t g = (int64_t)t * B;
+            const int64_t lo = offsets[g + b0], hi = offsets[g + b1];
+            if (hi > lo) {
+                EBAG_CUDA(h, cudaMemcpyAsync(h->s_indices + lo, indices + lo, sizeof(int64_t) * (hi - lo),
+                                             cudaMemcpyHostToDevice, h->s_h2d));
+                if (per_sample_weights)
+                    EBAG_CUDA(h, cudaMemcpyAsync(h->s_weights + lo, per_sample_weights + lo,
+                                                 sizeof(float) * (hi - lo), cudaMemcpyHostToDevice, h->s_h2d));
+            }
+            // (the entry at b0 came with the previous range; range 0 brings its own)
+            const int64_t first = c == 0 ? b0 : b0 + 1;
+            EBAG_CUDA(h, cudaMemcpyAsync(h->s_offsets + g + first, offsets + g + first,
+                                         sizeof(int64_t) * (b1 - first + 1), cudaMemcpyHostToDevice, h->s_h2d));
+        }
+        EBAG_CUDA(h, cudaEventRecord(h->ev_in[c], h->s_h2d));
+        EBAG_CUDA(h, cudaStreamWaitEvent(s, h->ev_in[c], 0));
+        st = forward_device(h, tables, h->s_indices, n_indices, h->s_offsets,
+                            per_sample_weights ? h->s_weights : nullptr, B, b0, b1, mode, h->s_out, s);
+        if (st != EBAG_OK) return st;
+        EBAG_CUDA(h, cudaEventRecord(h->ev_done[c], s));
+        EBAG_CUDA(h, cudaStreamWaitEvent(h->s_d2h, h->ev_done[c], 0));
+        EBAG_CUDA(h, cudaMemcpyAsync(out + b0 * (int64_t)h->sumD, h->s_out + b0 * (int64_t)h->sumD,
+                                     sizeof(float) * (b1 - b0) * h->sumD, cudaMemcpyDeviceToHost, h->s_d2h));
+    }
+    EBAG_CUDA(h, cudaEventRecord(h->ev_join, h->s_d2h));
+    EBAG_CUDA(h, cudaStreamWaitEvent(s, h->ev_join, 0));
     return EBAG_OK;
 }
 
@@ -388,6 +473,11 @@ ebag_status ebag_set_param(ebag_tbe* h, const char* name, int64_t value) {
     if (std::strcmp(name, "item_bytes") == 0) {
         if (value < 256 || value > (1ll << 30)) return EBAG_ERR_INVALID_ARG;
         h->item_bytes = (uint32_t)value;
+        return EBAG_OK;
+    }
+    if (std::strcmp(name, "host_chunks") == 0) {
+        if (value < 0 || value > kMaxHostChunks) return EBAG_ERR_INVALID_ARG;
+        h->host_chunks = (int)value;
         return EBAG_OK;
     }
     if (std::strcmp(name, "ctas_per_sm") == 0) {

@@ -72,7 +72,9 @@ struct FwdParams {
     Queue* queue;
     Status* status;
     int64_t n_indices;
-    int64_t B;
+    int64_t B;                   // bags per table in this launch
+    int64_t off_stride;          // offsets of table t start at offsets[t * off_stride] (B for a
+                                 // whole call; the full B when a launch covers a range of bags)
     int32_t T;
     int32_t sumD;
     int32_t mean;                // 1: divide by the bag length
@@ -193,7 +195,7 @@ __device__ __forceinline__ void process_item(const FwdParams& p, const TableMeta
     const int NG = 32 >> m.g_log2;                   // row groups (bags in progress) per warp
     const int lig = lane & (G - 1);
     const int grp = lane >> m.g_log2;
-    const int64_t g0 = (int64_t)t * p.B + bag0;
+    const int64_t g0 = (int64_t)t * p.off_stride + bag0;
 
     // The item's offsets: lane i holds the bounds of bag i, as 32-bit distances from the item's
     // first offset (an item's bags are consecutive, so its ids are one contiguous run).
@@ -425,8 +427,8 @@ ebag_fwd_kernel(const FwdParams p) {
     if (tid == 0) total_bytes = 0.0f;
     __syncthreads();
     for (int t = tid; t < p.T; t += kThreads) {
-        const int64_t n0 = p.offsets[(int64_t)t * p.B];
-        const int64_t n1 = p.offsets[(int64_t)(t + 1) * p.B];
+        const int64_t n0 = p.offsets[(int64_t)t * p.off_stride];
+        const int64_t n1 = p.offsets[(int64_t)t * p.off_stride + p.B];
         int64_t nt = n1 - n0;
         if (nt < 0) nt = 0;
         if (nt > p.n_indices) nt = p.n_indices;

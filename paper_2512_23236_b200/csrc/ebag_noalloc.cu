@@ -195,6 +195,7 @@ extern "C" ebag_status ebag_forward_noalloc(int32_t T, const int64_t* rows, cons
     p.status = status_counts ? reinterpret_cast<Status*>(status_counts) : &st->scratch->status;
     p.n_indices = n_indices;
     p.B = B;
+    p.off_stride = B;
     p.T = T;
     p.sumD = (int32_t)d_off;
     p.mean = mode == EBAG_MEAN ? 1 : 0;

@@ -75,10 +75,30 @@ def test_work_partition_settings_do_not_change_results(item_bytes, ctas):
     pu.check_workload(w, params=dict(item_bytes=item_bytes, ctas_per_sm=ctas))
 
 
-def test_host_buffer_entry_point():
+@pytest.mark.parametrize("chunks", [0, 1, 3, 16])
+def test_host_buffer_entry_point(chunks):
+    """Host buffers in and out, in one piece and pipelined over ragged ranges of bags."""
+    params = dict(host_chunks=chunks) if chunks else None
     pu.check_workload(wl.make_workload(4, scale_rows=0.002, scale_B=1 / 64, max_tables=3),
-                      host_path=True)
-    pu.check_workload(wl.make_workload(2, scale_rows=0.05, scale_B=1 / 8), host_path=True)
+                      host_path=True, params=params)
+    pu.check_workload(wl.make_workload(2, scale_rows=0.05, scale_B=1 / 8), host_path=True,
+                      params=params)
+    pu.check_workload(wl.make_workload(3, scale_rows=0.004, scale_B=1 / 97, max_tables=5),
+                      host_path=True, params=params)
+
+
+def test_host_buffer_entry_point_with_malformed_offsets_falls_back():
+    rng = np.random.default_rng(12)
+    rows, D, B = [100, 50], [16, 8], 40
+    lens = [rng.integers(1, 10, size=B) for _ in rows]
+    idx, off, lengths = _jagged_from_lengths(rng, lens, rows)
+    bad = off.copy()
+    bad[10] = bad[9] - 1 if bad[9] > 0 else 0
+    tabs = _rand_tables(rng, wl.F32, rows, D)
+    gpu, status, ref = _both(wl.F32, rows, D, tabs, idx, bad, B, wl.SUM, params=dict(host_chunks=4),
+                             host_path=True)
+    assert status == (eb.EBAG_ERR_BAD_OFFSETS, ref["n_oob"], ref["n_bad_offsets"])
+    pu.compare(gpu, ref, wl.F32)
 
 
 # ------------------------------------------------------------------ shapes: every row-group path
