@@ -28,6 +28,11 @@
 #ifndef EBAG_ROWS_IN_FLIGHT
 #define EBAG_ROWS_IN_FLIGHT 4
 #endif
+// The staged (cp.async) item processor is the default; EBAG_REGISTER_PATH selects the earlier one
+// that keeps rows in registers (kept for A/B measurements).
+#ifndef EBAG_REGISTER_PATH
+#define EBAG_ASYNC 1
+#endif
 #ifndef EBAG_MIN_BLOCKS
 #define EBAG_MIN_BLOCKS 4
 #endif
@@ -93,6 +98,21 @@ __device__ __forceinline__ int64_t ld_stream_i64(const int64_t* p) {
 __device__ __forceinline__ float ld_stream_f32(const float* p) { return __ldcs(p); }
 __device__ __forceinline__ void st_stream16(float* p, float a, float b, float c, float d) {
     __stcs(reinterpret_cast<float4*>(p), make_float4(a, b, c, d));
+}
+
+// Asynchronous copies global -> shared (through L1, so hot rows still hit there): the data does
+// not occupy registers while it is in flight.
+// (`smem` is an address in the shared window, from __cvta_generic_to_shared)
+__device__ __forceinline__ void cp_async16(uint32_t smem, const void* gmem) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 16;" ::"r"(smem), "l"(gmem));
+}
+__device__ __forceinline__ void cp_async8(uint32_t smem, const void* gmem) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(smem), "l"(gmem));
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() {
+    asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
 }
 
 __device__ __forceinline__ int64_t shfl64(int64_t v, int src) {
@@ -411,6 +431,296 @@ __device__ __forceinline__ void process_item(const FwdParams& p, const TableMeta
     }
 }
 
+// ------------------------------------------------------------------ one item, staged in smem
+// Same work split as process_item, but rows travel with cp.async into a per-warp ring of
+// kStages stages (kStageVecs 16-byte vectors per lane each) and are consumed one stage behind.
+// Row fetches therefore stay in flight across batch, id-chunk and bag boundaries, and hold no
+// registers.  Every lane reads back only the slots it copied itself, so its own wait_group is
+// all the synchronisation the row data needs.
+#ifndef EBAG_STAGE_VECS
+#define EBAG_STAGE_VECS 4
+#endif
+constexpr int kStageVecs = EBAG_STAGE_VECS;      // 16-byte vectors per lane per stage
+constexpr int kStages = 2;
+
+struct IdChunk {          // ids of up to G consecutive entries of the bags one slot works on
+    uint32_t r;           // per lane: validated row id of entry `lig`, or kInvalidRow
+    float w;              // per lane: its weight
+    int nmax;             // warp-uniform: most entries any group has in this chunk
+    int nmin;             // warp-uniform: fewest
+    bool clean;           // warp-uniform: no id was rejected (set when the chunk is first requested)
+    int slot;             // warp-uniform
+    bool last;            // warp-uniform: last chunk of its slot
+    bool valid;
+};
+
+template <int DT, bool WEIGHTED, int V>
+__device__ __forceinline__ void process_item_async(const FwdParams& p, const TableMeta& m,
+                                                   const char* __restrict__ tbase, int t,
+                                                   int64_t bag0, int cnt, int vec0, int lane,
+                                                   unsigned& n_oob, unsigned& n_bad,
+                                                   uint4* __restrict__ wbuf,
+                                                   float2* __restrict__ sbbuf) {
+    constexpr int NACC = Elem<DT>::kAcc;
+    constexpr int CR = kStageVecs / V;               // rows per stage
+    const int G = 1 << m.g_log2;
+    const int NG = 32 >> m.g_log2;
+    const int lig = lane & (G - 1);
+    const int grp = lane >> m.g_log2;
+    const int64_t g0 = (int64_t)t * p.off_stride + bag0;
+
+    const int64_t base_raw = ld_stream_i64(p.offsets + g0);
+    const int64_t base = base_raw < 0 ? 0 : (base_raw > p.n_indices ? p.n_indices : base_raw);
+    const int64_t room = p.n_indices - base;
+    uint32_t off_lo = 0, off_hi = 0;
+    uint32_t key = (uint32_t)lane;
+    if (lane < cnt) {
+        const int64_t lo = ld_stream_i64(p.offsets + g0 + lane) - base;
+        const int64_t hi = ld_stream_i64(p.offsets + g0 + lane + 1) - base;
+        if (base_raw != base || lo < 0 || hi < lo || hi > room || hi > 0x7fffffffll) {
+            if (vec0 == 0) ++n_bad;
+        } else {
+            off_lo = (uint32_t)lo;
+            off_hi = (uint32_t)hi;
+        }
+        const uint32_t len = off_hi - off_lo;
+        key = (((len > 0x3FFFFFEu ? 0x3FFFFFEu : len) + 1u) << 5) | (uint32_t)lane;
+    }
+    if (NG > 1 && cnt > NG) key = warp_sort_desc(key, lane);
+    const int64_t* __restrict__ idx_base = p.indices + base;
+    const float* __restrict__ w_base = WEIGHTED ? p.weights + base : nullptr;
+
+    bool col_on[V];
+    const char* lane_base[V];
+#pragma unroll
+    for (int v = 0; v < V; ++v) {
+        const int vec = vec0 + v * G + lig;
+        col_on[v] = vec < m.nvec;
+        lane_base[v] = tbase + vec * 16;
+    }
+    const uint32_t stride = (uint32_t)m.stride;
+    const uint64_t rows = (uint64_t)m.rows;
+    const char* sb_base = tbase + m.D;
+    const int nslots = (cnt + NG - 1) >> (5 - m.g_log2);
+
+    auto load_chunk = [&](uint32_t pos, uint32_t end, uint32_t& ridx, float& w) {
+        ridx = kInvalidRow;
+        w = 0.0f;
+        const uint32_t i = pos + lig;
+        if (i < end) {
+            const int64_t r = ld_stream_i64(idx_base + i);
+            float wl = 1.0f;
+            if (WEIGHTED) wl = ld_stream_f32(w_base + i);
+            if ((uint64_t)r < rows) {
+                ridx = (uint32_t)r;
+                w = wl;
+            } else if (vec0 == 0) {
+                ++n_oob;
+            }
+        }
+    };
+    auto slot_bag = [&](int pos_in_item, uint32_t& s, uint32_t& e, int& orig) {
+        const uint32_t k = __shfl_sync(0xffffffffu, key, pos_in_item & 31);
+        orig = (int)(k & 31u);
+        s = __shfl_sync(0xffffffffu, off_lo, orig);
+        e = __shfl_sync(0xffffffffu, off_hi, orig);
+        if (pos_in_item >= cnt) s = e = 0;
+    };
+
+    // ---- generator of id chunks, in the order they are consumed
+    int gslot = -1;
+    uint32_t ge = 0, gpos = 0;
+    bool gmore = false;
+    auto gen = [&](IdChunk& c) {
+        if (gslot >= 0 && gmore) {
+            gpos += G;
+        } else {
+            ++gslot;
+            if (gslot >= nslots) {
+                c.valid = false;
+                return;
+            }
+            uint32_t gs;
+            int o;
+            slot_bag(gslot * NG + grp, gs, ge, o);
+            gpos = gs;
+        }
+        load_chunk(gpos, ge, c.r, c.w);
+        const uint32_t left = ge - gpos;
+        const int nval = left > (uint32_t)G ? G : (int)left;
+        c.nmax = __reduce_max_sync(0xffffffffu, nval);
+        c.nmin = __reduce_min_sync(0xffffffffu, nval);
+        c.clean = false;
+        gmore = __any_sync(0xffffffffu, gpos + G < ge);
+        c.slot = gslot;
+        c.last = !gmore;
+        c.valid = true;
+    };
+
+    // ---- request / use one stage (CR rows of chunk c starting at entry j0)
+    bool my_cols = true;
+#pragma unroll
+    for (int v = 0; v < V; ++v) my_cols = my_cols && col_on[v];
+    const bool cols_full = __all_sync(0xffffffffu, my_cols);
+    // this lane's slots: vector k of stage st is at my_rows[(st * kStageVecs + k) * 32]
+    const uint4* my_rows = wbuf + lane;
+    const uint32_t my_rows_s = (uint32_t)__cvta_generic_to_shared(wbuf) + lane * 16;
+    const float2* my_sb = sbbuf + grp;               // int8: scale/bias of row u at [(st*kStageVecs+u)*8]
+    const uint32_t my_sb_s = (uint32_t)__cvta_generic_to_shared(sbbuf) + grp * 8;
+    auto issue = [&](const IdChunk& c, int j0, int st) {
+        if (c.clean && j0 + CR <= c.nmin) {          // full stage, nothing to check
+#pragma unroll
+            for (int u = 0; u < CR; ++u) {
+                const uint32_t r = __shfl_sync(0xffffffffu, c.r, j0 + u, G);
+                const uint64_t roff = (uint64_t)r * stride;
+#pragma unroll
+                for (int v = 0; v < V; ++v)
+                    cp_async16(my_rows_s + (st * kStageVecs + u * V + v) * 512, lane_base[v] + roff);
+                if (DT == DT_INT8 && lig == 0)
+                    cp_async8(my_sb_s + (st * kStageVecs + u) * 64, sb_base + roff);
+            }
+            return;
+        }
+#pragma unroll
+        for (int u = 0; u < CR; ++u) {
+            const uint32_t r = __shfl_sync(0xffffffffu, c.r, j0 + u, G);
+            if (j0 + u < c.nmax && r != kInvalidRow) {
+                const uint64_t roff = (uint64_t)r * stride;
+#pragma unroll
+                for (int v = 0; v < V; ++v)
+                    if (col_on[v])
+                        cp_async16(my_rows_s + (st * kStageVecs + u * V + v) * 512, lane_base[v] + roff);
+                if (DT == DT_INT8 && lig == 0)
+                    cp_async8(my_sb_s + (st * kStageVecs + u) * 64, sb_base + roff);
+            }
+        }
+    };
+    float acc[V][NACC];
+    float acc_bias = 0.0f;
+#pragma unroll
+    for (int v = 0; v < V; ++v)
+#pragma unroll
+        for (int a = 0; a < NACC; ++a) acc[v][a] = 0.0f;
+    auto consume = [&](const IdChunk& c, int j0, int st) {
+        if (c.clean && j0 + CR <= c.nmin) {
+#pragma unroll
+            for (int u = 0; u < CR; ++u) {
+                float wu = WEIGHTED ? __shfl_sync(0xffffffffu, c.w, j0 + u, G) : 1.0f;
+                if (DT == DT_INT8) {
+                    const float2 sb = my_sb[(st * kStageVecs + u) * 8];
+                    acc_bias = fmaf(wu, sb.y, acc_bias);
+                    wu *= sb.x;
+                }
+#pragma unroll
+                for (int v = 0; v < V; ++v) {
+                    const uint4 d = my_rows[(st * kStageVecs + u * V + v) * 32];
+                    accumulate<DT, WEIGHTED || DT == DT_INT8>(acc[v], d, wu);
+                }
+            }
+            return;
+        }
+#pragma unroll
+        for (int u = 0; u < CR; ++u) {
+            const uint32_t r = __shfl_sync(0xffffffffu, c.r, j0 + u, G);
+            float wu = WEIGHTED ? __shfl_sync(0xffffffffu, c.w, j0 + u, G) : 1.0f;
+            if (j0 + u < c.nmax && r != kInvalidRow) {
+                if (DT == DT_INT8) {
+                    const float2 sb = my_sb[(st * kStageVecs + u) * 8];
+                    acc_bias = fmaf(wu, sb.y, acc_bias);
+                    wu *= sb.x;
+                }
+#pragma unroll
+                for (int v = 0; v < V; ++v)
+                    if (col_on[v]) {
+                        const uint4 d = my_rows[(st * kStageVecs + u * V + v) * 32];
+                        accumulate<DT, WEIGHTED || DT == DT_INT8>(acc[v], d, wu);
+                    }
+            }
+        }
+    };
+    auto finalize = [&](int slot) {
+        uint32_t s, e;
+        int orig;
+        slot_bag(slot * NG + grp, s, e, orig);
+        if (slot * NG + grp < cnt) {
+            const uint32_t L = e - s;
+            float* orow = p.out + (bag0 + orig) * (int64_t)p.sumD + m.D_off;
+#pragma unroll
+            for (int v = 0; v < V; ++v) {
+                if (!col_on[v]) continue;
+                float* o = orow + (size_t)(vec0 + v * G + lig) * NACC;
+#pragma unroll
+                for (int a = 0; a < NACC; ++a) {
+                    float x = acc[v][a];
+                    if (DT == DT_INT8) x += acc_bias;
+                    if (p.mean && L > 0) x = __fdiv_rn(x, (float)L);
+                    acc[v][a] = x;
+                }
+#pragma unroll
+                for (int a = 0; a < NACC; a += 4)
+                    st_stream16(o + a, acc[v][a], acc[v][a + 1], acc[v][a + 2], acc[v][a + 3]);
+            }
+        }
+        acc_bias = 0.0f;
+#pragma unroll
+        for (int v = 0; v < V; ++v)
+#pragma unroll
+            for (int a = 0; a < NACC; ++a) acc[v][a] = 0.0f;
+    };
+
+    // ---- pipeline: the request side runs one stage ahead of the consuming side
+    static_assert(kStages == 2, "the consuming side assumes it is exactly one stage behind");
+    IdChunk cons, iss, pre;
+    gen(iss);                       // nslots >= 1, so the first chunk always exists
+    gen(pre);
+    int ji = 0;                     // next entry of chunk `iss` to request
+    bool iss_done = false;
+    // request the next stage (into stage ST) and close its copy group
+    auto issue_next = [&](int st) {
+        if (!iss_done) {
+            if (ji > 0 && ji >= iss.nmax) {              // chunk exhausted: move to the next one
+                if (pre.valid) {
+                    iss = pre;
+                    gen(pre);
+                    ji = 0;
+                } else {
+                    iss_done = true;
+                }
+            }
+            if (!iss_done) {
+                if (ji == 0)        // first request of this chunk: its ids are needed now anyway
+                    iss.clean = cols_full &&
+                                __all_sync(0xffffffffu, lig >= iss.nmin || iss.r != kInvalidRow);
+                issue(iss, ji, st);
+                ji += CR;
+            }
+        }
+        cp_async_commit();          // one group per step, empty or not, keeps the counting uniform
+    };
+    int jc = 0;
+    issue_next(0);                  // stage 0 of the first chunk (cannot leave that chunk)
+    cons = iss;
+    int st = 0;                     // stage being consumed; the next request goes to the other one
+    while (true) {
+        issue_next(st ^ 1);
+        cp_async_wait<1>();         // everything but the newest group has landed
+        if (DT == DT_INT8) __syncwarp();                 // scale/bias slots are shared by a group
+        consume(cons, jc, st);
+        if (DT == DT_INT8) __syncwarp();
+        jc += CR;
+        st ^= 1;
+        if (jc >= cons.nmax) {                           // chunk consumed (an empty chunk is one step)
+            const bool was_last = cons.last;
+            const int slot = cons.slot;
+            if (was_last) finalize(slot);
+            if (was_last && slot == nslots - 1) break;
+            cons = iss;                                  // the request side is already in the next chunk
+            jc = 0;
+        }
+    }
+    cp_async_wait<0>();
+}
+
 // ------------------------------------------------------------------ the kernel
 template <int DT, bool WEIGHTED>
 __global__ void __launch_bounds__(kThreads, EBAG_MIN_BLOCKS)
@@ -420,6 +730,12 @@ ebag_fwd_kernel(const FwdParams p) {
     int* item_bags = smem_i + p.T + 1;                         // [T]   bags per item of each table
     float* bag_bytes = reinterpret_cast<float*>(item_bags);    // [T]   (first pass) bytes per bag
     __shared__ float total_bytes;
+#ifdef EBAG_ASYNC
+    __shared__ uint4 stage_buf[kWarps * kStages * kStageVecs * 32];
+    __shared__ float2 sb_buf[DT == DT_INT8 ? kWarps * kStages * kStageVecs * 8 : 1];
+    uint4* wbuf = stage_buf + (threadIdx.x >> 5) * (kStages * kStageVecs * 32);
+    float2* sbbuf = sb_buf + (DT == DT_INT8 ? (threadIdx.x >> 5) * (kStages * kStageVecs * 8) : 0);
+#endif
     const int tid = threadIdx.x;
     const int lane = tid & 31;
 
@@ -492,6 +808,14 @@ ebag_fwd_kernel(const FwdParams p) {
         const int cnt = rest < ib ? (int)rest : ib;
         const char* tbase = static_cast<const char*>(p.tables[t]);
 
+#ifdef EBAG_ASYNC
+        if (m.V == 1) {
+            process_item_async<DT, WEIGHTED, 1>(p, m, tbase, t, bag0, cnt, 0, lane, n_oob, n_bad, wbuf, sbbuf);
+        } else {
+            for (int vec0 = 0; vec0 < m.nvec; vec0 += 64)
+                process_item_async<DT, WEIGHTED, 2>(p, m, tbase, t, bag0, cnt, vec0, lane, n_oob, n_bad, wbuf, sbbuf);
+        }
+#else
         if (m.V == 1) {
             process_item<DT, WEIGHTED, 1>(p, m, tbase, t, bag0, cnt, 0, lane, n_oob, n_bad);
         } else {
@@ -499,6 +823,7 @@ ebag_fwd_kernel(const FwdParams p) {
             for (int vec0 = 0; vec0 < m.nvec; vec0 += 64)
                 process_item<DT, WEIGHTED, 2>(p, m, tbase, t, bag0, cnt, vec0, lane, n_oob, n_bad);
         }
+#endif
         q = __shfl_sync(0xffffffffu, q_next, 0);
     }
 
