@@ -9,13 +9,16 @@
 // balanced dynamically.
 //
 // Inside an item a warp is split into row groups of G lanes (G*16 bytes cover one row, G in
-// {4,8,16,32}; rows above 512 bytes take 2 vectors per lane, in column tiles of 1 KB).  Each group owns one bag
-// at a time; the 32/G bags that run side by side are picked after sorting the item's bags by
-// length, so the groups finish together.  The lanes of a group read G ids (and weights) of their
-// bag with one coalesced load, one chunk ahead of use; each id is then broadcast inside the
-// group with a shuffle and up to U rows are requested with 128-bit loads before the first is
-// consumed.  Widening (bf16/fp16), rowwise-int8 dequantisation and the per-sample weight are
-// fused into the fp32 accumulation; the result is written once with 128-bit streaming stores.
+// {4,8,16,32}, a run-time property of the table; rows above 512 bytes take 2 vectors per lane, in
+// column tiles of 1 KB).  Each group owns one bag at a time; the 32/G bags that run side by side
+// are picked after sorting the item's bags by length, so the groups finish together.  The lanes
+// of a group read G ids (and weights) of their bag with one coalesced load, two chunks ahead of
+// use; each id is then broadcast inside the group with a shuffle and the row is requested with
+// 16-byte cp.async copies (through L1) into a per-warp two-stage ring in shared memory, one
+// stage (4 row vectors per lane) ahead of the stage being accumulated.  Row fetches therefore
+// stay in flight across stage, id-chunk and bag boundaries and occupy no registers.  Widening
+// (bf16/fp16), rowwise-int8 dequantisation and the per-sample weight are fused into the fp32
+// accumulation; the result is written once with 128-bit streaming stores.
 //
 // Ids outside the table and malformed bags never fault: they are skipped, counted and reported
 // through the handle's status words.
@@ -25,14 +28,6 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
-#ifndef EBAG_ROWS_IN_FLIGHT
-#define EBAG_ROWS_IN_FLIGHT 4
-#endif
-// The staged (cp.async) item processor is the default; EBAG_REGISTER_PATH selects the earlier one
-// that keeps rows in registers (kept for A/B measurements).
-#ifndef EBAG_REGISTER_PATH
-#define EBAG_ASYNC 1
-#endif
 #ifndef EBAG_MIN_BLOCKS
 #define EBAG_MIN_BLOCKS 4
 #endif
@@ -87,10 +82,6 @@ struct FwdParams {
 };
 
 // ------------------------------------------------------------------ memory access helpers
-__device__ __forceinline__ uint4 ld_row16(const void* p) {
-    // read-only path, default L1/L2 policy: hot (Zipf) rows are meant to be caught by L1/L2
-    return __ldg(reinterpret_cast<const uint4*>(p));
-}
 __device__ __forceinline__ int64_t ld_stream_i64(const int64_t* p) {
     // ids and offsets are read once: streaming (evict-first) so they do not displace table rows
     return __ldcs(reinterpret_cast<const long long*>(p));
@@ -199,244 +190,14 @@ __device__ __forceinline__ uint32_t warp_sort_desc(uint32_t v, int lane) {
     return v;
 }
 
-// ------------------------------------------------------------------ one item
+// ------------------------------------------------------------------ one item, staged in smem
 // Bags [bag0, bag0 + cnt) of table t; cnt <= 32.  V vectors per lane; the lanes per row (G) are
 // a run-time property of the table so that one instance of this code serves every row width.
-// vec0: first 16-byte vector of the column tile this call covers (0 unless the row is wider
-// than 32*4 vectors).
-template <int DT, bool WEIGHTED, int V>
-__device__ __forceinline__ void process_item(const FwdParams& p, const TableMeta& m,
-                                             const char* __restrict__ tbase, int t, int64_t bag0,
-                                             int cnt, int vec0, int lane, unsigned& n_oob,
-                                             unsigned& n_bad) {
-    constexpr int NACC = Elem<DT>::kAcc;
-    constexpr int U = EBAG_ROWS_IN_FLIGHT / V;       // rows requested before the first is used
-    const int G = 1 << m.g_log2;                     // lanes per row (runtime: 4, 8, 16 or 32)
-    const int NG = 32 >> m.g_log2;                   // row groups (bags in progress) per warp
-    const int lig = lane & (G - 1);
-    const int grp = lane >> m.g_log2;
-    const int64_t g0 = (int64_t)t * p.off_stride + bag0;
-
-    // The item's offsets: lane i holds the bounds of bag i, as 32-bit distances from the item's
-    // first offset (an item's bags are consecutive, so its ids are one contiguous run).
-    const int64_t base_raw = ld_stream_i64(p.offsets + g0);               // same address in all lanes
-    const int64_t base = base_raw < 0 ? 0 : (base_raw > p.n_indices ? p.n_indices : base_raw);
-    const int64_t room = p.n_indices - base;                              // ids left after base
-    uint32_t off_lo = 0, off_hi = 0;
-    uint32_t key = (uint32_t)lane;                   // lanes without a bag sort last
-    if (lane < cnt) {
-        const int64_t lo = ld_stream_i64(p.offsets + g0 + lane) - base;
-        const int64_t hi = ld_stream_i64(p.offsets + g0 + lane + 1) - base;
-        // malformed (backwards, outside the id list) or longer than 2^31-1: treated as empty
-        if (base_raw != base || lo < 0 || hi < lo || hi > room || hi > 0x7fffffffll) {
-            if (vec0 == 0) ++n_bad;
-        } else {
-            off_lo = (uint32_t)lo;
-            off_hi = (uint32_t)hi;
-        }
-        const uint32_t len = off_hi - off_lo;
-        key = (((len > 0x3FFFFFEu ? 0x3FFFFFEu : len) + 1u) << 5) | (uint32_t)lane;
-    }
-    // bags that share a slot run in lockstep: pair bags of similar length
-    if (NG > 1 && cnt > NG) key = warp_sort_desc(key, lane);
-    const int64_t* __restrict__ idx_base = p.indices + base;
-    const float* __restrict__ w_base = WEIGHTED ? p.weights + base : nullptr;
-
-    bool col_on[V];
-    const char* lane_base[V];
-#pragma unroll
-    for (int v = 0; v < V; ++v) {
-        const int vec = vec0 + v * G + lig;
-        col_on[v] = vec < m.nvec;
-        lane_base[v] = tbase + vec * 16;
-    }
-    bool my_cols = true;
-#pragma unroll
-    for (int v = 0; v < V; ++v) my_cols = my_cols && col_on[v];
-    const bool cols_full = __all_sync(0xffffffffu, my_cols);   // every lane owns V vectors
-    const uint32_t stride = (uint32_t)m.stride;
-    const uint64_t rows = (uint64_t)m.rows;
-    const char* sb_base = tbase + m.D;               // int8: scale and bias follow the codes
-
-    // ids (validated, narrowed to 32 bits) and weights of one chunk: lane `lig` of a group
-    // holds entry pos + lig of the group's bag
-    auto load_chunk = [&](uint32_t pos, uint32_t end, uint32_t& ridx, float& w) {
-        ridx = kInvalidRow;
-        w = 0.0f;
-        const uint32_t i = pos + lig;
-        if (i < end) {
-            const int64_t r = ld_stream_i64(idx_base + i);
-            float wl = 1.0f;
-            if (WEIGHTED) wl = ld_stream_f32(w_base + i);
-            if ((uint64_t)r < rows) {
-                ridx = (uint32_t)r;
-                w = wl;
-            } else if (vec0 == 0) {
-                ++n_oob;
-            }
-        }
-    };
-    // bounds and output row of the bag that sorted position `pos_in_item` holds
-    auto slot_bag = [&](int pos_in_item, uint32_t& s, uint32_t& e, int& orig) {
-        const uint32_t k = __shfl_sync(0xffffffffu, key, pos_in_item & 31);
-        orig = (int)(k & 31u);
-        s = __shfl_sync(0xffffffffu, off_lo, orig);
-        e = __shfl_sync(0xffffffffu, off_hi, orig);
-        if (pos_in_item >= cnt) s = e = 0;
-    };
-
-    const int nslots = (cnt + NG - 1) >> (5 - m.g_log2);
-    int slot = 0;
-    uint32_t s, e;
-    int orig;
-    slot_bag(grp, s, e, orig);
-    uint32_t pos = s;
-    uint32_t cur_r, nxt_r = kInvalidRow;
-    float cur_w, nxt_w = 0.0f;
-    load_chunk(pos, e, cur_r, cur_w);
-
-    float acc[V][NACC];
-    float acc_bias = 0.0f;                            // int8: sum of w * bias[row]
-#pragma unroll
-    for (int v = 0; v < V; ++v)
-#pragma unroll
-        for (int a = 0; a < NACC; ++a) acc[v][a] = 0.0f;
-
-    while (true) {
-        // ---- prefetch the ids of the next chunk (same bag, or first chunk of the next slot)
-        // (pos <= e < 2^31 and G <= 32, so pos + G cannot wrap)
-        const uint32_t pos_next = pos + G;
-        const bool more = __any_sync(0xffffffffu, pos_next < e);
-        uint32_t s2 = 0, e2 = 0;
-        int orig2 = 0;
-        if (more) {
-            load_chunk(pos_next, e, nxt_r, nxt_w);
-        } else if (slot + 1 < nslots) {
-            slot_bag((slot + 1) * NG + grp, s2, e2, orig2);
-            load_chunk(s2, e2, nxt_r, nxt_w);
-        }
-
-        // ---- gather and accumulate the rows of the current chunk
-        const uint32_t left = e - pos;               // pos <= e always
-        const int nval = left > (uint32_t)G ? G : (int)left;      // rows of my group's bag in this chunk
-        const int nmax = __reduce_max_sync(0xffffffffu, nval);
-        const int nmin = __reduce_min_sync(0xffffffffu, nval);
-        // no id of this chunk was rejected: full batches need no per-row checks
-        // (wide rows, V == 2, are bound by DRAM latency, not by instruction issue, and measured
-        // faster through the checked loop alone, which needs fewer registers)
-        const bool clean = V == 1 && cols_full &&
-                           __all_sync(0xffffffffu, lig >= nval || cur_r != kInvalidRow);
-        int j0 = 0;
-        if (clean) {
-#pragma unroll 1
-            for (; j0 + U <= nmin; j0 += U) {        // every group has U more valid rows
-                float w[U];
-                uint4 d[U][V];
-                float2 sb[U];
-#pragma unroll
-                for (int u = 0; u < U; ++u) {
-                    const uint32_t r = __shfl_sync(0xffffffffu, cur_r, j0 + u, G);
-                    if (WEIGHTED) w[u] = __shfl_sync(0xffffffffu, cur_w, j0 + u, G);
-                    const uint64_t roff = (uint64_t)r * stride;
-#pragma unroll
-                    for (int v = 0; v < V; ++v) d[u][v] = ld_row16(lane_base[v] + roff);
-                    if (DT == DT_INT8) sb[u] = __ldg(reinterpret_cast<const float2*>(sb_base + roff));
-                }
-#pragma unroll
-                for (int u = 0; u < U; ++u) {
-                    float wu = WEIGHTED ? w[u] : 1.0f;
-                    if (DT == DT_INT8) {
-                        acc_bias = fmaf(wu, sb[u].y, acc_bias);
-                        wu *= sb[u].x;
-                    }
-#pragma unroll
-                    for (int v = 0; v < V; ++v)
-                        accumulate<DT, WEIGHTED || DT == DT_INT8>(acc[v], d[u][v], wu);
-                }
-            }
-        }
-#pragma unroll 1
-        for (; j0 < nmax; j0 += U) {                 // ragged tail, rejected ids, partial columns
-            uint32_t okmask = 0;
-            float w[U];
-            uint4 d[U][V];
-            float2 sb[U];
-#pragma unroll
-            for (int u = 0; u < U; ++u) {
-                const uint32_t r = __shfl_sync(0xffffffffu, cur_r, j0 + u, G);
-                w[u] = WEIGHTED ? __shfl_sync(0xffffffffu, cur_w, j0 + u, G) : 1.0f;
-                if (j0 + u < nval && r != kInvalidRow) {
-                    okmask |= 1u << u;
-                    const uint64_t roff = (uint64_t)r * stride;
-#pragma unroll
-                    for (int v = 0; v < V; ++v)
-                        if (col_on[v]) d[u][v] = ld_row16(lane_base[v] + roff);
-                    if (DT == DT_INT8)
-                        sb[u] = __ldg(reinterpret_cast<const float2*>(sb_base + roff));
-                }
-            }
-#pragma unroll
-            for (int u = 0; u < U; ++u) {
-                if (okmask & (1u << u)) {
-                    float wu = w[u];
-                    if (DT == DT_INT8) {
-                        acc_bias = fmaf(wu, sb[u].y, acc_bias);
-                        wu *= sb[u].x;
-                    }
-#pragma unroll
-                    for (int v = 0; v < V; ++v)
-                        if (col_on[v])
-                            accumulate<DT, WEIGHTED || DT == DT_INT8>(acc[v], d[u][v], wu);
-                }
-            }
-        }
-
-        if (more) {
-            pos = pos_next;
-        } else {
-            // ---- the bags of this slot are complete: finalise and store
-            if (slot * NG + grp < cnt) {
-                const uint32_t L = e - s;
-                float* orow = p.out + (bag0 + orig) * (int64_t)p.sumD + m.D_off;
-#pragma unroll
-                for (int v = 0; v < V; ++v) {
-                    if (!col_on[v]) continue;
-                    float* o = orow + (size_t)(vec0 + v * G + lig) * NACC;
-#pragma unroll
-                    for (int a = 0; a < NACC; ++a) {
-                        float x = acc[v][a];
-                        if (DT == DT_INT8) x += acc_bias;
-                        if (p.mean && L > 0) x = __fdiv_rn(x, (float)L);
-                        acc[v][a] = x;
-                    }
-#pragma unroll
-                    for (int a = 0; a < NACC; a += 4)
-                        st_stream16(o + a, acc[v][a], acc[v][a + 1], acc[v][a + 2], acc[v][a + 3]);
-                }
-            }
-            ++slot;
-            if (slot >= nslots) break;
-            s = s2;
-            e = e2;
-            orig = orig2;
-            pos = s;
-            acc_bias = 0.0f;
-#pragma unroll
-            for (int v = 0; v < V; ++v)
-#pragma unroll
-                for (int a = 0; a < NACC; ++a) acc[v][a] = 0.0f;
-        }
-        cur_r = nxt_r;
-        cur_w = nxt_w;
-    }
-}
-
-// ------------------------------------------------------------------ one item, staged in smem
-// Same work split as process_item, but rows travel with cp.async into a per-warp ring of
-// kStages stages (kStageVecs 16-byte vectors per lane each) and are consumed one stage behind.
-// Row fetches therefore stay in flight across batch, id-chunk and bag boundaries, and hold no
-// registers.  Every lane reads back only the slots it copied itself, so its own wait_group is
-// all the synchronisation the row data needs.
+// vec0: first 16-byte vector of the column tile this call covers (0 unless the row is wider than
+// 64 vectors).  Rows travel with cp.async into this warp's ring `wbuf` of kStages stages
+// (kStageVecs 16-byte vectors per lane each) and are consumed one stage behind.  Every lane reads
+// back only the slots it copied itself, so its own wait_group is all the synchronisation the row
+// data needs (the int8 scale/bias slots are shared by a group and take a __syncwarp).
 #ifndef EBAG_STAGE_VECS
 #define EBAG_STAGE_VECS 4
 #endif
@@ -455,7 +216,7 @@ struct IdChunk {          // ids of up to G consecutive entries of the bags one 
 };
 
 template <int DT, bool WEIGHTED, int V>
-__device__ __forceinline__ void process_item_async(const FwdParams& p, const TableMeta& m,
+__device__ __forceinline__ void process_item(const FwdParams& p, const TableMeta& m,
                                                    const char* __restrict__ tbase, int t,
                                                    int64_t bag0, int cnt, int vec0, int lane,
                                                    unsigned& n_oob, unsigned& n_bad,
@@ -730,12 +491,10 @@ ebag_fwd_kernel(const FwdParams p) {
     int* item_bags = smem_i + p.T + 1;                         // [T]   bags per item of each table
     float* bag_bytes = reinterpret_cast<float*>(item_bags);    // [T]   (first pass) bytes per bag
     __shared__ float total_bytes;
-#ifdef EBAG_ASYNC
-    __shared__ uint4 stage_buf[kWarps * kStages * kStageVecs * 32];
+    __shared__ uint4 stage_buf[kWarps * kStages * kStageVecs * 32];          // 4 KB per warp
     __shared__ float2 sb_buf[DT == DT_INT8 ? kWarps * kStages * kStageVecs * 8 : 1];
     uint4* wbuf = stage_buf + (threadIdx.x >> 5) * (kStages * kStageVecs * 32);
     float2* sbbuf = sb_buf + (DT == DT_INT8 ? (threadIdx.x >> 5) * (kStages * kStageVecs * 8) : 0);
-#endif
     const int tid = threadIdx.x;
     const int lane = tid & 31;
 
@@ -808,22 +567,13 @@ ebag_fwd_kernel(const FwdParams p) {
         const int cnt = rest < ib ? (int)rest : ib;
         const char* tbase = static_cast<const char*>(p.tables[t]);
 
-#ifdef EBAG_ASYNC
         if (m.V == 1) {
-            process_item_async<DT, WEIGHTED, 1>(p, m, tbase, t, bag0, cnt, 0, lane, n_oob, n_bad, wbuf, sbbuf);
-        } else {
-            for (int vec0 = 0; vec0 < m.nvec; vec0 += 64)
-                process_item_async<DT, WEIGHTED, 2>(p, m, tbase, t, bag0, cnt, vec0, lane, n_oob, n_bad, wbuf, sbbuf);
-        }
-#else
-        if (m.V == 1) {
-            process_item<DT, WEIGHTED, 1>(p, m, tbase, t, bag0, cnt, 0, lane, n_oob, n_bad);
+            process_item<DT, WEIGHTED, 1>(p, m, tbase, t, bag0, cnt, 0, lane, n_oob, n_bad, wbuf, sbbuf);
         } else {
             // rows above 512 bytes: two vectors per lane, 1 KB column tiles
             for (int vec0 = 0; vec0 < m.nvec; vec0 += 64)
-                process_item<DT, WEIGHTED, 2>(p, m, tbase, t, bag0, cnt, vec0, lane, n_oob, n_bad);
+                process_item<DT, WEIGHTED, 2>(p, m, tbase, t, bag0, cnt, vec0, lane, n_oob, n_bad, wbuf, sbbuf);
         }
-#endif
         q = __shfl_sync(0xffffffffu, q_next, 0);
     }
 
