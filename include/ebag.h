@@ -140,6 +140,34 @@ ebag_status ebag_pack_int8_rowwise(const int8_t* q, const float* scale, const fl
                                    int64_t rows, int32_t D, void* dst, ebag_stream stream);
 
 /*
+ * MapId transform (paper Sec. 5.4.1 "MapId Transform"): `mapping` is a sorted (strictly
+ * increasing) list of the m known ids; every value becomes its 1-based position in it, 0 if it
+ * is not in it: insertion index by binary search, clamp to m-1, compare.
+ *   values, out  device int64 [n] (out may not alias values);  mapping  device int64 [m], m < 2^31
+ * m == 0 maps everything to 0.  One kernel on `stream`, no allocation.
+ */
+ebag_status ebag_mapid(const int64_t* values, int64_t n, const int64_t* mapping, int64_t m,
+                       int64_t* out, ebag_stream stream);
+
+/*
+ * The pooled forward with the MapId transform fused into the id fetch: `values` holds RAW ids
+ * (same jagged layout as `indices` of ebag_forward); table t looks every one up in mappings[t]
+ * (host array [T] of device pointers to sorted int64 lists, mapping_len[t] entries each, host
+ * array [T]) and pools row 0 for unknown ids, row k for the k-th known id.  Table t therefore
+ * has mapping_len[t] + 1 rows (create the handle with those row counts); a mapped id beyond the
+ * table's rows is skipped and counted like any out-of-range id.  Everything else as
+ * ebag_forward: one launch, no allocation, no synchronisation; the mapping arrays are read
+ * before the call returns.  This is the producer of embedding ids the paper's preprocessing
+ * section describes, placed directly in front of the gather so that the mapped ids never travel
+ * through memory.
+ */
+ebag_status ebag_forward_mapid(ebag_tbe* h, const void* const* tables, const int32_t* D,
+                               const int64_t* values, int64_t n_values, const int64_t* offsets,
+                               const float* per_sample_weights, const int64_t* const* mappings,
+                               const int64_t* mapping_len, int64_t B, ebag_mode mode, float* out,
+                               ebag_stream stream);
+
+/*
  * The same forward without a handle and without any allocation (the paper has no counterpart;
  * this exists for deployment).  Some callers cannot allocate device memory when they need a
  * forward: code that runs inside a memory pool whose owner forbids side allocations, a plugin in

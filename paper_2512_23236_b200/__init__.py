@@ -31,6 +31,9 @@ SIGNATURES = {
     "ebag_forward_host": (_int, [_vp, _vp, _vp, _vp, _i64, _vp, _vp, _i64, _int, _vp, _vp]),
     "ebag_forward_noalloc": (_int, [_i32, _vp, _vp, _int, _vp, _vp, _i64, _vp, _vp, _i64, _int, _vp,
                                     _vp, _vp]),
+    "ebag_mapid": (_int, [_vp, _i64, _vp, _i64, _vp, _vp]),
+    "ebag_forward_mapid": (_int, [_vp, _vp, _vp, _vp, _i64, _vp, _vp, _vp, _vp, _i64, _int, _vp,
+                                  _vp]),
     "ebag_last_status": (_int, [_vp, _vp, _vp, _vp]),
     "ebag_pack_int8_rowwise": (_int, [_vp, _vp, _vp, _i64, _i32, _vp, _vp]),
     "ebag_set_param": (_int, [_vp, ctypes.c_char_p, _i64]),
@@ -129,6 +132,32 @@ def ebag_forward_noalloc(rows: Sequence[int], D: Sequence[int], dtype: int,
     _check(st, "ebag_forward_noalloc")
 
 
+def ebag_mapid(values, mapping, out=None, stream=None):
+    """MapId transform of a device int64 tensor against a sorted device int64 mapping."""
+    import torch
+    if out is None:
+        out = torch.empty_like(values)
+    with torch.cuda.device(values.device):
+        st = lib().ebag_mapid(_ptr(values), int(values.numel()), _ptr(mapping), int(mapping.numel()),
+                              _ptr(out), _stream_ptr(stream))
+    _check(st, "ebag_mapid")
+    return out
+
+
+def ebag_forward_mapid(h: int, table_ptrs: Sequence[int], D: Sequence[int], values_ptr,
+                       n_values: int, offsets_ptr, weights_ptr, mapping_ptrs: Sequence[int],
+                       mapping_len: Sequence[int], B: int, mode: int, out_ptr, stream_ptr) -> None:
+    T = len(table_ptrs)
+    tp = (ctypes.c_void_p * T)(*[int(p) if p else None for p in table_ptrs])
+    d = (ctypes.c_int32 * T)(*[int(x) for x in D])
+    mp = (ctypes.c_void_p * T)(*[int(p) if p else None for p in mapping_ptrs])
+    ml = (ctypes.c_int64 * T)(*[int(x) for x in mapping_len])
+    st = lib().ebag_forward_mapid(h, ctypes.cast(tp, _vp), ctypes.cast(d, _vp), values_ptr,
+                                  n_values, offsets_ptr, weights_ptr, ctypes.cast(mp, _vp),
+                                  ctypes.cast(ml, _vp), B, mode, out_ptr, stream_ptr)
+    _check(st, "ebag_forward_mapid")
+
+
 def ebag_last_status(h: int, stream_ptr) -> tuple:
     """(status, n_oob, n_bad_offsets); synchronises the stream."""
     a, b = ctypes.c_int64(0), ctypes.c_int64(0)
@@ -207,6 +236,18 @@ class TBE:
         ebag_forward(self._h, [t.data_ptr() for t in tables], self.D, _ptr(indices),
                      int(indices.numel()), _ptr(offsets), _ptr(per_sample_weights), B, mode,
                      _ptr(out), _stream_ptr(stream))
+        return out
+
+    def forward_mapid(self, tables: List, values, offsets, mappings: List, B: int,
+                      mode: int = EBAG_SUM, per_sample_weights=None, out=None, stream=None):
+        """Raw ids in: table t maps them through the sorted device tensor mappings[t] first."""
+        import torch
+        if out is None:
+            out = torch.empty((B, self.sumD), dtype=torch.float32, device=values.device)
+        ebag_forward_mapid(self._h, [t.data_ptr() for t in tables], self.D, _ptr(values),
+                           int(values.numel()), _ptr(offsets), _ptr(per_sample_weights),
+                           [m.data_ptr() for m in mappings], [int(m.numel()) for m in mappings], B,
+                           mode, _ptr(out), _stream_ptr(stream))
         return out
 
     def forward_host(self, tables: List, indices, offsets, B: int, mode: int = EBAG_SUM,

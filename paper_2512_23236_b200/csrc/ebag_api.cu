@@ -43,13 +43,14 @@ struct ebag_tbe {
     TableMeta* d_meta = nullptr;
     Queue* d_queue = nullptr;
     Status* d_status = nullptr;
-    // table pointers: cached on the device, re-sent only when the caller's array changes
+    // per-call pointer block [tables T][mappings T][mapping lengths T]: cached on the device,
+    // re-sent only when the caller's arrays change
     const void** d_tables[kTableSlots] = {};
     const void** h_tables[kTableSlots] = {};       // pinned
     cudaEvent_t slot_event[kTableSlots] = {};
     bool slot_busy[kTableSlots] = {};
     int slot = -1;
-    int occupancy[2] = {0, 0};                     // CTAs per SM, [unweighted, weighted]
+    int occupancy[2][2] = {};                      // CTAs per SM, [plain, MapId][unweighted, weighted]
     uint32_t item_bytes = 32768;
     int ctas_per_sm = 0;                           // 0: occupancy limit
     int64_t launches = 0;
@@ -108,21 +109,22 @@ void free_handle(ebag_tbe* h) {
 
 size_t fwd_smem_bytes(int T) { return (size_t)(2 * T + 1) * sizeof(int); }
 
-cudaError_t launch_fwd(int dtype, const FwdParams& p, bool w, int grid, size_t smem, cudaStream_t s) {
+cudaError_t launch_fwd(int dtype, const FwdParams& p, bool w, bool mapid, int grid, size_t smem,
+                       cudaStream_t s) {
     switch (dtype) {
-        case EBAG_F32: return launch_fwd_f32(p, w, grid, smem, s);
-        case EBAG_F16: return launch_fwd_f16(p, w, grid, smem, s);
-        case EBAG_BF16: return launch_fwd_bf16(p, w, grid, smem, s);
-        default: return launch_fwd_int8(p, w, grid, smem, s);
+        case EBAG_F32: return launch_fwd_f32(p, w, mapid, grid, smem, s);
+        case EBAG_F16: return launch_fwd_f16(p, w, mapid, grid, smem, s);
+        case EBAG_BF16: return launch_fwd_bf16(p, w, mapid, grid, smem, s);
+        default: return launch_fwd_int8(p, w, mapid, grid, smem, s);
     }
 }
 
-cudaError_t occupancy_fwd(int dtype, bool w, size_t smem, int* n) {
+cudaError_t occupancy_fwd(int dtype, bool w, bool mapid, size_t smem, int* n) {
     switch (dtype) {
-        case EBAG_F32: return occupancy_fwd_f32(w, smem, n);
-        case EBAG_F16: return occupancy_fwd_f16(w, smem, n);
-        case EBAG_BF16: return occupancy_fwd_bf16(w, smem, n);
-        default: return occupancy_fwd_int8(w, smem, n);
+        case EBAG_F32: return occupancy_fwd_f32(w, mapid, smem, n);
+        case EBAG_F16: return occupancy_fwd_f16(w, mapid, smem, n);
+        case EBAG_BF16: return occupancy_fwd_bf16(w, mapid, smem, n);
+        default: return occupancy_fwd_int8(w, mapid, smem, n);
     }
 }
 
@@ -144,11 +146,19 @@ ebag_status check_forward_args(ebag_tbe* h, const void* const* tables, const int
     return EBAG_OK;
 }
 
-// Device copy of the caller's table-pointer array; re-sent only when it changed.
-ebag_status stage_tables(ebag_tbe* h, const void* const* tables, cudaStream_t stream,
-                         const void* const** d_out) {
-    const size_t bytes = (size_t)h->T * sizeof(void*);
-    if (h->slot >= 0 && std::memcmp(h->h_tables[h->slot], tables, bytes) == 0) {
+// Device copy of the caller's pointer block (tables, and for the MapId variant the mapping
+// pointers and lengths); re-sent only when it changed.
+ebag_status stage_tables(ebag_tbe* h, const void* const* tables, const int64_t* const* mappings,
+                         const int64_t* mapping_len, cudaStream_t stream, const void* const** d_out) {
+    const int T = h->T;
+    const size_t bytes = (size_t)3 * T * sizeof(void*);
+    std::vector<const void*> blob(3 * (size_t)T, nullptr);
+    for (int t = 0; t < T; ++t) {
+        blob[t] = tables[t];
+        if (mappings) blob[T + t] = mappings[t];
+        if (mapping_len) std::memcpy(&blob[2 * T + t], &mapping_len[t], sizeof(int64_t));
+    }
+    if (h->slot >= 0 && std::memcmp(h->h_tables[h->slot], blob.data(), bytes) == 0) {
         *d_out = h->d_tables[h->slot];
         return EBAG_OK;
     }
@@ -157,7 +167,7 @@ ebag_status stage_tables(ebag_tbe* h, const void* const* tables, cudaStream_t st
         EBAG_CUDA(h, cudaEventSynchronize(h->slot_event[s]));
         h->slot_busy[s] = false;
     }
-    std::memcpy(h->h_tables[s], tables, bytes);
+    std::memcpy(h->h_tables[s], blob.data(), bytes);
     EBAG_CUDA(h, cudaMemcpyAsync(h->d_tables[s], h->h_tables[s], bytes, cudaMemcpyHostToDevice, stream));
     EBAG_CUDA(h, cudaEventRecord(h->slot_event[s], stream));
     h->slot_busy[s] = true;
@@ -171,13 +181,14 @@ ebag_status stage_tables(ebag_tbe* h, const void* const* tables, cudaStream_t st
 ebag_status forward_device(ebag_tbe* h, const void* const* tables, const int64_t* indices,
                            int64_t n_indices, const int64_t* offsets, const float* weights,
                            int64_t B, int64_t b0, int64_t b1, ebag_mode mode, float* out,
-                           cudaStream_t stream) {
+                           cudaStream_t stream, const int64_t* const* mappings = nullptr,
+                           const int64_t* mapping_len = nullptr) {
     if (b1 <= b0) return EBAG_OK;
     if (((uintptr_t)out & 15u) || ((uintptr_t)indices & 7u) || ((uintptr_t)offsets & 7u) ||
         ((uintptr_t)weights & 3u))
         return EBAG_ERR_INVALID_ARG;
     const void* const* d_tables = nullptr;
-    ebag_status st = stage_tables(h, tables, stream, &d_tables);
+    ebag_status st = stage_tables(h, tables, mappings, mapping_len, stream, &d_tables);
     if (st != EBAG_OK) return st;
 
     FwdParams p;
@@ -189,6 +200,8 @@ ebag_status forward_device(ebag_tbe* h, const void* const* tables, const int64_t
     p.out = out + b0 * (int64_t)h->sumD;
     p.queue = h->d_queue;
     p.status = h->d_status;
+    p.mappings = reinterpret_cast<const int64_t* const*>(d_tables + h->T);
+    p.mapping_len = reinterpret_cast<const int64_t*>(d_tables + 2 * h->T);
     p.n_indices = n_indices;
     p.B = b1 - b0;
     p.off_stride = B;
@@ -197,10 +210,11 @@ ebag_status forward_device(ebag_tbe* h, const void* const* tables, const int64_t
     p.mean = mode == EBAG_MEAN ? 1 : 0;
     p.item_bytes = h->item_bytes;
     const bool w = weights != nullptr;
-    int per_sm = h->occupancy[w ? 1 : 0];
+    const bool mapid = mappings != nullptr;
+    int per_sm = h->occupancy[mapid ? 1 : 0][w ? 1 : 0];
     if (h->ctas_per_sm > 0 && h->ctas_per_sm < per_sm) per_sm = h->ctas_per_sm;
     const int grid = h->num_sms * per_sm;
-    EBAG_CUDA(h, launch_fwd(h->dtype, p, w, grid, fwd_smem_bytes(h->T), stream));
+    EBAG_CUDA(h, launch_fwd(h->dtype, p, w, mapid, grid, fwd_smem_bytes(h->T), stream));
     ++h->launches;
     return EBAG_OK;
 }
@@ -243,9 +257,52 @@ __global__ void pack_int8_rowwise_kernel(const int8_t* __restrict__ q, const flo
     }
 }
 
+// MapId alone: one thread per value, coalesced in and out.
+__global__ void mapid_kernel(const int64_t* __restrict__ values, int64_t n,
+                             const int64_t* __restrict__ mapping, uint32_t mlen, int steps,
+                             int64_t* __restrict__ out) {
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n;
+         i += (int64_t)gridDim.x * blockDim.x)
+        out[i] = map_id(mapping, mlen, steps, __ldcs(reinterpret_cast<const long long*>(values + i)));
+}
+
 }  // namespace
 
 extern "C" {
+
+ebag_status ebag_mapid(const int64_t* values, int64_t n, const int64_t* mapping, int64_t m,
+                       int64_t* out, ebag_stream stream) {
+    if (n < 0 || m < 0 || m >= (1ll << 31)) return EBAG_ERR_INVALID_ARG;
+    if (n == 0) return EBAG_OK;
+    if (!values || !out || (m > 0 && !mapping)) return EBAG_ERR_INVALID_ARG;
+    int steps = 0;
+    while ((1ll << steps) <= m) ++steps;             // bit length of m
+    int64_t blocks = (n + 255) / 256;
+    if (blocks > 148 * 16) blocks = 148 * 16;
+    mapid_kernel<<<(int)blocks, 256, 0, (cudaStream_t)stream>>>(values, n, mapping, (uint32_t)m, steps, out);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(nullptr, e);
+    return EBAG_OK;
+}
+
+ebag_status ebag_forward_mapid(ebag_tbe* h, const void* const* tables, const int32_t* D,
+                               const int64_t* values, int64_t n_values, const int64_t* offsets,
+                               const float* per_sample_weights, const int64_t* const* mappings,
+                               const int64_t* mapping_len, int64_t B, ebag_mode mode, float* out,
+                               ebag_stream stream) {
+    ebag_status st = check_forward_args(h, tables, D, values, n_values, offsets, per_sample_weights,
+                                        B, mode, out);
+    if (st != EBAG_OK) return st;
+    if (!mappings || !mapping_len) return EBAG_ERR_INVALID_ARG;
+    for (int t = 0; t < h->T; ++t) {
+        if (mapping_len[t] < 0 || mapping_len[t] >= (1ll << 31)) return EBAG_ERR_INVALID_ARG;
+        if (mapping_len[t] > 0 && (!mappings[t] || ((uintptr_t)mappings[t] & 7u))) return EBAG_ERR_INVALID_ARG;
+    }
+    DeviceGuard guard(h->device);
+    if (!guard.ok) return EBAG_ERR_CUDA;
+    return forward_device(h, tables, values, n_values, offsets, per_sample_weights, B, 0, B, mode,
+                          out, (cudaStream_t)stream, mappings, mapping_len);
+}
 
 int64_t ebag_row_stride(ebag_dtype dtype, int32_t D) {
     if (D <= 0 || dtype < EBAG_F32 || dtype > EBAG_INT8_ROWWISE) return -1;
@@ -307,8 +364,8 @@ ebag_status ebag_create_tbe(int32_t T, const int64_t* rows, const int32_t* D, eb
         EBAG_CUDA(h, cudaMalloc((void**)&h->d_status, sizeof(Status)));
         EBAG_CUDA(h, cudaMemset(h->d_status, 0, sizeof(Status)));
         for (int i = 0; i < kTableSlots; ++i) {
-            EBAG_CUDA(h, cudaMalloc((void**)&h->d_tables[i], sizeof(void*) * T));
-            EBAG_CUDA(h, cudaMallocHost((void**)&h->h_tables[i], sizeof(void*) * T));
+            EBAG_CUDA(h, cudaMalloc((void**)&h->d_tables[i], sizeof(void*) * 3 * T));
+            EBAG_CUDA(h, cudaMallocHost((void**)&h->h_tables[i], sizeof(void*) * 3 * T));
             EBAG_CUDA(h, cudaEventCreateWithFlags(&h->slot_event[i], cudaEventDisableTiming));
         }
         EBAG_CUDA(h, cudaStreamCreateWithFlags(&h->s_h2d, cudaStreamNonBlocking));
@@ -319,10 +376,11 @@ ebag_status ebag_create_tbe(int32_t T, const int64_t* rows, const int32_t* D, eb
             EBAG_CUDA(h, cudaEventCreateWithFlags(&h->ev_in[i], cudaEventDisableTiming));
             EBAG_CUDA(h, cudaEventCreateWithFlags(&h->ev_done[i], cudaEventDisableTiming));
         }
-        for (int w = 0; w < 2; ++w) {
-            EBAG_CUDA(h, occupancy_fwd(dtype, w != 0, fwd_smem_bytes(T), &h->occupancy[w]));
-            if (h->occupancy[w] < 1) h->occupancy[w] = 1;
-        }
+        for (int mp = 0; mp < 2; ++mp)
+            for (int w = 0; w < 2; ++w) {
+                EBAG_CUDA(h, occupancy_fwd(dtype, w != 0, mp != 0, fwd_smem_bytes(T), &h->occupancy[mp][w]));
+                if (h->occupancy[mp][w] < 1) h->occupancy[mp][w] = 1;
+            }
         return EBAG_OK;
     };
     st = body();

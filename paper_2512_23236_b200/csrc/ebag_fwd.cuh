@@ -72,6 +72,8 @@ struct FwdParams {
     float* out;
     Queue* queue;
     Status* status;
+    const int64_t* const* mappings;   // MapId variant: device [T] sorted id lists (else unused)
+    const int64_t* mapping_len;       // MapId variant: device [T] their lengths
     int64_t n_indices;
     int64_t B;                   // bags per table in this launch
     int64_t off_stride;          // offsets of table t start at offsets[t * off_stride] (B for a
@@ -191,6 +193,26 @@ __device__ __forceinline__ uint32_t warp_sort_desc(uint32_t v, int lane) {
     return v;
 }
 
+// ------------------------------------------------------------------ MapId (paper Sec. 5.4.1)
+// 1-based position of v in the sorted list M, 0 if v is not in it: insertion index by binary
+// search, clamp to the last entry, compare.  The search runs a fixed number of branch-free
+// halving steps (the bit length of |M|), as the paper's kernel does with its fixed 20.
+__device__ __forceinline__ int64_t map_id(const int64_t* __restrict__ M, uint32_t mlen, int steps,
+                                          int64_t v) {
+    if (mlen == 0) return 0;
+    uint32_t lo = 0, hi = mlen;                      // first position with M[pos] >= v is in [lo, hi]
+    for (int s = 0; s < steps; ++s) {
+        const uint32_t mid = (lo + hi) >> 1;
+        const int64_t mv = __ldg(M + (mid < mlen ? mid : mlen - 1));
+        const bool active = lo < hi;
+        const bool right = mv < v;
+        lo = (active && right) ? mid + 1 : lo;
+        hi = (active && !right) ? mid : hi;
+    }
+    const uint32_t idx = lo < mlen ? lo : mlen - 1;
+    return __ldg(M + idx) == v ? (int64_t)idx + 1 : 0;
+}
+
 // ------------------------------------------------------------------ one item, staged in smem
 // Bags [bag0, bag0 + cnt) of table t; cnt <= 32.  V vectors per lane; the lanes per row (G) are
 // a run-time property of the table so that one instance of this code serves every row width.
@@ -216,7 +238,7 @@ struct IdChunk {          // ids of up to G consecutive entries of the bags one 
     bool valid;
 };
 
-template <int DT, bool WEIGHTED, int V>
+template <int DT, bool WEIGHTED, bool MAPID, int V>
 __device__ __forceinline__ void process_item(const FwdParams& p, const TableMeta& m,
                                                    const char* __restrict__ tbase, int t,
                                                    int64_t bag0, int cnt, int vec0, int lane,
@@ -265,14 +287,19 @@ __device__ __forceinline__ void process_item(const FwdParams& p, const TableMeta
     const char* sb_base = tbase + m.D;
     const int nslots = (cnt + NG - 1) >> (5 - m.g_log2);
 
+    const int64_t* __restrict__ map_ptr = MAPID ? p.mappings[t] : nullptr;
+    const int64_t map_len64 = MAPID ? p.mapping_len[t] : 0;
+    const uint32_t map_len = (uint32_t)(map_len64 < 0 ? 0 : map_len64);
+    const int map_steps = 32 - __clz(map_len);
     auto load_chunk = [&](uint32_t pos, uint32_t end, uint32_t& ridx, float& w) {
         ridx = kInvalidRow;
         w = 0.0f;
         const uint32_t i = pos + lig;
         if (i < end) {
-            const int64_t r = ld_stream_i64(idx_base + i);
+            int64_t r = ld_stream_i64(idx_base + i);
             float wl = 1.0f;
             if (WEIGHTED) wl = ld_stream_f32(w_base + i);
+            if (MAPID) r = map_id(map_ptr, map_len, map_steps, r);     // raw id -> row
             if ((uint64_t)r < rows) {
                 ridx = (uint32_t)r;
                 w = wl;
@@ -484,7 +511,7 @@ __device__ __forceinline__ void process_item(const FwdParams& p, const TableMeta
 }
 
 // ------------------------------------------------------------------ the kernel
-template <int DT, bool WEIGHTED>
+template <int DT, bool WEIGHTED, bool MAPID>
 __global__ void __launch_bounds__(kThreads, EBAG_MIN_BLOCKS)
 ebag_fwd_kernel(const FwdParams p) {
     extern __shared__ int smem_i[];
@@ -571,11 +598,11 @@ ebag_fwd_kernel(const FwdParams p) {
         const char* tbase = static_cast<const char*>(p.tables[t]);
 
         if (m.V == 1) {
-            process_item<DT, WEIGHTED, 1>(p, m, tbase, t, bag0, cnt, 0, lane, n_oob, n_bad, wbuf, sbbuf);
+            process_item<DT, WEIGHTED, MAPID, 1>(p, m, tbase, t, bag0, cnt, 0, lane, n_oob, n_bad, wbuf, sbbuf);
         } else {
             // rows above 512 bytes: two vectors per lane, 1 KB column tiles
             for (int vec0 = 0; vec0 < m.nvec; vec0 += 64)
-                process_item<DT, WEIGHTED, 2>(p, m, tbase, t, bag0, cnt, vec0, lane, n_oob, n_bad, wbuf, sbbuf);
+                process_item<DT, WEIGHTED, MAPID, 2>(p, m, tbase, t, bag0, cnt, vec0, lane, n_oob, n_bad, wbuf, sbbuf);
         }
         q = __shfl_sync(0xffffffffu, q_next, 0);
     }
@@ -600,27 +627,33 @@ ebag_fwd_kernel(const FwdParams p) {
 }
 
 // one launcher per dtype, each compiled in its own translation unit
-cudaError_t launch_fwd_f32(const FwdParams& p, bool weighted, int grid, size_t smem, cudaStream_t s);
-cudaError_t launch_fwd_f16(const FwdParams& p, bool weighted, int grid, size_t smem, cudaStream_t s);
-cudaError_t launch_fwd_bf16(const FwdParams& p, bool weighted, int grid, size_t smem, cudaStream_t s);
-cudaError_t launch_fwd_int8(const FwdParams& p, bool weighted, int grid, size_t smem, cudaStream_t s);
-cudaError_t occupancy_fwd_f32(bool weighted, size_t smem, int* ctas_per_sm);
-cudaError_t occupancy_fwd_f16(bool weighted, size_t smem, int* ctas_per_sm);
-cudaError_t occupancy_fwd_bf16(bool weighted, size_t smem, int* ctas_per_sm);
-cudaError_t occupancy_fwd_int8(bool weighted, size_t smem, int* ctas_per_sm);
+#define EBAG_DECLARE_LAUNCHERS(NAME)                                                             \
+    cudaError_t launch_fwd_##NAME(const FwdParams& p, bool weighted, bool mapid, int grid,        \
+                                  size_t smem, cudaStream_t s);                                  \
+    cudaError_t occupancy_fwd_##NAME(bool weighted, bool mapid, size_t smem, int* ctas_per_sm);
+EBAG_DECLARE_LAUNCHERS(f32)
+EBAG_DECLARE_LAUNCHERS(f16)
+EBAG_DECLARE_LAUNCHERS(bf16)
+EBAG_DECLARE_LAUNCHERS(int8)
 
 #define EBAG_DEFINE_LAUNCHERS(NAME, DT)                                                          \
-    cudaError_t launch_fwd_##NAME(const FwdParams& p, bool weighted, int grid, size_t smem,       \
-                                  cudaStream_t s) {                                              \
-        if (weighted) ebag_fwd_kernel<DT, true><<<grid, kThreads, smem, s>>>(p);                  \
-        else ebag_fwd_kernel<DT, false><<<grid, kThreads, smem, s>>>(p);                          \
+    cudaError_t launch_fwd_##NAME(const FwdParams& p, bool weighted, bool mapid, int grid,        \
+                                  size_t smem, cudaStream_t s) {                                 \
+        if (mapid) {                                                                             \
+            if (weighted) ebag_fwd_kernel<DT, true, true><<<grid, kThreads, smem, s>>>(p);        \
+            else ebag_fwd_kernel<DT, false, true><<<grid, kThreads, smem, s>>>(p);                \
+        } else {                                                                                 \
+            if (weighted) ebag_fwd_kernel<DT, true, false><<<grid, kThreads, smem, s>>>(p);       \
+            else ebag_fwd_kernel<DT, false, false><<<grid, kThreads, smem, s>>>(p);               \
+        }                                                                                        \
         return cudaGetLastError();                                                               \
     }                                                                                            \
-    cudaError_t occupancy_fwd_##NAME(bool weighted, size_t smem, int* n) {                        \
-        return weighted ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(                         \
-                              n, ebag_fwd_kernel<DT, true>, kThreads, smem)                       \
-                        : cudaOccupancyMaxActiveBlocksPerMultiprocessor(                         \
-                              n, ebag_fwd_kernel<DT, false>, kThreads, smem);                     \
+    cudaError_t occupancy_fwd_##NAME(bool weighted, bool mapid, size_t smem, int* n) {            \
+        const void* k = mapid ? (weighted ? (const void*)ebag_fwd_kernel<DT, true, true>          \
+                                          : (const void*)ebag_fwd_kernel<DT, false, true>)        \
+                              : (weighted ? (const void*)ebag_fwd_kernel<DT, true, false>         \
+                                          : (const void*)ebag_fwd_kernel<DT, false, false>);      \
+        return cudaOccupancyMaxActiveBlocksPerMultiprocessor(n, k, kThreads, smem);              \
     }
 
 }  // namespace ebag

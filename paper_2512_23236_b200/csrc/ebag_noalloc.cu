@@ -75,19 +75,19 @@ size_t fwd_smem_bytes(int T) { return (size_t)(2 * T + 1) * sizeof(int); }
 
 cudaError_t launch(int dtype, const FwdParams& p, bool w, int grid, size_t smem, cudaStream_t s) {
     switch (dtype) {
-        case EBAG_F32: return launch_fwd_f32(p, w, grid, smem, s);
-        case EBAG_F16: return launch_fwd_f16(p, w, grid, smem, s);
-        case EBAG_BF16: return launch_fwd_bf16(p, w, grid, smem, s);
-        default: return launch_fwd_int8(p, w, grid, smem, s);
+        case EBAG_F32: return launch_fwd_f32(p, w, false, grid, smem, s);
+        case EBAG_F16: return launch_fwd_f16(p, w, false, grid, smem, s);
+        case EBAG_BF16: return launch_fwd_bf16(p, w, false, grid, smem, s);
+        default: return launch_fwd_int8(p, w, false, grid, smem, s);
     }
 }
 
 cudaError_t occupancy(int dtype, bool w, size_t smem, int* n) {
     switch (dtype) {
-        case EBAG_F32: return occupancy_fwd_f32(w, smem, n);
-        case EBAG_F16: return occupancy_fwd_f16(w, smem, n);
-        case EBAG_BF16: return occupancy_fwd_bf16(w, smem, n);
-        default: return occupancy_fwd_int8(w, smem, n);
+        case EBAG_F32: return occupancy_fwd_f32(w, false, smem, n);
+        case EBAG_F16: return occupancy_fwd_f16(w, false, smem, n);
+        case EBAG_BF16: return occupancy_fwd_bf16(w, false, smem, n);
+        default: return occupancy_fwd_int8(w, false, smem, n);
     }
 }
 
@@ -192,6 +192,8 @@ extern "C" ebag_status ebag_forward_noalloc(int32_t T, const int64_t* rows, cons
     p.weights = per_sample_weights;
     p.out = out;
     p.queue = &st->scratch->queue;
+    p.mappings = nullptr;
+    p.mapping_len = nullptr;
     p.status = status_counts ? reinterpret_cast<Status*>(status_counts) : &st->scratch->status;
     p.n_indices = n_indices;
     p.B = B;

@@ -1,0 +1,113 @@
+"""GPU parity of the MapId transform (paper Sec. 5.4.1) and of the pooled forward with MapId
+fused into the id fetch, against the CPU oracle.  Integer work: bit-exact."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2512_23236_b200 as eb
+from golden_io import read_fixture
+from oracle import ebag_oracle as orc
+from oracle import mapid_oracle as mo
+from paper_2512_23236_b200 import workloads as wl
+
+import parity_util as pu
+
+pytestmark = pytest.mark.gpu
+
+
+def _gpu_mapid(values, mapping):
+    v = torch.from_numpy(np.ascontiguousarray(values, dtype=np.int64)).cuda()
+    m = torch.from_numpy(np.ascontiguousarray(mapping, dtype=np.int64)).cuda()
+    return eb.ebag_mapid(v, m).cpu().numpy()
+
+
+def test_paper_worked_example_on_gpu():
+    fx = read_fixture("mapid_example.txt")
+    got = _gpu_mapid(fx["values"].astype(np.int64), fx["mapping"].astype(np.int64))
+    assert np.array_equal(got, fx["output"].astype(np.int64))
+
+
+@pytest.mark.parametrize("m,n", [(1, 1000), (2, 1000), (5, 77), (100, 10_000), (10_000, 50_000),
+                                 (1_048_576, 300_000), (1_000_003, 300_001)])
+def test_mapid_matches_oracle_bit_for_bit(m, n):
+    """Includes the paper's shapes (unique ids x batch = 100 x 10000 ... 10000 x 50000), a full
+    2^20-entry mapping, odd sizes, members, non-members, below-range and above-range values."""
+    rng = np.random.default_rng(m + n)
+    mapping = np.sort(rng.choice(np.arange(-2 * m, 4 * m + 10, dtype=np.int64), size=m, replace=False))
+    values = rng.integers(-3 * m - 5, 5 * m + 20, size=n).astype(np.int64)
+    values[::3] = mapping[rng.integers(0, m, size=values[::3].shape[0])]      # plenty of members
+    values[:2] = [np.iinfo(np.int64).min, np.iinfo(np.int64).max]
+    assert np.array_equal(_gpu_mapid(values, mapping), mo.mapid(values, mapping))
+
+
+def test_mapid_degenerate_sizes():
+    assert _gpu_mapid(np.zeros(0, np.int64), np.array([1, 2, 3])).shape == (0,)
+    v = torch.tensor([5, 6, 7], dtype=torch.int64, device="cuda")
+    empty = torch.zeros(0, dtype=torch.int64, device="cuda")
+    assert torch.equal(eb.ebag_mapid(v, empty).cpu(), torch.zeros(3, dtype=torch.int64))
+
+
+@pytest.mark.parametrize("dtype", [wl.F32, wl.BF16, wl.INT8_ROWWISE])
+@pytest.mark.parametrize("mode,weighted", [(wl.SUM, False), (wl.MEAN, False), (wl.SUM, True)])
+def test_fused_mapid_forward(dtype, mode, weighted):
+    rng = np.random.default_rng(31 + dtype)
+    T, B = 5, 300
+    Ds = {wl.F32: [64, 8, 256, 132, 32], wl.BF16: [64, 128, 256, 8, 1032],
+          wl.INT8_ROWWISE: [128, 16, 512, 48, 1040]}[dtype]
+    mlens = [1000, 1, 37, 5000, 64]
+    mappings = [np.sort(rng.choice(np.arange(0, 20 * m + 50, dtype=np.int64), size=m, replace=False))
+                for m in mlens]
+    rows = [m + 1 for m in mlens]
+    lengths = np.concatenate([rng.integers(0, 40, size=B) for _ in range(T)])
+    offsets = np.zeros(T * B + 1, np.int64)
+    np.cumsum(lengths, out=offsets[1:])
+    vals = []
+    for t in range(T):
+        n = int(offsets[(t + 1) * B] - offsets[t * B])
+        v = rng.integers(-10, 20 * mlens[t] + 100, size=n).astype(np.int64)          # mostly unknown
+        hit = rng.random(n) < 0.7
+        v[hit] = mappings[t][rng.integers(0, mlens[t], size=int(hit.sum()))]         # mostly known
+        vals.append(v)
+    values = np.concatenate(vals)
+    w = rng.random(values.shape[0]).astype(np.float32) if weighted else None
+    tabs = []
+    for r, d in zip(rows, Ds):
+        if dtype == wl.INT8_ROWWISE:
+            tabs.append((torch.from_numpy(rng.integers(-128, 128, size=(r, d)).astype(np.int8)),
+                         torch.from_numpy(rng.uniform(0.01, 0.03, r).astype(np.float32)),
+                         torch.from_numpy(rng.normal(0, 0.1, r).astype(np.float32))))
+        else:
+            x = torch.from_numpy(rng.standard_normal((r, d)).astype(np.float32))
+            tabs.append(x.to(torch.bfloat16) if dtype == wl.BF16 else x)
+    dev = pu.device_tables(dtype, tabs)
+    dmaps = [torch.from_numpy(m).cuda() for m in mappings]
+    tbe = eb.TBE(rows, Ds, dtype, device=torch.cuda.current_device())
+    out = torch.full((B, sum(Ds)), float("nan"), dtype=torch.float32, device="cuda")
+    tbe.forward_mapid(dev, torch.from_numpy(values).cuda(), torch.from_numpy(offsets).cuda(), dmaps, B,
+                      mode, None if w is None else torch.from_numpy(w).cuda(), out=out)
+    assert tbe.last_status() == (0, 0, 0)
+    # the fused call equals MapId followed by the plain forward, bit for bit
+    ids = torch.cat([eb.ebag_mapid(torch.from_numpy(vals[t]).cuda(), dmaps[t]) for t in range(T)])
+    out2 = tbe.forward(dev, ids, torch.from_numpy(offsets).cuda(), B, mode,
+                       None if w is None else torch.from_numpy(w).cuda())
+    assert torch.equal(out, out2)
+    tbe.close()
+    ot, sc, bi = pu.oracle_tables(dtype, tabs)
+    ref = mo.forward_mapid(ot, dtype, values, offsets, B, mappings, mode, weights=w, scales=sc, biases=bi)
+    pu.compare(out.cpu().numpy(), ref, dtype, lengths, T, B, Ds)
+
+
+def test_fused_mapid_rejects_bad_arguments_and_counts_rows_beyond_the_table():
+    tab = torch.randn(4, 8, device="cuda")                 # 4 rows: room for 3 known ids
+    mapping = torch.tensor([10, 20, 30, 40, 50], dtype=torch.int64, device="cuda")   # 5 known ids
+    vals = torch.tensor([10, 50, 99, 40], dtype=torch.int64, device="cuda")
+    off = torch.tensor([0, 4], dtype=torch.int64, device="cuda")
+    tbe = eb.TBE([4], [8], eb.EBAG_F32, device=torch.cuda.current_device())
+    out = tbe.forward_mapid([tab], vals, off, [mapping], 1)
+    # 10 -> row 1, 99 -> row 0; 50 -> row 5 and 40 -> row 4 do not exist: skipped and counted
+    assert tbe.last_status() == (eb.EBAG_ERR_INDEX_OOB, 2, 0)
+    assert torch.allclose(out[0], tab[1] + tab[0])
+    with pytest.raises(eb.EbagError):
+        eb.ebag_forward_mapid(tbe._h, [tab.data_ptr()], [8], vals.data_ptr(), 4, off.data_ptr(), None,
+                              [mapping.data_ptr()], [-1], 1, 0, out.data_ptr(), 0)
+    tbe.close()
