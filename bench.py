@@ -1,7 +1,7 @@
 #!/usr/bin/env python
 """Benchmark of the pooled embedding-bag forward on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 1..5] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 1..6] [--impl reference]
 
 One step = one pass of the whole hot path (one ebag_forward launch over all tables of the
 workload).  Default workload: 3, the batched 32-table bf16 TBE (the largest batched-table
@@ -64,23 +64,36 @@ def parse_args():
     return ap.parse_args()
 
 
+MAPID_WORKLOAD = 6     # workload 3 with 1/100 of the rows and RAW ids, MapId fused into the forward
+
+
 def make_workload(args, seed):
+    if args.workload == MAPID_WORKLOAD:
+        w = wl.make_workload(3, scale_rows=0.01 * args.scale_rows, scale_B=args.scale_b,
+                             max_tables=args.max_tables or None, seed=seed)
+        w.name = "cfg3_rows_div100_raw_ids_mapid_fused"
+        return w
     return wl.make_workload(args.workload, scale_rows=args.scale_rows, scale_B=args.scale_b,
                             max_tables=args.max_tables or None, seed=seed)
 
 
 def workload_config(w, ab, args=None):
     shrunk = args is not None and (args.max_tables or args.scale_rows != 1.0 or args.scale_b != 1.0)
+    extra = {}
+    if args is not None and args.workload == MAPID_WORKLOAD:
+        extra = {"mapid": "per table a sorted list of rows-1 known raw ids (1 k - 100 k; the paper's "
+                          "MapId sizes are 100 - 10 000); ids arrive raw and are searched in the kernel"}
     return {"workload": w.name + ("_SHRUNK" if shrunk else ""), "tables": w.T, "bags_per_table": w.B, "sum_D": w.sumD,
             "table_dtype": wl.DTYPE_NAMES[w.dtype],
             "pooling": "mean" if w.mode == wl.MEAN else ("weighted_sum" if w.weighted else "sum"),
             "lookups_per_step": ab["lookups"], "algorithmic_bytes_per_step": ab["total"],
             "index_dtype": "int64", "seed": w.seed,
-            "l2": f"{L2_FLUSH_BYTES >> 20} MiB written between timed steps (L2 flush)"}
+            "l2": f"{L2_FLUSH_BYTES >> 20} MiB written between timed steps (L2 flush)", **extra}
 
 
-def oracle_inputs(w, jag, host_table, max_lookups):
-    """Host arrays of the bounded CPU sample.  host_table(t) returns table t as host tensors."""
+def oracle_inputs(w, jag, host_table, max_lookups, mapid=None):
+    """Host arrays of the bounded CPU sample.  host_table(t) returns table t as host tensors.
+    mapid = (raw values, mappings) makes it a sample of the fused MapId workload."""
     k, idx, off, wts, nb, n = bl.cpu_sample(w, jag, max_lookups)
     tabs, sc, bi = [], [], []
     for t in range(k):
@@ -91,26 +104,36 @@ def oracle_inputs(w, jag, host_table, max_lookups):
             bi.append(wl.raw_numpy(tab[2]))
         else:
             tabs.append(wl.raw_numpy(tab))
-    return dict(tables=tabs, scales=sc or None, biases=bi or None, indices=idx, offsets=off,
-                weights=wts, B=nb, lookups=n, n_tables=k, rows=w.rows[:k], D=w.D[:k])
+    inp = dict(tables=tabs, scales=sc or None, biases=bi or None, indices=idx, offsets=off,
+               weights=wts, B=nb, lookups=n, n_tables=k, rows=w.rows[:k], D=w.D[:k])
+    if mapid is not None:
+        inp["values"] = mapid[0][:n]
+        inp["mappings"] = mapid[1][:k]
+    return inp
 
 
 def time_oracle(w, inp):
     from oracle import ebag_oracle as orc
     t0 = time.perf_counter()
-    orc.forward(inp["tables"], w.dtype, inp["indices"], inp["offsets"], inp["B"], w.mode,
-                weights=inp["weights"], scales=inp["scales"], biases=inp["biases"], want64=True)
+    if "mappings" in inp:
+        from oracle import mapid_oracle as mo
+        mo.forward_mapid(inp["tables"], w.dtype, inp["values"], inp["offsets"], inp["B"],
+                         inp["mappings"], w.mode, weights=inp["weights"], scales=inp["scales"],
+                         biases=inp["biases"])
+    else:
+        orc.forward(inp["tables"], w.dtype, inp["indices"], inp["offsets"], inp["B"], w.mode,
+                    weights=inp["weights"], scales=inp["scales"], biases=inp["biases"], want64=True)
     return time.perf_counter() - t0
 
 
-def sized_cpu_sample(w, jag, host_table, seconds):
+def sized_cpu_sample(w, jag, host_table, seconds, mapid=None):
     """Pick the sample size from a short probe so that one oracle pass takes about `seconds`
     (the whole workload if that is less work)."""
     from oracle import ebag_oracle as orc
-    probe = oracle_inputs(w, jag, host_table, 200_000)
+    probe = oracle_inputs(w, jag, host_table, 200_000, mapid)
     t = max(time_oracle(w, probe), 1e-4)
     rate = probe["lookups"] / t
-    inp = oracle_inputs(w, jag, host_table, int(rate * seconds))
+    inp = oracle_inputs(w, jag, host_table, int(rate * seconds), mapid)
     whole = inp["lookups"] == int(jag.indices.shape[0])
     desc = (("the whole workload: " if whole else "") +
             f"the first {inp['n_tables']} of {w.T} tables, {inp['B']} bags each, "
@@ -135,7 +158,11 @@ def run_reference(args, rank):
 
     # a step must stay short enough for warmup + steps to end within a few minutes
     per_step = max(0.5, min(args.cpu_seconds, 120.0 / max(1, args.steps + args.warmup)))
-    inp, desc, cores = sized_cpu_sample(w, jag, host_table, per_step)
+    mapid = None
+    if args.workload == MAPID_WORKLOAD:
+        maps = wl.gen_mappings(w)
+        mapid = (wl.raw_values(w, jag, maps), maps)
+    inp, desc, cores = sized_cpu_sample(w, jag, host_table, per_step, mapid)
     for _ in range(args.warmup):
         time_oracle(w, inp)
     t0 = time.perf_counter()
@@ -183,6 +210,13 @@ def main():
         x = raw_tables[t]
         return tuple(y.cpu() for y in x) if isinstance(x, tuple) else x.cpu()
 
+    mapid = args.workload == MAPID_WORKLOAD
+    d_maps = None
+    if mapid:
+        maps = wl.gen_mappings(w)
+        raw = wl.raw_values(w, jag, maps)
+        d_maps = [torch.from_numpy(m).to(dev) for m in maps]
+        d_raw = torch.from_numpy(raw).to(dev)
     h_idx = torch.from_numpy(jag.indices).pin_memory()
     h_off = torch.from_numpy(jag.offsets).pin_memory()
     h_w = None if jag.weights is None else torch.from_numpy(jag.weights).pin_memory()
@@ -200,7 +234,10 @@ def main():
     stream = torch.cuda.Stream(device=dev)
 
     def step():
-        tbe.forward(tables, d_idx, d_off, w.B, w.mode, d_w, out=d_out, stream=stream)
+        if mapid:
+            tbe.forward_mapid(tables, d_raw, d_off, d_maps, w.B, w.mode, d_w, out=d_out, stream=stream)
+        else:
+            tbe.forward(tables, d_idx, d_off, w.B, w.mode, d_w, out=d_out, stream=stream)
 
     def step_host():
         tbe.forward_host(tables, h_idx, h_off, w.B, w.mode, h_w, out=h_out, stream=stream)
@@ -247,6 +284,41 @@ def main():
         torch.cuda.synchronize()
         bl.barrier()
         e2e_ms = float(sum(a.elapsed_time(b) for a, b in ev2))
+    mapid_extra = None
+    if mapid:
+        # the same work unfused: one MapId kernel per table, then the plain forward
+        ids = torch.empty_like(d_raw)
+
+        def unfused():
+            tbe.mapid(d_raw, d_off, d_maps, w.B, out=ids, stream=stream)
+            tbe.forward(tables, ids, d_off, w.B, w.mode, d_w, out=d_out, stream=stream)
+
+        def mapid_only():
+            tbe.mapid(d_raw, d_off, d_maps, w.B, out=ids, stream=stream)
+
+        def plain():
+            tbe.forward(tables, d_idx, d_off, w.B, w.mode, d_w, out=d_out, stream=stream)
+
+        def timed(fn, reps=10):
+            with torch.cuda.stream(stream):
+                fn()
+                total = 0.0
+                for _ in range(reps):
+                    flush.fill_(1)
+                    a = torch.cuda.Event(enable_timing=True)
+                    b = torch.cuda.Event(enable_timing=True)
+                    a.record(stream)
+                    fn()
+                    b.record(stream)
+                    stream.synchronize()
+                    total += a.elapsed_time(b)
+            return total / reps
+
+        fused_out = d_out.clone()
+        mapid_extra = {"mapid_then_forward_ms": timed(unfused), "mapid_alone_ms": timed(mapid_only),
+                       "plain_forward_ms": timed(plain), "fused_ms": elapsed_ms / args.steps}
+        assert torch.equal(fused_out, d_out), "fused MapId forward and plain forward disagree"
+        assert torch.equal(ids, d_idx)
     clocks = sampler.stop()
     assert tbe.last_status(stream) == (0, 0, 0)
     assert torch.equal(h_out, d_out.cpu()), "host-buffer path and device path disagree"
@@ -279,8 +351,11 @@ def main():
                      "traffic": NCU_DRAM_BYTES_PER_LAUNCH.get(w.number)},
         "bags_per_sec": w.T * w.B * world * args.steps / (max_ms * 1e-3),
     }
+    if mapid_extra:
+        line["mapid"] = mapid_extra
     if world == 1 and not args.no_cpu_baseline:
-        inp, desc, cores = sized_cpu_sample(w, jag, host_table, args.cpu_seconds)
+        inp, desc, cores = sized_cpu_sample(w, jag, host_table, args.cpu_seconds,
+                                            (raw, maps) if mapid else None)
         dt = time_oracle(w, inp)
         line["cpu_baseline"] = {"value": inp["lookups"] / dt, "unit": UNIT, "cores": cores,
                                 "kind": "oracle", "sample": desc, "seconds": dt}

@@ -150,6 +150,18 @@ ebag_status ebag_mapid(const int64_t* values, int64_t n, const int64_t* mapping,
                        int64_t* out, ebag_stream stream);
 
 /*
+ * MapId for every table of a TBE call in ONE launch: values is the jagged raw-id list of
+ * ebag_forward_mapid (device int64 [n_values]), offsets the device array [T*B + 1] that cuts it
+ * into tables, mappings / mapping_len as for ebag_forward_mapid; out (device int64 [n_values])
+ * receives the row ids, ready for ebag_forward.  The table slices are read from offsets on the
+ * device, so there is no host synchronisation.  Measured faster than the fused call when the
+ * mappings are large (the search then stalls the gather).
+ */
+ebag_status ebag_mapid_tbe(ebag_tbe* h, const int64_t* values, int64_t n_values,
+                           const int64_t* offsets, const int64_t* const* mappings,
+                           const int64_t* mapping_len, int64_t B, int64_t* out, ebag_stream stream);
+
+/*
  * The pooled forward with the MapId transform fused into the id fetch: `values` holds RAW ids
  * (same jagged layout as `indices` of ebag_forward); table t looks every one up in mappings[t]
  * (host array [T] of device pointers to sorted int64 lists, mapping_len[t] entries each, host

@@ -32,6 +32,7 @@ SIGNATURES = {
     "ebag_forward_noalloc": (_int, [_i32, _vp, _vp, _int, _vp, _vp, _i64, _vp, _vp, _i64, _int, _vp,
                                     _vp, _vp]),
     "ebag_mapid": (_int, [_vp, _i64, _vp, _i64, _vp, _vp]),
+    "ebag_mapid_tbe": (_int, [_vp, _vp, _i64, _vp, _vp, _vp, _i64, _vp, _vp]),
     "ebag_forward_mapid": (_int, [_vp, _vp, _vp, _vp, _i64, _vp, _vp, _vp, _vp, _i64, _int, _vp,
                                   _vp]),
     "ebag_last_status": (_int, [_vp, _vp, _vp, _vp]),
@@ -248,6 +249,20 @@ class TBE:
                            int(values.numel()), _ptr(offsets), _ptr(per_sample_weights),
                            [m.data_ptr() for m in mappings], [int(m.numel()) for m in mappings], B,
                            mode, _ptr(out), _stream_ptr(stream))
+        return out
+
+    def mapid(self, values, offsets, mappings: List, B: int, out=None, stream=None):
+        """MapId of all tables in one launch: raw ids -> row ids (device int64 tensors)."""
+        import torch
+        if out is None:
+            out = torch.empty_like(values)
+        T = self.T
+        mp = (ctypes.c_void_p * T)(*[int(m.data_ptr()) if m.numel() else None for m in mappings])
+        ml = (ctypes.c_int64 * T)(*[int(m.numel()) for m in mappings])
+        st = lib().ebag_mapid_tbe(self._h, _ptr(values), int(values.numel()), _ptr(offsets),
+                                  ctypes.cast(mp, _vp), ctypes.cast(ml, _vp), B, _ptr(out),
+                                  _stream_ptr(stream))
+        _check(st, "ebag_mapid_tbe")
         return out
 
     def forward_host(self, tables: List, indices, offsets, B: int, mode: int = EBAG_SUM,

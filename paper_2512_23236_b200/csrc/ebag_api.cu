@@ -257,18 +257,87 @@ __global__ void pack_int8_rowwise_kernel(const int8_t* __restrict__ q, const flo
     }
 }
 
-// MapId alone: one thread per value, coalesced in and out.
+// MapId of values[lo, hi): every thread runs four searches at a time, on values a block-width
+// apart, so that loads and stores stay coalesced and the four dependent-load chains overlap.
+__device__ __forceinline__ void mapid_range(const int64_t* __restrict__ values, int64_t lo, int64_t hi,
+                                            const int64_t* __restrict__ M, uint32_t mlen, int steps,
+                                            int64_t* __restrict__ out, int64_t first, int64_t stride) {
+    const int64_t step = stride * 4;
+    for (int64_t i = lo + first; i < hi; i += step) {
+        int64_t v[4], r[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const int64_t j = i + k * stride;
+            v[k] = j < hi ? __ldcs(reinterpret_cast<const long long*>(values + j)) : 0;
+        }
+        map_id4(M, mlen, steps, v, r);
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const int64_t j = i + k * stride;
+            if (j < hi) out[j] = r[k];
+        }
+    }
+}
+
 __global__ void mapid_kernel(const int64_t* __restrict__ values, int64_t n,
                              const int64_t* __restrict__ mapping, uint32_t mlen, int steps,
                              int64_t* __restrict__ out) {
-    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n;
-         i += (int64_t)gridDim.x * blockDim.x)
-        out[i] = map_id(mapping, mlen, steps, __ldcs(reinterpret_cast<const long long*>(values + i)));
+    mapid_range(values, 0, n, mapping, mlen, steps, out, blockIdx.x * (int64_t)blockDim.x + threadIdx.x,
+                (int64_t)gridDim.x * blockDim.x);
+}
+
+// MapId for all tables of a TBE call in one launch: blockIdx.y is the table, whose slice of the
+// jagged value list is read from the offsets array on the device (no host synchronisation).
+__global__ void mapid_tbe_kernel(const int64_t* __restrict__ values, int64_t n_values,
+                                 const int64_t* __restrict__ offsets, int64_t B,
+                                 const int64_t* const* __restrict__ mappings,
+                                 const int64_t* __restrict__ mapping_len, int64_t* __restrict__ out) {
+    const int t = blockIdx.y;
+    int64_t lo = offsets[(int64_t)t * B], hi = offsets[(int64_t)(t + 1) * B];
+    if (lo < 0) lo = 0;
+    if (hi > n_values) hi = n_values;
+    const int64_t* M = mappings[t];
+    const int64_t ml = mapping_len[t];
+    const uint32_t mlen = (uint32_t)(ml < 0 ? 0 : ml);
+    const int steps = 32 - __clz(mlen);
+    mapid_range(values, lo, hi, M, mlen, steps, out, blockIdx.x * (int64_t)blockDim.x + threadIdx.x,
+                (int64_t)gridDim.x * blockDim.x);
 }
 
 }  // namespace
 
 extern "C" {
+
+ebag_status ebag_mapid_tbe(ebag_tbe* h, const int64_t* values, int64_t n_values,
+                           const int64_t* offsets, const int64_t* const* mappings,
+                           const int64_t* mapping_len, int64_t B, int64_t* out, ebag_stream stream) {
+    if (!h || !offsets || !mappings || !mapping_len || B < 0 || n_values < 0) return EBAG_ERR_INVALID_ARG;
+    if (n_values > 0 && (!values || !out)) return EBAG_ERR_INVALID_ARG;
+    if ((int64_t)h->T * B >= (1ll << 31) || h->T > 65535) return EBAG_ERR_UNSUPPORTED;
+    for (int t = 0; t < h->T; ++t) {
+        if (mapping_len[t] < 0 || mapping_len[t] >= (1ll << 31)) return EBAG_ERR_INVALID_ARG;
+        if (mapping_len[t] > 0 && (!mappings[t] || ((uintptr_t)mappings[t] & 7u))) return EBAG_ERR_INVALID_ARG;
+    }
+    if (B == 0 || n_values == 0) return EBAG_OK;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) return EBAG_ERR_CUDA;
+    // the pointer block carries the mappings; the table slots of the block are left empty
+    std::vector<const void*> no_tables(h->T, nullptr);
+    const void* const* d_block = nullptr;
+    ebag_status st = stage_tables(h, no_tables.data(), mappings, mapping_len, (cudaStream_t)stream, &d_block);
+    if (st != EBAG_OK) return st;
+    const int64_t per_table = (n_values + h->T - 1) / h->T;
+    int64_t bx = (per_table + 255) / 256;
+    const int64_t cap = (int64_t)h->num_sms * 16 / h->T + 1;
+    if (bx > cap) bx = cap;
+    if (bx < 1) bx = 1;
+    mapid_tbe_kernel<<<dim3((unsigned)bx, (unsigned)h->T), 256, 0, (cudaStream_t)stream>>>(
+        values, n_values, offsets, B, reinterpret_cast<const int64_t* const*>(d_block + h->T),
+        reinterpret_cast<const int64_t*>(d_block + 2 * h->T), out);
+    EBAG_CUDA(h, cudaGetLastError());
+    ++h->launches;
+    return EBAG_OK;
+}
 
 ebag_status ebag_mapid(const int64_t* values, int64_t n, const int64_t* mapping, int64_t m,
                        int64_t* out, ebag_stream stream) {

@@ -196,6 +196,28 @@ def gen_tables(w: Workload, device="cpu"):
     return [gen_table(w, t, device) for t in range(w.T)]
 
 
+def gen_mappings(w: Workload) -> List[np.ndarray]:
+    """MapId inputs for workload ``w``: per table a strictly increasing int64 list of
+    rows[t] - 1 known raw ids (row 0 of the table is the "unknown" embedding), gaps of 1..3."""
+    out = []
+    for t in range(w.T):
+        rng = np.random.default_rng(np.random.SeedSequence([w.seed, w.number, 2, t]))
+        out.append(np.cumsum(rng.integers(1, 4, size=max(w.rows[t] - 1, 0), dtype=np.int64)))
+    return out
+
+
+def raw_values(w: Workload, jag: Jagged, mappings: List[np.ndarray]) -> np.ndarray:
+    """Raw ids whose MapId image is ``jag.indices``: row k >= 1 comes from the k-th known id,
+    row 0 from -1, which no mapping contains."""
+    vals = np.empty_like(jag.indices)
+    for t in range(w.T):
+        lo, hi = int(jag.offsets[t * w.B]), int(jag.offsets[(t + 1) * w.B])
+        idx = jag.indices[lo:hi]
+        m = mappings[t]
+        vals[lo:hi] = np.where(idx == 0, -1, m[np.maximum(idx, 1) - 1]) if m.size else -1
+    return vals
+
+
 def raw_numpy(x: torch.Tensor) -> np.ndarray:
     """Host numpy view of a table for the oracle: float32 / int8 as is, fp16 and bf16 as their
     uint16 bit patterns."""

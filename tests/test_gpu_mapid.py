@@ -91,6 +91,9 @@ def test_fused_mapid_forward(dtype, mode, weighted):
     out2 = tbe.forward(dev, ids, torch.from_numpy(offsets).cuda(), B, mode,
                        None if w is None else torch.from_numpy(w).cuda())
     assert torch.equal(out, out2)
+    # ... and so does MapId for all tables in one launch
+    ids3 = tbe.mapid(torch.from_numpy(values).cuda(), torch.from_numpy(offsets).cuda(), dmaps, B)
+    assert torch.equal(ids3, ids)
     tbe.close()
     ot, sc, bi = pu.oracle_tables(dtype, tabs)
     ref = mo.forward_mapid(ot, dtype, values, offsets, B, mappings, mode, weights=w, scales=sc, biases=bi)

@@ -59,3 +59,17 @@ def test_algorithmic_bytes_cfg1():
     n = int(j.lengths.sum())
     assert ab["lookups"] == n and ab["gathered"] == n * 256 and ab["indices"] == 8 * n
     assert ab["out"] == 512 * 64 * 4 and ab["offsets"] == 8 * 513 and ab["weights"] == 0
+
+
+def test_mapid_inputs_round_trip():
+    """raw_values() produces raw ids whose 1-based rank in the mapping is the row index."""
+    w = wl.make_workload(3, scale_rows=0.001, scale_B=1 / 256, max_tables=3)
+    j = wl.gen_jagged(w)
+    maps = wl.gen_mappings(w)
+    vals = wl.raw_values(w, j, maps)
+    for t in range(w.T):
+        assert maps[t].shape[0] == w.rows[t] - 1 and np.all(np.diff(maps[t]) > 0)
+        lo, hi = j.offsets[t * w.B], j.offsets[(t + 1) * w.B]
+        pos = np.searchsorted(maps[t], vals[lo:hi])
+        rank = np.where((pos < maps[t].shape[0]) & (maps[t][np.minimum(pos, maps[t].shape[0] - 1)] == vals[lo:hi]), pos + 1, 0)
+        assert np.array_equal(rank, j.indices[lo:hi])
