@@ -1,7 +1,7 @@
 #!/usr/bin/env python
 """Benchmark of the pooled embedding-bag forward on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 1..6] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 1..7] [--impl reference]
 
 One step = one pass of the whole hot path (one ebag_forward launch over all tables of the
 workload).  Default workload: 3, the batched 32-table bf16 TBE (the largest batched-table
@@ -181,9 +181,142 @@ def run_reference(args, rank):
     print(json.dumps(line), flush=True)
 
 
+MBDT_WORKLOAD = 7      # MergeBucketizedDense transform (paper Sec. 5.4.2), a NEXT row
+
+
+def run_mbdt(args, rank, local_rank, world):
+    """Workload 7: MBDT on F=64 features x B=1,048,576 values with 10 borders each (the paper
+    measures Batch x Features x Borders up to 2048 x 2 x 4, which is launch-bound here and is
+    reported beside it).  12 algorithmic bytes per value (fp32 in, int64 out)."""
+    from oracle import mbdt_oracle as mb
+    F, B, K = 64, 1 << 20, 10
+    rng = np.random.default_rng(bl.rank_seed(0, rank))
+    borders = [np.sort(rng.standard_normal(K)).astype(np.float32) for _ in range(F)]
+    values = rng.standard_normal((F, B)).astype(np.float32)
+    flat, boff = mb.flatten_borders(borders)
+    ooff = mb.bin_offsets(borders)
+    config = {"workload": "mbdt_F64_B1048576_K10", "features": F, "batch": B, "borders": K,
+              "algorithmic_bytes_per_step": 12 * F * B, "data": "N(0,1) values and borders, seed 0",
+              "l2": f"{L2_FLUSH_BYTES >> 20} MiB written between timed steps (L2 flush)"}
+    if args.impl == "reference":
+        if rank != 0:
+            return
+        sample = values[:, :B // 8]
+        for _ in range(args.warmup):
+            mb.mbdt_fast(sample, borders, ooff)
+        t0 = time.perf_counter()
+        for _ in range(args.steps):
+            mb.mbdt_fast(sample, borders, ooff)
+        dt = time.perf_counter() - t0
+        v = sample.size * args.steps / dt
+        print(json.dumps({"impl": "reference", "metric": "bucketized_values_per_sec", "value": v,
+                          "unit": "values/s", "n_gpus": args.gpus, "steps": args.steps,
+                          "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
+                          "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+                          "dtype": "f32", "data": "synthetic", "config": config,
+                          "cpu_baseline": {"value": v, "unit": "values/s", "cores": 1, "kind": "oracle",
+                                           "sample": "the first eighth of every feature's values"},
+                          "e2e": {"value": v, "unit": "values/s", "h2d_bytes_per_step": 0,
+                                  "d2h_bytes_per_step": 0}, "gpu_launches": 0}), flush=True)
+        return
+    import paper_2512_23236_b200 as eb
+    eb.lib()
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    bl.init_process_group("nccl")
+    warmup = max(3, args.warmup)
+    h_val = torch.from_numpy(values).pin_memory()
+    d_val = h_val.to(dev)
+    d_flat, d_boff, d_ooff = (torch.from_numpy(x).to(dev) for x in (flat, boff, ooff))
+    d_out = torch.empty((F, B), dtype=torch.int64, device=dev)
+    h_out = torch.empty((F, B), dtype=torch.int64).pin_memory()
+    d_stage = torch.empty_like(d_val)
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
+    stream = torch.cuda.Stream(device=dev)
+    sampler = bl.ClockSampler(f"GPU-{torch.cuda.get_device_properties(dev).uuid}").start()
+    with torch.cuda.stream(stream):
+        for _ in range(warmup):
+            flush.fill_(1)
+            eb.ebag_mbdt(d_val, d_flat, d_boff, d_ooff, out=d_out, stream=stream)
+        bl.barrier()
+        torch.cuda.synchronize()
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+              for _ in range(args.steps)]
+        for a, b in ev:
+            flush.fill_(1)
+            a.record(stream)
+            eb.ebag_mbdt(d_val, d_flat, d_boff, d_ooff, out=d_out, stream=stream)
+            b.record(stream)
+        torch.cuda.synchronize()
+        bl.barrier()
+        step_ms = [a.elapsed_time(b) for a, b in ev]
+        elapsed_ms = float(sum(step_ms))
+        e2e_steps = args.e2e_steps or min(args.steps, 10)
+        ev2 = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+               for _ in range(e2e_steps)]
+        for a, b in ev2:                      # host values in, host ids out, copies timed
+            a.record(stream)
+            d_stage.copy_(h_val, non_blocking=True)
+            eb.ebag_mbdt(d_stage, d_flat, d_boff, d_ooff, out=d_out, stream=stream)
+            h_out.copy_(d_out, non_blocking=True)
+            b.record(stream)
+        torch.cuda.synchronize()
+        bl.barrier()
+        e2e_ms = float(sum(a.elapsed_time(b) for a, b in ev2))
+        # the paper's largest measured shape, Batch x Features x Borders = 2048 x 2 x 4
+        pb = [np.sort(rng.standard_normal(4)).astype(np.float32) for _ in range(2)]
+        pflat, pboff = mb.flatten_borders(pb)
+        pv = torch.randn(2, 2048, device=dev)
+        pargs = (pv, torch.from_numpy(pflat).to(dev), torch.from_numpy(pboff).to(dev),
+                 torch.from_numpy(mb.bin_offsets(pb)).to(dev))
+        pout = torch.empty((2, 2048), dtype=torch.int64, device=dev)
+        eb.ebag_mbdt(*pargs, out=pout, stream=stream)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for _ in range(100):
+            eb.ebag_mbdt(*pargs, out=pout, stream=stream)
+        b.record(stream)
+        torch.cuda.synchronize()
+        paper_shape_us = a.elapsed_time(b) * 10.0
+    clocks = sampler.stop()
+    assert torch.equal(h_out, d_out.cpu())
+    total, max_ms = bl.reduce_job(F * B * args.steps, elapsed_ms, dev)
+    e2e_total, e2e_max = bl.reduce_job(F * B * e2e_steps, e2e_ms, dev)
+    if rank != 0:
+        return
+    peaks = bl.measured_peaks(ROOT)
+    ms = elapsed_ms / args.steps
+    achieved = 12.0 * F * B / (ms * 1e-3) / 1e9
+    t0 = time.perf_counter()
+    ref = mb.mbdt_fast(values[:, :B // 8], borders, ooff)
+    dt = time.perf_counter() - t0
+    assert np.array_equal(ref, h_out.numpy()[:, :B // 8])
+    line = {"metric": "bucketized_values_per_sec", "value": total / (max_ms * 1e-3), "unit": "values/s",
+            "n_gpus": world, "steps": args.steps, "warmup": warmup, "ms_per_step": max_ms / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+            "data": "synthetic", "config": config, "clocks": clocks, "gpu_launches": args.steps,
+            "e2e": {"value": e2e_total / (e2e_max * 1e-3), "unit": "values/s",
+                    "h2d_bytes_per_step": 4 * F * B, "d2h_bytes_per_step": 8 * F * B,
+                    "steps": e2e_steps, "ms_per_step": e2e_max / e2e_steps},
+            "roofline": {"bound": "hbm", "kernel": "mbdt_kernel", "achieved": achieved,
+                         "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
+                         "peak_source": f"{peaks['source']} HBM copy bandwidth (burst)",
+                         "algorithmic_bytes_per_launch": 12 * F * B, "ms_per_launch": ms,
+                         "ms_per_launch_min": min(step_ms), "traffic": None},
+            "cpu_baseline": {"value": ref.size / dt, "unit": "values/s", "cores": 1, "kind": "oracle",
+                             "sample": "the first eighth of every feature's values (numpy searchsorted "
+                                       "per feature, one thread)", "seconds": dt},
+            "paper_shape": {"batch_x_features_x_borders": "2048 x 2 x 4", "us_per_call": paper_shape_us,
+                            "paper_ms": "0.027-0.064 (MTIA v2i), 0.029-0.045 (MTIA v3), other hardware"}}
+    print(json.dumps(line), flush=True)
+
+
 def main():
     args = parse_args()
     rank, local_rank, world = bl.rank_info()
+    if args.workload == MBDT_WORKLOAD:
+        run_mbdt(args, rank, local_rank, world)
+        return
     if args.impl == "reference":
         run_reference(args, rank)
         return

@@ -180,6 +180,22 @@ ebag_status ebag_forward_mapid(ebag_tbe* h, const void* const* tables, const int
                                ebag_stream stream);
 
 /*
+ * MergeBucketizedDense transform (paper Sec. 5.4.2): continuous features become embedding ids.
+ *   values   device fp32 [F, B] feature-major
+ *   borders  device fp32: the sorted border lists of the F features back to back
+ *   border_offsets  device int64 [F+1]: feature f owns borders[border_offsets[f] .. [f+1])
+ *   out_offsets     device int64 [F]: added to the bins of feature f (the paper's `offsets`,
+ *                   which make the bins of different features distinct ids)
+ *   out      device int64 [F, B]:  out[f,i] = #borders of f strictly below values[f,i] + out_offsets[f]
+ * A value equal to a border falls in the bin on its left (the reading of the paper's worked
+ * example and pseudocode, i.e. torch.bucketize's default); NaN falls in the last bin.
+ * F <= 65535.  One kernel on `stream`, no allocation.  Borders must be sorted (not checked).
+ */
+ebag_status ebag_mbdt(const float* values, int32_t F, int64_t B, const float* borders,
+                      const int64_t* border_offsets, const int64_t* out_offsets, int64_t* out,
+                      ebag_stream stream);
+
+/*
  * The same forward without a handle and without any allocation (the paper has no counterpart;
  * this exists for deployment).  Some callers cannot allocate device memory when they need a
  * forward: code that runs inside a memory pool whose owner forbids side allocations, a plugin in

@@ -32,6 +32,7 @@ SIGNATURES = {
     "ebag_forward_noalloc": (_int, [_i32, _vp, _vp, _int, _vp, _vp, _i64, _vp, _vp, _i64, _int, _vp,
                                     _vp, _vp]),
     "ebag_mapid": (_int, [_vp, _i64, _vp, _i64, _vp, _vp]),
+    "ebag_mbdt": (_int, [_vp, _i32, _i64, _vp, _vp, _vp, _vp, _vp]),
     "ebag_mapid_tbe": (_int, [_vp, _vp, _i64, _vp, _vp, _vp, _i64, _vp, _vp]),
     "ebag_forward_mapid": (_int, [_vp, _vp, _vp, _vp, _i64, _vp, _vp, _vp, _vp, _i64, _int, _vp,
                                   _vp]),
@@ -142,6 +143,19 @@ def ebag_mapid(values, mapping, out=None, stream=None):
         st = lib().ebag_mapid(_ptr(values), int(values.numel()), _ptr(mapping), int(mapping.numel()),
                               _ptr(out), _stream_ptr(stream))
     _check(st, "ebag_mapid")
+    return out
+
+
+def ebag_mbdt(values, borders, border_offsets, out_offsets, out=None, stream=None):
+    """MergeBucketizedDense: device fp32 [F, B] values -> device int64 [F, B] bin ids."""
+    import torch
+    F, B = values.shape
+    if out is None:
+        out = torch.empty((F, B), dtype=torch.int64, device=values.device)
+    with torch.cuda.device(values.device):
+        st = lib().ebag_mbdt(_ptr(values), F, B, _ptr(borders), _ptr(border_offsets),
+                             _ptr(out_offsets), _ptr(out), _stream_ptr(stream))
+    _check(st, "ebag_mbdt")
     return out
 
 
