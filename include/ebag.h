@@ -196,6 +196,33 @@ ebag_status ebag_mbdt(const float* values, int32_t F, int64_t B, const float* bo
                       ebag_stream stream);
 
 /*
+ * Batch Event Truncate (paper Sec. 5.5 "Sequence Learning: Batch Event Truncate"): a nested
+ * jagged batch of event features keeps only the first N events of every user, in all F features
+ * at once, in four launches whatever F is.
+ *   outer_lengths  device int64 [U]: events per user (shared by all features)
+ *   inner_lengths  device int64 [F, E] row-major: attributes per event, E = sum(outer_lengths)
+ *   values         device int64: the attribute values of feature 0, then feature 1, ...;
+ *   value_offsets  device int64 [F+1]: feature f owns values[value_offsets[f] .. [f+1])
+ *   outer_out      device int64 [U]: min(outer_lengths[u], N)
+ *   inner_out      device int64 [F, E] (same pitch as the input): row f holds the inner lengths
+ *                  of the kept events, counts_out[0] = sum(outer_out) of them
+ *   values_out     device int64, same size and feature offsets as `values`: feature f holds the
+ *                  values of the kept events, counts_out[1 + f] of them, from value_offsets[f] on
+ *   counts_out     device int64 [1 + F]
+ *   workspace      device, ebag_bet_workspace_bytes(F, U) bytes, 8-byte aligned, caller-owned
+ * Order is preserved everywhere.  Negative lengths count as 0; ranges that would leave the
+ * caller's arrays (E or a feature's value range too small for the lengths) are cut short
+ * instead of read.  No allocation, no synchronisation; outputs must not alias inputs.
+ */
+int64_t ebag_bet_workspace_bytes(int32_t F, int64_t U);
+ebag_status ebag_batch_event_truncate(const int64_t* outer_lengths, int64_t U,
+                                      const int64_t* inner_lengths, int64_t E,
+                                      const int64_t* values, const int64_t* value_offsets,
+                                      int32_t F, int64_t N, int64_t* outer_out, int64_t* inner_out,
+                                      int64_t* values_out, int64_t* counts_out, void* workspace,
+                                      int64_t workspace_bytes, ebag_stream stream);
+
+/*
  * The same forward without a handle and without any allocation (the paper has no counterpart;
  * this exists for deployment).  Some callers cannot allocate device memory when they need a
  * forward: code that runs inside a memory pool whose owner forbids side allocations, a plugin in

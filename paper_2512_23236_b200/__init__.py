@@ -32,6 +32,9 @@ SIGNATURES = {
     "ebag_forward_noalloc": (_int, [_i32, _vp, _vp, _int, _vp, _vp, _i64, _vp, _vp, _i64, _int, _vp,
                                     _vp, _vp]),
     "ebag_mapid": (_int, [_vp, _i64, _vp, _i64, _vp, _vp]),
+    "ebag_bet_workspace_bytes": (_i64, [_i32, _i64]),
+    "ebag_batch_event_truncate": (_int, [_vp, _i64, _vp, _i64, _vp, _vp, _i32, _i64, _vp, _vp, _vp, _vp,
+                                         _vp, _i64, _vp]),
     "ebag_mbdt": (_int, [_vp, _i32, _i64, _vp, _vp, _vp, _vp, _vp]),
     "ebag_mapid_tbe": (_int, [_vp, _vp, _i64, _vp, _vp, _vp, _i64, _vp, _vp]),
     "ebag_forward_mapid": (_int, [_vp, _vp, _vp, _vp, _i64, _vp, _vp, _vp, _vp, _i64, _int, _vp,
@@ -157,6 +160,29 @@ def ebag_mbdt(values, borders, border_offsets, out_offsets, out=None, stream=Non
                              _ptr(out_offsets), _ptr(out), _stream_ptr(stream))
     _check(st, "ebag_mbdt")
     return out
+
+
+def ebag_batch_event_truncate(outer, inner, values, value_offsets, N: int, stream=None):
+    """Batch Event Truncate on device int64 tensors: outer [U], inner [F, E], values (features back
+    to back), value_offsets [F+1].  Returns (outer_out [U], inner_out [F, E], values_out, counts
+    [1+F]); only the leading counts[0] entries of every inner_out row and counts[1+f] values of
+    feature f (from value_offsets[f] on) are meaningful."""
+    import torch
+    F, E = inner.shape
+    U = int(outer.numel())
+    outer_out = torch.empty_like(outer)
+    inner_out = torch.empty_like(inner)
+    values_out = torch.empty_like(values)
+    counts = torch.empty(1 + F, dtype=torch.int64, device=outer.device)
+    nbytes = int(lib().ebag_bet_workspace_bytes(F, U))
+    ws = torch.empty(max(nbytes, 8) // 8, dtype=torch.int64, device=outer.device)
+    with torch.cuda.device(outer.device):
+        st = lib().ebag_batch_event_truncate(_ptr(outer), U, _ptr(inner), E, _ptr(values),
+                                             _ptr(value_offsets), F, int(N), _ptr(outer_out),
+                                             _ptr(inner_out), _ptr(values_out), _ptr(counts), _ptr(ws),
+                                             nbytes, _stream_ptr(stream))
+    _check(st, "ebag_batch_event_truncate")
+    return outer_out, inner_out, values_out, counts
 
 
 def ebag_forward_mapid(h: int, table_ptrs: Sequence[int], D: Sequence[int], values_ptr,
