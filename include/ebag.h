@@ -154,8 +154,8 @@ ebag_status ebag_mapid(const int64_t* values, int64_t n, const int64_t* mapping,
  * ebag_forward_mapid (device int64 [n_values]), offsets the device array [T*B + 1] that cuts it
  * into tables, mappings / mapping_len as for ebag_forward_mapid; out (device int64 [n_values])
  * receives the row ids, ready for ebag_forward.  The table slices are read from offsets on the
- * device, so there is no host synchronisation.  Measured faster than the fused call when the
- * mappings are large (the search then stalls the gather).
+ * device, so there is no host synchronisation.  Followed by ebag_forward this was measured
+ * faster than the fused call for mappings of 1 k - 100 k ids (the fused search stalls the gather).
  */
 ebag_status ebag_mapid_tbe(ebag_tbe* h, const int64_t* values, int64_t n_values,
                            const int64_t* offsets, const int64_t* const* mappings,
