@@ -268,15 +268,29 @@ class TBE:
     def last_cuda_error(self) -> str:
         return lib().ebag_last_cuda_error(self._h).decode()
 
+    def _table_array(self, tables):
+        """ctypes array of the tables' device pointers, rebuilt only when they change."""
+        ptrs = tuple(t.data_ptr() for t in tables)
+        cached = getattr(self, "_tp_cache", None)
+        if cached is None or cached[0] != ptrs:
+            arr = (ctypes.c_void_p * len(ptrs))(*[p if p else None for p in ptrs])
+            cached = (ptrs, arr, ctypes.cast(arr, _vp))
+            self._tp_cache = cached
+        return cached[2]
+
     def forward(self, tables: List, indices, offsets, B: int, mode: int = EBAG_SUM,
                 per_sample_weights=None, out=None, stream=None):
         """Device tensors in, device tensor out ([B, sum D] float32).  Enqueues only."""
         import torch
         if out is None:
             out = torch.empty((B, self.sumD), dtype=torch.float32, device=indices.device)
-        ebag_forward(self._h, [t.data_ptr() for t in tables], self.D, _ptr(indices),
-                     int(indices.numel()), _ptr(offsets), _ptr(per_sample_weights), B, mode,
-                     _ptr(out), _stream_ptr(stream))
+        if not hasattr(self, "_d_arr"):
+            self._d_arr = (ctypes.c_int32 * self.T)(*self.D)
+            self._d_ptr = ctypes.cast(self._d_arr, _vp)
+        st = lib().ebag_forward(self._h, self._table_array(tables), self._d_ptr, _ptr(indices),
+                                int(indices.numel()), _ptr(offsets), _ptr(per_sample_weights), B, mode,
+                                _ptr(out), _stream_ptr(stream))
+        _check(st, "ebag_forward")
         return out
 
     def forward_mapid(self, tables: List, values, offsets, mappings: List, B: int,
