@@ -56,6 +56,8 @@ def parse_args():
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--item-bytes", type=int, default=0)
+    ap.add_argument("--split-bytes", type=int, default=-1,
+                    help="bags gathering this many bytes or more are pooled in parts (0: never)")
     ap.add_argument("--ctas-per-sm", type=int, default=0)
     # shrunk variants of a workload, for profiler captures and quick checks (not bench lines)
     ap.add_argument("--max-tables", type=int, default=0)
@@ -511,6 +513,8 @@ def main():
     tbe = eb.TBE(w.rows, w.D, w.dtype, device=local_rank)
     if args.item_bytes:
         tbe.set_param("item_bytes", args.item_bytes)
+    if args.split_bytes >= 0:
+        tbe.set_param("split_bytes", args.split_bytes)
     if args.ctas_per_sm:
         tbe.set_param("ctas_per_sm", args.ctas_per_sm)
     stream = torch.cuda.Stream(device=dev)
@@ -612,7 +616,9 @@ def main():
         return
 
     peaks = bl.measured_peaks(ROOT)
-    ms_per_launch = elapsed_ms / max(1, launches)
+    # one forward kernel per step (the short parts kernel that may follow it is inside the same
+    # event pair and counted in gpu_launches)
+    ms_per_launch = elapsed_ms / max(1, args.steps)
     achieved = ab["total"] / (ms_per_launch * 1e-3) / 1e9
     line = {
         "metric": METRIC, "value": total_lookups / (max_ms * 1e-3), "unit": UNIT, "n_gpus": world,

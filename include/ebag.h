@@ -70,7 +70,8 @@ int64_t ebag_row_stride(ebag_dtype dtype, int32_t D);
  * Create a handle for T tables of `dtype` with rows[t] rows (0 <= rows[t] < 2^31) of D[t]
  * elements on CUDA device `device`.  rows and D are host arrays [T], copied.  1 <= T <=
  * EBAG_MAX_TABLES.  Allocates a few KB of device memory (per-table metadata, work-queue
- * counters, status words) that the handle owns until ebag_destroy.  Synchronous.
+ * counters, status words) plus up to 64 MB of scratch for the partial sums of split bags (see
+ * "split_bytes" under ebag_set_param), all owned by the handle until ebag_destroy.  Synchronous.
  * Errors: INVALID_ARG, UNSUPPORTED (T or rows too large), CUDA.
  */
 ebag_status ebag_create_tbe(int32_t T, const int64_t* rows, const int32_t* D, ebag_dtype dtype,
@@ -78,7 +79,11 @@ ebag_status ebag_create_tbe(int32_t T, const int64_t* rows, const int32_t* D, eb
 
 /*
  * Pooled forward for all T tables in ONE kernel launch on `stream` (the operator defined at
- * the top of this file).
+ * the top of this file), followed on the same stream by a second, short launch that pools the
+ * bags too long for one warp in parts (see "split_bytes" under ebag_set_param; the second launch
+ * is skipped when the call is too small to hold such a bag or splitting is off).  Both kernels
+ * are launched with programmatic stream serialization and begin by waiting for the kernel ahead
+ * of them on the stream, so stream order is what the caller sees.
  *   tables   host array [T] of DEVICE pointers; table t is row-major with row pitch
  *            ebag_row_stride(dtype, D[t]) bytes, 16-byte aligned.  The array is read before the
  *            call returns.
@@ -168,7 +173,7 @@ ebag_status ebag_mapid_tbe(ebag_tbe* h, const int64_t* values, int64_t n_values,
  * array [T]) and pools row 0 for unknown ids, row k for the k-th known id.  Table t therefore
  * has mapping_len[t] + 1 rows (create the handle with those row counts); a mapped id beyond the
  * table's rows is skipped and counted like any out-of-range id.  Everything else as
- * ebag_forward: one launch, no allocation, no synchronisation; the mapping arrays are read
+ * ebag_forward: no allocation, no synchronisation; the mapping arrays are read
  * before the call returns.  This is the producer of embedding ids the paper's preprocessing
  * section describes, placed directly in front of the gather so that the mapped ids never travel
  * through memory.
@@ -260,11 +265,20 @@ ebag_status ebag_forward_noalloc(int32_t T, const int64_t* rows, const int32_t* 
  *   "item_bytes"   target bytes of gathered rows per work item (default 32768)
  *   "ctas_per_sm"  resident CTAs per SM of the persistent grid (default: occupancy limit)
  *   "host_chunks"  bag ranges per ebag_forward_host call, 1..16 (default 0: from the size)
+ *   "split_bytes"  a bag whose rows add up to this many bytes or more (rows narrower than 256
+ *                  bytes count as 256) is pooled in parts by many warps instead of by one, the
+ *                  partial sums added in lookup order by a second, short kernel launched after
+ *                  the forward kernel on the same stream (default 65536; 0: never split, one
+ *                  launch per forward; otherwise 1024 .. 2^31-1).  The library raises the
+ *                  threshold for very large calls so that the bookkeeping always fits, which
+ *                  makes the choice of bags to split, and so the result, independent of timing.
+ *                  A call whose lookups could not add up to one such bag skips the second launch.
  * Returns INVALID_ARG for an unknown name or a value out of range.
  */
 ebag_status ebag_set_param(ebag_tbe* h, const char* name, int64_t value);
 
-/* Number of kernels this handle has launched so far (forward and host-forward). */
+/* Number of kernels this handle has launched so far (forward and host-forward; a forward whose
+ * call is large enough to hold a bag that would be split counts two, see "split_bytes"). */
 int64_t ebag_launch_count(const ebag_tbe* h);
 
 /* Text of the last CUDA error seen by this handle ("" if none). */

@@ -2,6 +2,7 @@
 // kernel launches.  Declarations and the contract of every entry point are in include/ebag.h.
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <cstring>
 #include <new>
 #include <string>
@@ -17,6 +18,8 @@ namespace {
 constexpr int kTableSlots = 4;   // device copies of the table-pointer array that may be in flight
 constexpr int kMaxHostChunks = 16;                 // bag ranges per ebag_forward_host call
 constexpr int64_t kHostChunkBytes = 64ll << 20;    // transfer size one range aims for
+constexpr uint64_t kLongScratchBytes = 64ull << 20;  // partial sums of split bags, per handle
+constexpr uint64_t kLongMaxParts = 8 * kMaxLongBags; // parts of split bags per launch (see forward_device)
 constexpr int kAutoHostChunks = 6;                 // more ranges cost more in small copies than they hide
 
 struct DeviceGuard {             // make the handle's device current for the duration of a call
@@ -53,6 +56,12 @@ struct ebag_tbe {
     int occupancy[2][2] = {};                      // CTAs per SM, [plain, MapId][unweighted, weighted]
     uint32_t item_bytes = 32768;
     int ctas_per_sm = 0;                           // 0: occupancy limit
+    // long bags (pooled in parts by a second kernel): one device block carved into the control
+    // words, the recorded bags, their arrival counters and the partial sums
+    void* d_long = nullptr;
+    LongParams lg = {};
+    uint32_t max_stride = 0;
+    uint32_t split_bytes = 65536;                  // a bag gathering this much or more is split; 0: never
     int64_t launches = 0;
     std::string cuda_error;
     // staging for ebag_forward_host
@@ -87,6 +96,7 @@ void free_handle(ebag_tbe* h) {
     cudaFree(h->d_meta);
     cudaFree(h->d_queue);
     cudaFree(h->d_status);
+    cudaFree(h->d_long);
     for (int i = 0; i < kTableSlots; ++i) {
         cudaFree(h->d_tables[i]);
         if (h->h_tables[i]) cudaFreeHost(h->h_tables[i]);
@@ -116,6 +126,15 @@ cudaError_t launch_fwd(int dtype, const FwdParams& p, bool w, bool mapid, int gr
         case EBAG_F16: return launch_fwd_f16(p, w, mapid, grid, smem, s);
         case EBAG_BF16: return launch_fwd_bf16(p, w, mapid, grid, smem, s);
         default: return launch_fwd_int8(p, w, mapid, grid, smem, s);
+    }
+}
+
+cudaError_t launch_parts(int dtype, const FwdParams& p, bool w, bool mapid, int grid, cudaStream_t s) {
+    switch (dtype) {
+        case EBAG_F32: return launch_parts_f32(p, w, mapid, grid, s);
+        case EBAG_F16: return launch_parts_f16(p, w, mapid, grid, s);
+        case EBAG_BF16: return launch_parts_bf16(p, w, mapid, grid, s);
+        default: return launch_parts_int8(p, w, mapid, grid, s);
     }
 }
 
@@ -209,6 +228,23 @@ ebag_status forward_device(ebag_tbe* h, const void* const* tables, const int64_t
     p.sumD = h->sumD;
     p.mean = mode == EBAG_MEAN ? 1 : 0;
     p.item_bytes = h->item_bytes;
+    // Long bags.  The bytes this call can gather are at most n_indices * (widest row), so at most
+    // that / long_bytes bags can reach long_bytes; with long_bytes = 4 * part_bytes (a power of two) and
+    // part_bytes >= 2 * bound / max_parts, at most max_parts / 8 bags are recorded and they ask
+    // for at most bound / part_bytes + (bags) <= 5/8 max_parts parts: both always fit, so which
+    // bags are split never depends on timing.  A call too small to hold a long bag skips the
+    // second launch altogether.
+    p.lg = h->lg;
+    const uint64_t bound = (uint64_t)n_indices * std::max<uint32_t>(h->max_stride, kLongMinRowBytes);
+    if (h->split_bytes == 0 || bound < h->split_bytes) {
+        p.lg.ctl = nullptr;
+    } else {
+        const uint64_t fit = (2 * bound + p.lg.max_parts - 1) / p.lg.max_parts;
+        const uint64_t part_bytes = std::max<uint64_t>(h->split_bytes / 4, fit);
+        p.lg.part_shift = 8;
+        while ((1ull << p.lg.part_shift) < part_bytes) ++p.lg.part_shift;   // a power of two: no division on the device
+        p.lg.long_bytes = 4ull << p.lg.part_shift;
+    }
     const bool w = weights != nullptr;
     const bool mapid = mappings != nullptr;
     int per_sm = h->occupancy[mapid ? 1 : 0][w ? 1 : 0];
@@ -216,6 +252,10 @@ ebag_status forward_device(ebag_tbe* h, const void* const* tables, const int64_t
     const int grid = h->num_sms * per_sm;
     EBAG_CUDA(h, launch_fwd(h->dtype, p, w, mapid, grid, fwd_smem_bytes(h->T), stream));
     ++h->launches;
+    if (p.lg.ctl) {
+        EBAG_CUDA(h, launch_parts(h->dtype, p, w, mapid, grid, stream));
+        ++h->launches;
+    }
     return EBAG_OK;
 }
 
@@ -432,6 +472,30 @@ ebag_status ebag_create_tbe(int32_t T, const int64_t* rows, const int32_t* D, eb
         EBAG_CUDA(h, cudaMemset(h->d_queue, 0, sizeof(Queue)));
         EBAG_CUDA(h, cudaMalloc((void**)&h->d_status, sizeof(Status)));
         EBAG_CUDA(h, cudaMemset(h->d_status, 0, sizeof(Status)));
+        {
+            // one slot of partial sums holds a row per bag that a warp pools side by side
+            uint32_t slot = 4;
+            for (int t = 0; t < T; ++t) {
+                slot = std::max<uint32_t>(slot, (uint32_t)(32 >> meta[t].g_log2) * (uint32_t)meta[t].D);
+                h->max_stride = std::max<uint32_t>(h->max_stride, (uint32_t)meta[t].stride);
+            }
+            uint64_t parts = kLongScratchBytes / ((uint64_t)slot * sizeof(float));
+            parts = std::min<uint64_t>(std::max<uint64_t>(parts, kMaxLongBags), kLongMaxParts);
+            auto up = [](size_t x) { return (x + 255) & ~(size_t)255; };
+            const size_t o_bags = up(sizeof(LongCtl));
+            const size_t o_arr = o_bags + up(sizeof(LongBag) * kMaxLongBags);
+            const size_t o_part = o_arr + up(sizeof(unsigned) * kMaxLongBags);
+            const size_t total = o_part + (size_t)parts * slot * sizeof(float);
+            EBAG_CUDA(h, cudaMalloc(&h->d_long, total));
+            EBAG_CUDA(h, cudaMemset(h->d_long, 0, o_part));
+            char* base = static_cast<char*>(h->d_long);
+            h->lg.ctl = reinterpret_cast<LongCtl*>(base);
+            h->lg.bags = reinterpret_cast<LongBag*>(base + o_bags);
+            h->lg.arrivals = reinterpret_cast<unsigned*>(base + o_arr);
+            h->lg.partial = reinterpret_cast<float*>(base + o_part);
+            h->lg.slot_floats = slot;
+            h->lg.max_parts = (uint32_t)parts;
+        }
         for (int i = 0; i < kTableSlots; ++i) {
             EBAG_CUDA(h, cudaMalloc((void**)&h->d_tables[i], sizeof(void*) * 3 * T));
             EBAG_CUDA(h, cudaMallocHost((void**)&h->h_tables[i], sizeof(void*) * 3 * T));
@@ -600,6 +664,11 @@ ebag_status ebag_set_param(ebag_tbe* h, const char* name, int64_t value) {
     if (std::strcmp(name, "item_bytes") == 0) {
         if (value < 256 || value > (1ll << 30)) return EBAG_ERR_INVALID_ARG;
         h->item_bytes = (uint32_t)value;
+        return EBAG_OK;
+    }
+    if (std::strcmp(name, "split_bytes") == 0) {
+        if (value != 0 && (value < 1024 || value > (1ll << 31) - 1)) return EBAG_ERR_INVALID_ARG;
+        h->split_bytes = (uint32_t)value;
         return EBAG_OK;
     }
     if (std::strcmp(name, "host_chunks") == 0) {

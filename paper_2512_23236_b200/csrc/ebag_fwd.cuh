@@ -63,6 +63,48 @@ struct Status {
     unsigned long long n_bad_offsets;
 };
 
+// ---- long bags.  A bag whose rows add up to `long_bytes` or more is not pooled by the warp that
+// meets it in the forward kernel: that warp records it, and a second kernel pools the recorded
+// bags in PARTS (equal runs of lookups), one part per warp, each row group of the warp leaving a
+// row of partial sums in the part's slot; the warp that delivers a bag's last part adds the
+// partial sums in lookup order (so the result does not depend on which warp ran what, or when)
+// and writes the output row.  The host picks `long_bytes` so that the recorded bags and their
+// parts always fit (at most total bytes / long_bytes bags can be that long); should malformed
+// offsets make bags overlap and the room run out all the same, the bags that do not fit are
+// pooled whole by the warp that met them.
+constexpr int kMaxLongBags = 2048;
+constexpr uint32_t kLongMinRowBytes = 256;   // narrow rows count as this much: a lone warp is latency bound
+constexpr int kMaxPartsPerBag = 2048;
+
+struct LongCtl {                         // all zero between launches
+    unsigned int count;                  // bags the forward kernel recorded
+    unsigned int part_next;              // next part to pool
+    unsigned int exited;                 // CTAs of the parts kernel that have finished
+    unsigned int pad;
+};
+
+struct LongBag {                         // what the forward kernel leaves about a bag it did not pool
+    int32_t t;
+    int32_t bag;                         // bag number within the launch (of its table)
+};
+
+struct LongParams {                      // ctl == nullptr: bags are never split
+    LongCtl* ctl;
+    LongBag* bags;                       // [kMaxLongBags]
+    unsigned int* arrivals;              // [kMaxLongBags] parts delivered per bag; zero between launches
+    float* partial;                      // [max_parts * slot_floats]
+    uint64_t long_bytes;                 // 4 parts' worth
+    uint32_t part_shift;                 // a part aims at 2^part_shift bytes of rows
+    uint32_t slot_floats;                // floats per part: (bags side by side) * D, the widest of the call
+    uint32_t max_parts;                  // >= kMaxLongBags
+};
+
+struct PartArgs {                        // one part of a long bag (parts kernel only)
+    int64_t base;                        // first lookup of the part
+    uint32_t len;                        // lookups in the part
+    float* slot;                         // where its rows of partial sums go
+};
+
 struct FwdParams {
     const void* const* tables;   // device [T]
     const TableMeta* meta;       // device [T]
@@ -82,6 +124,7 @@ struct FwdParams {
     int32_t sumD;
     int32_t mean;                // 1: divide by the bag length
     uint32_t item_bytes;
+    LongParams lg;
 };
 
 // ------------------------------------------------------------------ memory access helpers
@@ -260,6 +303,7 @@ __device__ __forceinline__ void map_id4(const int64_t* __restrict__ M, uint32_t 
 #endif
 constexpr int kStageVecs = EBAG_STAGE_VECS;      // 16-byte vectors per lane per stage
 constexpr int kStages = 2;
+constexpr int kWarpSmemVecs = kStages * kStageVecs * 32 + 24;   // a warp's ring, then 96 words about its item's bags
 
 struct IdChunk {          // ids of up to G consecutive entries of the bags one slot works on
     uint32_t r;           // per lane: validated row id of entry `lig`, or kInvalidRow
@@ -272,39 +316,95 @@ struct IdChunk {          // ids of up to G consecutive entries of the bags one 
     bool valid;
 };
 
-template <int DT, bool WEIGHTED, bool MAPID, int V>
+// Offsets of bag `lane` of an item relative to the item's first lookup (both 0 for a malformed
+// bag, which is reported through `bad`).
+__device__ __forceinline__ void load_bag_range(const FwdParams& p, int64_t g0, int lane,
+                                               int64_t base_raw, int64_t base, uint32_t& off_lo,
+                                               uint32_t& off_hi, bool& bad) {
+    const int64_t room = p.n_indices - base;
+    const int64_t lo = ld_stream_i64(p.offsets + g0 + lane) - base;
+    const int64_t hi = ld_stream_i64(p.offsets + g0 + lane + 1) - base;
+    off_lo = off_hi = 0;
+    bad = base_raw != base || lo < 0 || hi < lo || hi > room || hi > 0x7fffffffll;
+    if (!bad) {
+        off_lo = (uint32_t)lo;
+        off_hi = (uint32_t)hi;
+    }
+}
+
+// PART: the "item" is one part of a long bag (`pa`): its lookups are shared out among the row
+// groups as if they were NG bags, and the rows of sums go to the part's slot, never divided.
+// `skip` (forward kernel, splitting on): bit i set = bag i of the item is pooled elsewhere; the
+// call for the first column tile of an item works it out, the calls for the other tiles reuse it.
+template <int DT, bool WEIGHTED, bool MAPID, int V, bool PART = false>
 __device__ __forceinline__ void process_item(const FwdParams& p, const TableMeta& m,
                                                    const char* __restrict__ tbase, int t,
                                                    int64_t bag0, int cnt, int vec0, int lane,
                                                    unsigned& n_oob, unsigned& n_bad,
                                                    uint4* __restrict__ wbuf,
-                                                   float2* __restrict__ sbbuf) {
+                                                   float2* __restrict__ sbbuf,
+                                                   unsigned& skip, const PartArgs& pa) {
     constexpr int NACC = Elem<DT>::kAcc;
     constexpr int CR = kStageVecs / V;               // rows per stage
     const int G = 1 << m.g_log2;
     const int NG = 32 >> m.g_log2;
     const int lig = lane & (G - 1);
     const int grp = lane >> m.g_log2;
-    const int64_t g0 = (int64_t)t * p.off_stride + bag0;
 
-    const int64_t base_raw = ld_stream_i64(p.offsets + g0);
-    const int64_t base = base_raw < 0 ? 0 : (base_raw > p.n_indices ? p.n_indices : base_raw);
-    const int64_t room = p.n_indices - base;
+    int64_t base;
     uint32_t off_lo = 0, off_hi = 0;
     uint32_t key = (uint32_t)lane;
-    if (lane < cnt) {
-        const int64_t lo = ld_stream_i64(p.offsets + g0 + lane) - base;
-        const int64_t hi = ld_stream_i64(p.offsets + g0 + lane + 1) - base;
-        if (base_raw != base || lo < 0 || hi < lo || hi > room || hi > 0x7fffffffll) {
-            if (vec0 == 0) ++n_bad;
-        } else {
-            off_lo = (uint32_t)lo;
-            off_hi = (uint32_t)hi;
+    if constexpr (PART) {
+        base = pa.base;
+        if (lane < cnt) {
+            off_lo = (uint32_t)((uint64_t)pa.len * (uint32_t)lane / (uint32_t)cnt);
+            off_hi = (uint32_t)((uint64_t)pa.len * (uint32_t)(lane + 1) / (uint32_t)cnt);
+            key = ((off_hi - off_lo + 1u) << 6) | (uint32_t)lane;
         }
-        const uint32_t len = off_hi - off_lo;
-        key = (((len > 0x3FFFFFEu ? 0x3FFFFFEu : len) + 1u) << 5) | (uint32_t)lane;
+    } else {
+        const int64_t g0 = (int64_t)t * p.off_stride + bag0;
+        const int64_t base_raw = ld_stream_i64(p.offsets + g0);
+        base = base_raw < 0 ? 0 : (base_raw > p.n_indices ? p.n_indices : base_raw);
+        if (lane < cnt) {
+            bool bad;
+            load_bag_range(p, g0, lane, base_raw, base, off_lo, off_hi, bad);
+            if (bad && vec0 == 0) ++n_bad;
+        }
+        if (p.lg.ctl) {
+            // ---- bags long enough to be split are recorded for the parts kernel (by the call
+            // for the first column tile) and count as empty here
+            if (vec0 == 0) {
+                bool is_long = false;
+                const uint32_t len = off_hi - off_lo;
+                const uint64_t bytes = (uint64_t)len * max((uint32_t)m.stride, kLongMinRowBytes);
+                if (len > 0 && bytes >= p.lg.long_bytes) {
+                    const unsigned idx = atomicAdd(&p.lg.ctl->count, 1u);
+                    if (idx < (unsigned)kMaxLongBags) {          // else: no room, pooled whole here
+                        is_long = true;
+                        p.lg.bags[idx].t = t;
+                        p.lg.bags[idx].bag = (int32_t)(bag0 + lane);
+                    }
+                }
+                skip = __ballot_sync(0xffffffffu, is_long);
+            }
+            if ((skip >> lane) & 1u) {
+                off_hi = off_lo;
+                key |= 32u;                  // carried through the sort in the key
+            }
+        }
+        if (lane < cnt) {
+            const uint32_t len = off_hi - off_lo;
+            key |= ((len > 0x1FFFFFEu ? 0x1FFFFFEu : len) + 1u) << 6;
+        }
     }
     if (NG > 1 && cnt > NG) key = warp_sort_desc(key, lane);
+    // the item's bags, readable by every lane: [0,32) first lookup, [32,64) end, [64,96) sorted keys
+    uint32_t* bagw = reinterpret_cast<uint32_t*>(wbuf + kStages * kStageVecs * 32);
+    __syncwarp();                                    // the previous item's readers are done
+    bagw[lane] = off_lo;
+    bagw[32 + lane] = off_hi;
+    bagw[64 + lane] = key;
+    __syncwarp();
     const int64_t* __restrict__ idx_base = p.indices + base;
     const float* __restrict__ w_base = WEIGHTED ? p.weights + base : nullptr;
 
@@ -317,7 +417,7 @@ __device__ __forceinline__ void process_item(const FwdParams& p, const TableMeta
         lane_base[v] = tbase + vec * 16;
     }
     const uint32_t stride = (uint32_t)m.stride;
-    const uint64_t rows = (uint64_t)m.rows;
+    const uint32_t rows = (uint32_t)m.rows;          // tables have fewer than 2^31 rows
     const char* sb_base = tbase + m.D;
     const int nslots = (cnt + NG - 1) >> (5 - m.g_log2);
 
@@ -334,7 +434,7 @@ __device__ __forceinline__ void process_item(const FwdParams& p, const TableMeta
             float wl = 1.0f;
             if (WEIGHTED) wl = ld_stream_f32(w_base + i);
             if (MAPID) r = map_id(map_ptr, map_len, map_steps, r);     // raw id -> row
-            if ((uint64_t)r < rows) {
+            if ((uint64_t)r < (uint64_t)rows) {
                 ridx = (uint32_t)r;
                 w = wl;
             } else if (vec0 == 0) {
@@ -342,11 +442,12 @@ __device__ __forceinline__ void process_item(const FwdParams& p, const TableMeta
             }
         }
     };
-    auto slot_bag = [&](int pos_in_item, uint32_t& s, uint32_t& e, int& orig) {
-        const uint32_t k = __shfl_sync(0xffffffffu, key, pos_in_item & 31);
+    auto slot_bag = [&](int pos_in_item, uint32_t& s, uint32_t& e, int& orig, bool& elsewhere) {
+        const uint32_t k = bagw[64 + (pos_in_item & 31)];
         orig = (int)(k & 31u);
-        s = __shfl_sync(0xffffffffu, off_lo, orig);
-        e = __shfl_sync(0xffffffffu, off_hi, orig);
+        elsewhere = (k & 32u) != 0;
+        s = bagw[orig];
+        e = bagw[32 + orig];
         if (pos_in_item >= cnt) s = e = 0;
     };
 
@@ -365,7 +466,8 @@ __device__ __forceinline__ void process_item(const FwdParams& p, const TableMeta
             }
             uint32_t gs;
             int o;
-            slot_bag(gslot * NG + grp, gs, ge, o);
+            bool unused;
+            slot_bag(gslot * NG + grp, gs, ge, o, unused);
             gpos = gs;
         }
         load_chunk(gpos, ge, c.r, c.w);
@@ -464,10 +566,14 @@ __device__ __forceinline__ void process_item(const FwdParams& p, const TableMeta
     auto finalize = [&](int slot) {
         uint32_t s, e;
         int orig;
-        slot_bag(slot * NG + grp, s, e, orig);
-        if (slot * NG + grp < cnt) {
+        bool elsewhere;
+        slot_bag(slot * NG + grp, s, e, orig, elsewhere);
+        bool write = slot * NG + grp < cnt;
+        if (!PART) write = write && !elsewhere;
+        if (write) {
             const uint32_t L = e - s;
-            float* orow = p.out + (bag0 + orig) * (int64_t)p.sumD + m.D_off;
+            float* orow = PART ? pa.slot + (size_t)orig * m.D
+                               : p.out + (bag0 + orig) * (int64_t)p.sumD + m.D_off;
 #pragma unroll
             for (int v = 0; v < V; ++v) {
                 if (!col_on[v]) continue;
@@ -476,7 +582,7 @@ __device__ __forceinline__ void process_item(const FwdParams& p, const TableMeta
                 for (int a = 0; a < NACC; ++a) {
                     float x = acc[v][a];
                     if (DT == DT_INT8) x += acc_bias;
-                    if (p.mean && L > 0) x = __fdiv_rn(x, (float)L);
+                    if (!PART && p.mean && L > 0) x = __fdiv_rn(x, (float)L);
                     acc[v][a] = x;
                 }
 #pragma unroll
@@ -553,12 +659,18 @@ ebag_fwd_kernel(const FwdParams p) {
     int* item_bags = smem_i + p.T + 1;                         // [T]   bags per item of each table
     float* bag_bytes = reinterpret_cast<float*>(item_bags);    // [T]   (first pass) bytes per bag
     __shared__ float total_bytes;
-    __shared__ uint4 stage_buf[kWarps * kStages * kStageVecs * 32];          // 4 KB per warp
+    __shared__ uint4 stage_buf[kWarps * kWarpSmemVecs];      // per warp: 4 KB ring + the item's bags
     __shared__ float2 sb_buf[DT == DT_INT8 ? kWarps * kStages * kStageVecs * 8 : 1];
-    uint4* wbuf = stage_buf + (threadIdx.x >> 5) * (kStages * kStageVecs * 32);
+    uint4* wbuf = stage_buf + (threadIdx.x >> 5) * kWarpSmemVecs;
     float2* sbbuf = sb_buf + (DT == DT_INT8 ? (threadIdx.x >> 5) * (kStages * kStageVecs * 8) : 0);
     const int tid = threadIdx.x;
     const int lane = tid & 31;
+
+    // This launch may have been made resident before the kernel ahead of it on the stream
+    // finished: wait for it (and its writes).  In turn the kernel that follows (the parts kernel,
+    // or the next forward) may take the place of CTAs that finish here; it waits the same way.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;");
 
     // ---- size the items of every table from its share of the offsets prefix sum
     if (tid == 0) total_bytes = 0.0f;
@@ -631,12 +743,16 @@ ebag_fwd_kernel(const FwdParams p) {
         const int cnt = rest < ib ? (int)rest : ib;
         const char* tbase = static_cast<const char*>(p.tables[t]);
 
+        const PartArgs no_part{};
+        unsigned skip = 0;
         if (m.V == 1) {
-            process_item<DT, WEIGHTED, MAPID, 1>(p, m, tbase, t, bag0, cnt, 0, lane, n_oob, n_bad, wbuf, sbbuf);
+            process_item<DT, WEIGHTED, MAPID, 1>(p, m, tbase, t, bag0, cnt, 0, lane, n_oob, n_bad, wbuf,
+                                                 sbbuf, skip, no_part);
         } else {
             // rows above 512 bytes: two vectors per lane, 1 KB column tiles
             for (int vec0 = 0; vec0 < m.nvec; vec0 += 64)
-                process_item<DT, WEIGHTED, MAPID, 2>(p, m, tbase, t, bag0, cnt, vec0, lane, n_oob, n_bad, wbuf, sbbuf);
+                process_item<DT, WEIGHTED, MAPID, 2>(p, m, tbase, t, bag0, cnt, vec0, lane, n_oob, n_bad,
+                                                     wbuf, sbbuf, skip, no_part);
         }
         q = __shfl_sync(0xffffffffu, q_next, 0);
     }
@@ -660,11 +776,174 @@ ebag_fwd_kernel(const FwdParams p) {
     }
 }
 
+// ------------------------------------------------------------------ the parts kernel
+// Pools the long bags the forward kernel recorded (it runs after it on the same stream).  A launch
+// that finds nothing recorded ends at once.
+template <int DT, bool WEIGHTED, bool MAPID>
+__global__ void __launch_bounds__(kThreads, EBAG_MIN_BLOCKS)
+ebag_parts_kernel(const FwdParams p) {
+    __shared__ uint4 stage_buf[kWarps * kWarpSmemVecs];
+    __shared__ float2 sb_buf[DT == DT_INT8 ? kWarps * kStages * kStageVecs * 8 : 1];
+    __shared__ unsigned part0_s[kMaxLongBags + 1];     // first part of every recorded bag
+    __shared__ unsigned scan_warp_s[kWarps], scan_carry_s;
+    uint4* wbuf = stage_buf + (threadIdx.x >> 5) * kWarpSmemVecs;
+    float2* sbbuf = sb_buf + (DT == DT_INT8 ? (threadIdx.x >> 5) * (kStages * kStageVecs * 8) : 0);
+    const int tid = threadIdx.x;
+    const int lane = tid & 31;
+
+    // this launch may have been made resident before the forward kernel finished: wait for it
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    unsigned nb = p.lg.ctl->count;
+    if (nb == 0) return;                               // nothing was recorded (and nothing to re-arm)
+    if (nb > (unsigned)kMaxLongBags) nb = kMaxLongBags;
+
+    // ---- plan: parts per bag from its length, first part of every bag by a prefix sum.  Every
+    // CTA works out the same plan from the same records.
+    auto want_of = [&](unsigned i) -> unsigned {
+        const LongBag r = p.lg.bags[i];
+        const int64_t g = (int64_t)r.t * p.off_stride + r.bag;
+        const uint64_t len = (uint64_t)(p.offsets[g + 1] - p.offsets[g]);   // checked by the forward kernel
+        const uint64_t bytes = len * max((uint32_t)p.meta[r.t].stride, kLongMinRowBytes);
+        uint64_t want = (bytes + ((1ull << p.lg.part_shift) - 1)) >> p.lg.part_shift;
+        if (want > (uint64_t)kMaxPartsPerBag) want = kMaxPartsPerBag;
+        if (want > len) want = len;
+        return (unsigned)want;
+    };
+    for (int pass = 0; pass < 2; ++pass) {
+        // pass 0 with the parts each bag wants; should they not fit (only overlapping bags can
+        // ask for that much), pass 1 with one part per bag, which always fits
+        if (tid == 0) scan_carry_s = 0;
+        __syncthreads();
+        for (unsigned i0 = 0; i0 < nb; i0 += kThreads) {
+            const unsigned i = i0 + tid;
+            unsigned x = i < nb ? (pass == 0 ? want_of(i) : 1u) : 0u;
+            const unsigned mine = x;
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                const unsigned y = __shfl_up_sync(0xffffffffu, x, d);
+                if (lane >= d) x += y;
+            }
+            if (lane == 31) scan_warp_s[tid >> 5] = x;
+            __syncthreads();
+            unsigned before = scan_carry_s;
+            for (int w = 0; w < (tid >> 5); ++w) before += scan_warp_s[w];
+            if (i < nb) part0_s[i] = before + x - mine;
+            __syncthreads();
+            if (tid == kThreads - 1) scan_carry_s = before + x;
+            __syncthreads();
+        }
+        if (scan_carry_s <= p.lg.max_parts) break;
+        __syncthreads();
+    }
+    const unsigned part_total = scan_carry_s;
+    if (tid == 0) part0_s[nb] = part_total;
+    __syncthreads();
+
+    unsigned n_oob = 0, n_bad = 0;
+    while (true) {
+        unsigned pq = 0;
+        if (lane == 0) pq = atomicAdd(&p.lg.ctl->part_next, 1u);
+        pq = __shfl_sync(0xffffffffu, pq, 0);
+        if (pq >= part_total) break;
+        // the bag of part pq: last record with part0 <= pq
+        unsigned blo = 0, bhi = nb;
+        while (bhi - blo > 1) {
+            const unsigned mid = (blo + bhi) >> 1;
+            if (part0_s[mid] <= pq) blo = mid; else bhi = mid;
+        }
+        const unsigned bi = blo;
+        const unsigned bag_part0 = part0_s[bi];
+        const unsigned bag_parts = part0_s[bi + 1] - bag_part0;
+        const LongBag rec = p.lg.bags[bi];
+        const int t = rec.t;
+        const TableMeta m = p.meta[t];
+        const int ng = 32 >> m.g_log2;
+        const int64_t g = (int64_t)t * p.off_stride + rec.bag;
+        const int64_t lo = p.offsets[g];
+        const uint64_t len = (uint64_t)(p.offsets[g + 1] - lo);
+        {
+            const char* tbase = static_cast<const char*>(p.tables[t]);
+            const uint64_t k = pq - bag_part0;
+            const uint64_t s0 = len * k / bag_parts, s1 = len * (k + 1) / bag_parts;
+            unsigned no_skip = 0;
+            PartArgs pa;
+            pa.base = lo + (int64_t)s0;
+            pa.len = (uint32_t)(s1 - s0);
+            pa.slot = p.lg.partial + (size_t)pq * p.lg.slot_floats;
+            if (m.V == 1) {
+                process_item<DT, WEIGHTED, MAPID, 1, true>(p, m, tbase, t, 0, ng, 0, lane, n_oob, n_bad,
+                                                           wbuf, sbbuf, no_skip, pa);
+            } else {
+                for (int vec0 = 0; vec0 < m.nvec; vec0 += 64)
+                    process_item<DT, WEIGHTED, MAPID, 2, true>(p, m, tbase, t, 0, ng, vec0, lane, n_oob,
+                                                               n_bad, wbuf, sbbuf, no_skip, pa);
+            }
+        }
+        // ---- deliver the part; whoever delivers a bag's last part adds them up, in lookup order
+        __threadfence();
+        __syncwarp();
+        unsigned prev = 0;
+        if (lane == 0) prev = atomicAdd(&p.lg.arrivals[bi], 1u);
+        prev = __shfl_sync(0xffffffffu, prev, 0);
+        if (prev == bag_parts - 1) {
+            __threadfence();
+            const float* src = p.lg.partial + (size_t)bag_part0 * p.lg.slot_floats;
+            float* orow = p.out + rec.bag * (int64_t)p.sumD + m.D_off;
+            // rows of partial sums, in lookup order: row r is at src + (r / ng) * slot + (r % ng) * D
+            const unsigned nrows = bag_parts * (unsigned)ng;
+            for (int c = lane * 4; c < m.D; c += 128) {
+                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                constexpr int kBatch = 8;                // loads in flight; the adds stay in order
+                for (unsigned r0 = 0; r0 < nrows; r0 += kBatch) {
+                    float4 x[kBatch];
+#pragma unroll
+                    for (int i = 0; i < kBatch; ++i) {
+                        const unsigned r = r0 + i;
+                        x[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+                        if (r < nrows)
+                            x[i] = __ldcg(reinterpret_cast<const float4*>(
+                                src + (size_t)(r >> (5 - m.g_log2)) * p.lg.slot_floats +
+                                (size_t)(r & (ng - 1)) * m.D + c));
+                    }
+#pragma unroll
+                    for (int i = 0; i < kBatch; ++i)
+                        if (r0 + i < nrows) {
+                            acc.x += x[i].x; acc.y += x[i].y; acc.z += x[i].z; acc.w += x[i].w;
+                        }
+                }
+                if (p.mean && len > 0) {
+                    const float fl = (float)len;
+                    acc.x = __fdiv_rn(acc.x, fl); acc.y = __fdiv_rn(acc.y, fl);
+                    acc.z = __fdiv_rn(acc.z, fl); acc.w = __fdiv_rn(acc.w, fl);
+                }
+                st_stream16(orow + c, acc.x, acc.y, acc.z, acc.w);
+            }
+            if (lane == 0) p.lg.arrivals[bi] = 0;       // ready for the next launch
+        }
+    }
+
+    n_oob = __reduce_add_sync(0xffffffffu, n_oob);
+    if (lane == 0 && n_oob) atomicAdd(&p.status->n_oob, (unsigned long long)n_oob);
+    __syncthreads();
+    if (tid == 0) {                                    // the last CTA out re-arms the bookkeeping
+        __threadfence();
+        const unsigned prev = atomicAdd(&p.lg.ctl->exited, 1u);
+        if (prev == gridDim.x - 1) {
+            p.lg.ctl->count = 0;
+            p.lg.ctl->part_next = 0;
+            p.lg.ctl->exited = 0;
+            __threadfence();
+        }
+    }
+}
+
 // one launcher per dtype, each compiled in its own translation unit
 #define EBAG_DECLARE_LAUNCHERS(NAME)                                                             \
     cudaError_t launch_fwd_##NAME(const FwdParams& p, bool weighted, bool mapid, int grid,        \
                                   size_t smem, cudaStream_t s);                                  \
-    cudaError_t occupancy_fwd_##NAME(bool weighted, bool mapid, size_t smem, int* ctas_per_sm);
+    cudaError_t occupancy_fwd_##NAME(bool weighted, bool mapid, size_t smem, int* ctas_per_sm);  \
+    cudaError_t launch_parts_##NAME(const FwdParams& p, bool weighted, bool mapid, int grid,      \
+                                    cudaStream_t s);
 EBAG_DECLARE_LAUNCHERS(f32)
 EBAG_DECLARE_LAUNCHERS(f16)
 EBAG_DECLARE_LAUNCHERS(bf16)
@@ -673,14 +952,44 @@ EBAG_DECLARE_LAUNCHERS(int8)
 #define EBAG_DEFINE_LAUNCHERS(NAME, DT)                                                          \
     cudaError_t launch_fwd_##NAME(const FwdParams& p, bool weighted, bool mapid, int grid,        \
                                   size_t smem, cudaStream_t s) {                                 \
+        /* may be made resident while the kernel before it on the stream drains: the kernel's    \
+           first instruction waits for that kernel to finish and for its writes */               \
+        cudaLaunchAttribute attr[1];                                                             \
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;                         \
+        attr[0].val.programmaticStreamSerializationAllowed = 1;                                  \
+        cudaLaunchConfig_t cfg = {};                                                             \
+        cfg.gridDim = dim3((unsigned)grid);                                                      \
+        cfg.blockDim = dim3(kThreads);                                                           \
+        cfg.dynamicSmemBytes = smem;                                                             \
+        cfg.stream = s;                                                                          \
+        cfg.attrs = attr;                                                                        \
+        cfg.numAttrs = 1;                                                                        \
         if (mapid) {                                                                             \
-            if (weighted) ebag_fwd_kernel<DT, true, true><<<grid, kThreads, smem, s>>>(p);        \
-            else ebag_fwd_kernel<DT, false, true><<<grid, kThreads, smem, s>>>(p);                \
-        } else {                                                                                 \
-            if (weighted) ebag_fwd_kernel<DT, true, false><<<grid, kThreads, smem, s>>>(p);       \
-            else ebag_fwd_kernel<DT, false, false><<<grid, kThreads, smem, s>>>(p);               \
+            if (weighted) return cudaLaunchKernelEx(&cfg, ebag_fwd_kernel<DT, true, true>, p);    \
+            return cudaLaunchKernelEx(&cfg, ebag_fwd_kernel<DT, false, true>, p);                \
         }                                                                                        \
-        return cudaGetLastError();                                                               \
+        if (weighted) return cudaLaunchKernelEx(&cfg, ebag_fwd_kernel<DT, true, false>, p);       \
+        return cudaLaunchKernelEx(&cfg, ebag_fwd_kernel<DT, false, false>, p);                   \
+    }                                                                                            \
+    cudaError_t launch_parts_##NAME(const FwdParams& p, bool weighted, bool mapid, int grid,      \
+                                    cudaStream_t s) {                                            \
+        /* may be made resident while the forward kernel drains (it waits for it on the device) */\
+        cudaLaunchAttribute attr[1];                                                             \
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;                         \
+        attr[0].val.programmaticStreamSerializationAllowed = 1;                                  \
+        cudaLaunchConfig_t cfg = {};                                                             \
+        cfg.gridDim = dim3((unsigned)grid);                                                      \
+        cfg.blockDim = dim3(kThreads);                                                           \
+        cfg.dynamicSmemBytes = 0;                                                                \
+        cfg.stream = s;                                                                          \
+        cfg.attrs = attr;                                                                        \
+        cfg.numAttrs = 1;                                                                        \
+        if (mapid) {                                                                             \
+            if (weighted) return cudaLaunchKernelEx(&cfg, ebag_parts_kernel<DT, true, true>, p);  \
+            return cudaLaunchKernelEx(&cfg, ebag_parts_kernel<DT, false, true>, p);              \
+        }                                                                                        \
+        if (weighted) return cudaLaunchKernelEx(&cfg, ebag_parts_kernel<DT, true, false>, p);     \
+        return cudaLaunchKernelEx(&cfg, ebag_parts_kernel<DT, false, false>, p);                 \
     }                                                                                            \
     cudaError_t occupancy_fwd_##NAME(bool weighted, bool mapid, size_t smem, int* n) {            \
         const void* k = mapid ? (weighted ? (const void*)ebag_fwd_kernel<DT, true, true>          \

@@ -202,6 +202,7 @@ extern "C" ebag_status ebag_forward_noalloc(int32_t T, const int64_t* rows, cons
     p.sumD = (int32_t)d_off;
     p.mean = mode == EBAG_MEAN ? 1 : 0;
     p.item_bytes = 32768;
+    p.lg = LongParams{};                     // no room for partial sums here: bags are not split
     const bool w = per_sample_weights != nullptr;
     const int grid = st->num_sms * st->occupancy[dtype][w ? 1 : 0];
     if (launch(dtype, p, w, grid, fwd_smem_bytes(T), s) != cudaSuccess) {

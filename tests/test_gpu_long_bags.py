@@ -1,0 +1,148 @@
+"""Bags long enough to be split: the grid pools them in parts and the partial sums are added in
+part order.  Parity with the oracle at the usual tolerance, the same answer bit for bit on every
+run, agreement with the unsplit path, and the fall-backs when the bookkeeping runs out of room."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2512_23236_b200 as eb
+from oracle import ebag_oracle as orc
+from paper_2512_23236_b200 import workloads as wl
+
+from parity_util import compare, device_tables, oracle_tables, run_gpu
+
+pytestmark = pytest.mark.gpu
+
+
+def _tables(dtype, rows, D, seed):
+    w = wl.Workload(number=0, name="long bags", dtype=dtype, rows=list(rows), D=list(D), B=1,
+                    mode=wl.SUM, weighted=False, length_kind="uniform_int", length_params=[1.0] * len(rows),
+                    length_cap=1, index_kind="uniform", zipf_alpha=0.0, value_std=1.0, seed=seed)
+    return wl.gen_tables(w, "cpu")
+
+
+def _jagged(rng, rows, B, lengths, weighted):
+    """lengths: [T*B] ints.  Ids uniform over each table's rows."""
+    T = len(rows)
+    lengths = np.asarray(lengths, dtype=np.int64)
+    offsets = np.zeros(T * B + 1, dtype=np.int64)
+    np.cumsum(lengths, out=offsets[1:])
+    idx = np.concatenate([rng.integers(0, rows[t], size=int(lengths[t * B:(t + 1) * B].sum()))
+                          for t in range(T)]).astype(np.int64)
+    w = rng.uniform(-1.0, 1.0, size=idx.size).astype(np.float32) if weighted else None
+    return idx, offsets, w, lengths
+
+
+def _check(dtype, rows, D, B, lengths, mode=wl.SUM, weighted=False, seed=0, params=None,
+           spoil=None, raw=None, same_bits=True):
+    rng = np.random.default_rng(seed)
+    tables = _tables(dtype, rows, D, seed)
+    if raw is not None:
+        idx, off, w = raw
+    else:
+        idx, off, w, lengths = _jagged(rng, rows, B, lengths, weighted)
+    if spoil is not None:
+        spoil(idx, off)
+    dev = device_tables(dtype, tables)
+    tabs, sc, bi = oracle_tables(dtype, tables)
+    ref = orc.forward(tabs, dtype, idx, off, B, mode, weights=w, scales=sc, biases=bi)
+    gpu1, st1 = run_gpu(dtype, rows, D, dev, idx, off, B, mode, w, params)
+    gpu2, st2 = run_gpu(dtype, rows, D, dev, idx, off, B, mode, w, params)
+    whole, st3 = run_gpu(dtype, rows, D, dev, idx, off, B, mode, w, {"split_bytes": 0})
+    assert st1[1:] == st2[1:] == st3[1:] == (ref["n_oob"], ref["n_bad_offsets"])
+    T = len(rows)
+    clean = lengths if spoil is None and raw is None else None
+    compare(gpu1, ref, dtype, clean, T, B, D)
+    compare(gpu2, ref, dtype, clean, T, B, D)
+    compare(whole, ref, dtype, clean, T, B, D)
+    if same_bits:
+        assert np.array_equal(gpu1.view(np.uint32), gpu2.view(np.uint32)), "split bags: runs differ"
+    return gpu1, whole
+
+
+def _mixed_lengths(rng, T, B, long_at):
+    lengths = rng.integers(0, 20, size=T * B)
+    for pos, n in long_at.items():
+        lengths[pos] = n
+    return lengths
+
+
+@pytest.mark.parametrize("dtype,D", [(wl.F32, 64), (wl.BF16, 32), (wl.F16, 128), (wl.INT8_ROWWISE, 128),
+                                     (wl.F32, 512), (wl.BF16, 1024)])
+@pytest.mark.parametrize("mode,weighted", [(wl.SUM, False), (wl.MEAN, False), (wl.SUM, True)])
+def test_long_bags_among_short_ones(dtype, D, mode, weighted):
+    rng = np.random.default_rng(5)
+    T, B = 3, 40
+    rows = [50_000, 3_000, 20_000]
+    stride = max(eb.ebag_row_stride(dtype, D), 256)      # narrower rows count as 256 bytes
+    long_len = -(-65536 // stride)                       # shortest bag that is split by default
+    lengths = _mixed_lengths(rng, T, B, {3: 9 * long_len, 17: long_len, 39: 2 * long_len + 5,
+                                          40: long_len - 1, 2 * B: 3 * long_len,
+                                          3 * B - 1: 5 * long_len + 1})
+    gpu, whole = _check(dtype, rows, [D] * T, B, lengths, mode, weighted, seed=int(dtype) + D)
+    # the bag one lookup short of the threshold took the ordinary path in both runs
+    assert np.array_equal(gpu[0, D:2 * D].view(np.uint32), whole[0, D:2 * D].view(np.uint32))
+
+
+@pytest.mark.parametrize("dtype,D,L", [(wl.BF16, 128, 200_000), (wl.F32, 16, 300_000),
+                                       (wl.INT8_ROWWISE, 64, 150_000)])
+def test_one_huge_bag(dtype, D, L):
+    # a single bag: the most parts a bag may have, every row group of a part busy
+    _check(dtype, [100_000], [D], 1, [L], wl.MEAN, False, seed=L)
+
+
+def test_mixed_widths_in_one_call():
+    rng = np.random.default_rng(9)
+    rows = [10_000, 10_000, 10_000, 10_000]
+    D = [16, 64, 256, 1024]
+    B = 12
+    lengths = _mixed_lengths(rng, 4, B, {5: 9000, B + 1: 2100, 2 * B + 11: 700, 3 * B: 300})
+    _check(wl.F32, rows, D, B, lengths, wl.SUM, True, seed=2)
+
+
+def test_many_long_bags():
+    # 1500 bags a little over the threshold, five parts each
+    B = 1500
+    lengths = np.full(B, 260)
+    _check(wl.F32, [40_000], [64], B, lengths, wl.SUM, False, seed=3)
+
+
+def test_low_threshold_many_parts():
+    # a low threshold makes every bag long: the library raises it just enough for all parts to fit
+    B = 300
+    lengths = np.full(B, 100)
+    _check(wl.F32, [40_000], [64], B, lengths, wl.MEAN, False, seed=4, params={"split_bytes": 1024})
+
+
+def test_overlapping_bags_outrun_the_bookkeeping():
+    # Offsets that go 0, N, 0, N, ... make every other bag cover the same N lookups (the bags in
+    # between are malformed): far more long bags than the lookups of the call could otherwise
+    # hold, so the records run out and the bags that find no room are pooled whole.  Which ones
+    # those are depends on timing, so only the tolerance is checked.
+    N, B = 300, 10_000
+    rng = np.random.default_rng(8)
+    idx = rng.integers(0, 40_000, size=N).astype(np.int64)
+    off = np.zeros(B + 1, dtype=np.int64)
+    off[1::2] = N
+    off[B] = N
+    _check(wl.F32, [40_000], [64], B, None, wl.SUM, False, seed=5, raw=(idx, off, None), same_bits=False)
+
+
+def test_rejected_ids_and_malformed_bags_next_to_long_ones():
+    def spoil(idx, off):
+        idx[100:140] = -7                 # inside the long bag 0
+        idx[5000] = 10**12
+        off[6] = off[5] - 3               # bags 5 and 6 become malformed
+    lengths = [6000, 3, 0, 700, 2, 9, 4, 1, 650, 12]
+    _check(wl.BF16, [9_000], [128], 10, lengths, wl.SUM, True, seed=6, spoil=spoil)
+
+
+def test_split_parameter_is_validated():
+    tbe = eb.TBE([10], [16], wl.F32)
+    try:
+        with pytest.raises(Exception):
+            tbe.set_param("split_bytes", 100)
+        tbe.set_param("split_bytes", 0)
+        tbe.set_param("split_bytes", 1 << 20)
+    finally:
+        tbe.close()
