@@ -174,22 +174,35 @@ template <> struct Elem<DT_F16>  { static constexpr int kAcc = 8; };
 template <> struct Elem<DT_BF16> { static constexpr int kAcc = 8; };
 template <> struct Elem<DT_INT8> { static constexpr int kAcc = 16; };
 
+// Two fp32 operations per instruction (sm_100a): the pair sits in an aligned register pair.
+__device__ __forceinline__ void fma2(float& a0, float& a1, float w, float x0, float x1) {
+    const float2 r = __ffma2_rn(make_float2(w, w), make_float2(x0, x1), make_float2(a0, a1));
+    a0 = r.x;
+    a1 = r.y;
+}
+__device__ __forceinline__ void add2(float& a0, float& a1, float x0, float x1) {
+    const float2 r = __fadd2_rn(make_float2(a0, a1), make_float2(x0, x1));
+    a0 = r.x;
+    a1 = r.y;
+}
+
 // acc[0..kAcc) += w * widen(d)        (int8: w is w*scale; the bias term is summed separately)
 template <int DT, bool WEIGHTED>
 __device__ __forceinline__ void accumulate(float* acc, const uint4& d, float w) {
     const uint32_t r[4] = {d.x, d.y, d.z, d.w};
     if constexpr (DT == DT_F32) {
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const float x = __uint_as_float(r[i]);
-            acc[i] = WEIGHTED ? fmaf(w, x, acc[i]) : acc[i] + x;
+        for (int i = 0; i < 4; i += 2) {
+            const float x0 = __uint_as_float(r[i]), x1 = __uint_as_float(r[i + 1]);
+            if constexpr (WEIGHTED) fma2(acc[i], acc[i + 1], w, x0, x1);
+            else add2(acc[i], acc[i + 1], x0, x1);
         }
     } else if constexpr (DT == DT_BF16) {
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
             if constexpr (WEIGHTED) {
-                acc[2 * i] = fmaf(w, __uint_as_float(r[i] << 16), acc[2 * i]);
-                acc[2 * i + 1] = fmaf(w, __uint_as_float(r[i] & 0xffff0000u), acc[2 * i + 1]);
+                fma2(acc[2 * i], acc[2 * i + 1], w, __uint_as_float(r[i] << 16),
+                     __uint_as_float(r[i] & 0xffff0000u));
             } else {
                 add_bf16(acc[2 * i], r[i]);
                 add_bf16(acc[2 * i + 1], r[i] >> 16);
@@ -200,8 +213,7 @@ __device__ __forceinline__ void accumulate(float* acc, const uint4& d, float w) 
         for (int i = 0; i < 4; ++i) {
             if constexpr (WEIGHTED) {
                 const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&r[i]));
-                acc[2 * i] = fmaf(w, f.x, acc[2 * i]);
-                acc[2 * i + 1] = fmaf(w, f.y, acc[2 * i + 1]);
+                fma2(acc[2 * i], acc[2 * i + 1], w, f.x, f.y);
             } else {
                 add_f16(acc[2 * i], r[i]);
                 add_f16(acc[2 * i + 1], r[i] >> 16);
@@ -213,9 +225,11 @@ __device__ __forceinline__ void accumulate(float* acc, const uint4& d, float w) 
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
 #pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                const float f = __uint_as_float(__byte_perm(r[i], 0x4B000000u, 0x7440 + k));
-                acc[4 * i + k] = fmaf(w, f - 8388736.0f, acc[4 * i + k]);
+            for (int k = 0; k < 4; k += 2) {
+                float f0 = __uint_as_float(__byte_perm(r[i], 0x4B000000u, 0x7440 + k));
+                float f1 = __uint_as_float(__byte_perm(r[i], 0x4B000000u, 0x7441 + k));
+                add2(f0, f1, -8388736.0f, -8388736.0f);
+                fma2(acc[4 * i + k], acc[4 * i + k + 1], w, f0, f1);
             }
         }
     }
