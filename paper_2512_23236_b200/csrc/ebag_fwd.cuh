@@ -175,37 +175,33 @@ template <> struct Elem<DT_BF16> { static constexpr int kAcc = 8; };
 template <> struct Elem<DT_INT8> { static constexpr int kAcc = 16; };
 
 // Two fp32 operations per instruction (sm_100a): the pair sits in an aligned register pair.
-__device__ __forceinline__ void fma2(float& a0, float& a1, float w, float x0, float x1) {
-    const float2 r = __ffma2_rn(make_float2(w, w), make_float2(x0, x1), make_float2(a0, a1));
-    a0 = r.x;
-    a1 = r.y;
+__device__ __forceinline__ void fma2(float2& a, float w, float x0, float x1) {
+    a = __ffma2_rn(make_float2(w, w), make_float2(x0, x1), a);
 }
-__device__ __forceinline__ void add2(float& a0, float& a1, float x0, float x1) {
-    const float2 r = __fadd2_rn(make_float2(a0, a1), make_float2(x0, x1));
-    a0 = r.x;
-    a1 = r.y;
+__device__ __forceinline__ void add2(float2& a, float x0, float x1) {
+    a = __fadd2_rn(a, make_float2(x0, x1));
 }
 
 // acc[0..kAcc) += w * widen(d)        (int8: w is w*scale; the bias term is summed separately)
 template <int DT, bool WEIGHTED>
-__device__ __forceinline__ void accumulate(float* acc, const uint4& d, float w) {
+__device__ __forceinline__ void accumulate(float2* acc, const uint4& d, float w) {
     const uint32_t r[4] = {d.x, d.y, d.z, d.w};
     if constexpr (DT == DT_F32) {
 #pragma unroll
         for (int i = 0; i < 4; i += 2) {
             const float x0 = __uint_as_float(r[i]), x1 = __uint_as_float(r[i + 1]);
-            if constexpr (WEIGHTED) fma2(acc[i], acc[i + 1], w, x0, x1);
-            else add2(acc[i], acc[i + 1], x0, x1);
+            if constexpr (WEIGHTED) fma2(acc[i / 2], w, x0, x1);
+            else add2(acc[i / 2], x0, x1);
         }
     } else if constexpr (DT == DT_BF16) {
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
             if constexpr (WEIGHTED) {
-                fma2(acc[2 * i], acc[2 * i + 1], w, __uint_as_float(r[i] << 16),
+                fma2(acc[i], w, __uint_as_float(r[i] << 16),
                      __uint_as_float(r[i] & 0xffff0000u));
             } else {
-                add_bf16(acc[2 * i], r[i]);
-                add_bf16(acc[2 * i + 1], r[i] >> 16);
+                add_bf16(acc[i].x, r[i]);
+                add_bf16(acc[i].y, r[i] >> 16);
             }
         }
     } else if constexpr (DT == DT_F16) {
@@ -213,27 +209,32 @@ __device__ __forceinline__ void accumulate(float* acc, const uint4& d, float w) 
         for (int i = 0; i < 4; ++i) {
             if constexpr (WEIGHTED) {
                 const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&r[i]));
-                fma2(acc[2 * i], acc[2 * i + 1], w, f.x, f.y);
+                fma2(acc[i], w, f.x, f.y);
             } else {
-                add_f16(acc[2 * i], r[i]);
-                add_f16(acc[2 * i + 1], r[i] >> 16);
+                add_f16(acc[i].x, r[i]);
+                add_f16(acc[i].y, r[i] >> 16);
             }
         }
     } else {
-        // Stored code u = q + 128 (0..255).  Dropping the byte into the mantissa of 2^23 gives the
-        // float 2^23 + u; subtracting 2^23 + 128 leaves q, exactly, without the conversion pipe.
+        // Stored code u = q + 128 (0..255).  The byte dropped into bits 16..23 of a zero word IS
+        // the float u * 2^-133, exactly, for every u (subnormal below 128, and the subnormal to
+        // normal step at 128 is seamless), so widening costs one byte-permute and no arithmetic.
+        // The caller passes w = weight * scale * 2^kInt8Up, the sums come out scaled by
+        // 2^(kInt8Up - 133) and are scaled back, exactly, when the bag is written; the -128 of
+        // every code goes into the bias term, one scalar per row.
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
 #pragma unroll
             for (int k = 0; k < 4; k += 2) {
-                float f0 = __uint_as_float(__byte_perm(r[i], 0x4B000000u, 0x7440 + k));
-                float f1 = __uint_as_float(__byte_perm(r[i], 0x4B000000u, 0x7441 + k));
-                add2(f0, f1, -8388736.0f, -8388736.0f);
-                fma2(acc[4 * i + k], acc[4 * i + k + 1], w, f0, f1);
+                const float f0 = __uint_as_float(__byte_perm(r[i], 0u, 0x4044 + (k << 8)));
+                const float f1 = __uint_as_float(__byte_perm(r[i], 0u, 0x4144 + (k << 8)));
+                fma2(acc[2 * i + k / 2], w, f0, f1);
             }
         }
     }
 }
+constexpr float kInt8Up = 0x1p64f;       // weight * scale travels as weight * scale * 2^64
+constexpr float kInt8Down = 0x1p69f;     // 2^(133 - 64)
 
 // Sort 32 keys, one per lane, in descending order (bitonic network, 15 exchange steps).
 __device__ __forceinline__ uint32_t warp_sort_desc(uint32_t v, int lane) {
@@ -534,12 +535,12 @@ __device__ __forceinline__ void process_item(const FwdParams& p, const TableMeta
             }
         }
     };
-    float acc[V][NACC];
+    float2 acc[V][NACC / 2];                         // pairs: two fp32 operations per instruction
     float acc_bias = 0.0f;
 #pragma unroll
     for (int v = 0; v < V; ++v)
 #pragma unroll
-        for (int a = 0; a < NACC; ++a) acc[v][a] = 0.0f;
+        for (int a = 0; a < NACC / 2; ++a) acc[v][a] = make_float2(0.0f, 0.0f);
     auto consume = [&](const IdChunk& c, int j0, int st) {
         if (c.clean && j0 + CR <= c.nmin) {
 #pragma unroll
@@ -549,6 +550,8 @@ __device__ __forceinline__ void process_item(const FwdParams& p, const TableMeta
                     const float2 sb = my_sb[(st * kStageVecs + u) * 8];
                     acc_bias = fmaf(wu, sb.y, acc_bias);
                     wu *= sb.x;
+                    acc_bias = fmaf(wu, -128.0f, acc_bias);
+                    wu *= kInt8Up;
                 }
 #pragma unroll
                 for (int v = 0; v < V; ++v) {
@@ -567,6 +570,8 @@ __device__ __forceinline__ void process_item(const FwdParams& p, const TableMeta
                     const float2 sb = my_sb[(st * kStageVecs + u) * 8];
                     acc_bias = fmaf(wu, sb.y, acc_bias);
                     wu *= sb.x;
+                    acc_bias = fmaf(wu, -128.0f, acc_bias);
+                    wu *= kInt8Up;
                 }
 #pragma unroll
                 for (int v = 0; v < V; ++v)
@@ -593,22 +598,28 @@ __device__ __forceinline__ void process_item(const FwdParams& p, const TableMeta
                 if (!col_on[v]) continue;
                 float* o = orow + (size_t)(vec0 + v * G + lig) * NACC;
 #pragma unroll
-                for (int a = 0; a < NACC; ++a) {
-                    float x = acc[v][a];
-                    if (DT == DT_INT8) x += acc_bias;
-                    if (!PART && p.mean && L > 0) x = __fdiv_rn(x, (float)L);
+                for (int a = 0; a < NACC / 2; ++a) {
+                    float2 x = acc[v][a];
+                    if (DT == DT_INT8) {
+                        x.x = fmaf(x.x, kInt8Down, acc_bias);
+                        x.y = fmaf(x.y, kInt8Down, acc_bias);
+                    }
+                    if (!PART && p.mean && L > 0) {
+                        x.x = __fdiv_rn(x.x, (float)L);
+                        x.y = __fdiv_rn(x.y, (float)L);
+                    }
                     acc[v][a] = x;
                 }
 #pragma unroll
-                for (int a = 0; a < NACC; a += 4)
-                    st_stream16(o + a, acc[v][a], acc[v][a + 1], acc[v][a + 2], acc[v][a + 3]);
+                for (int a = 0; a < NACC / 2; a += 2)
+                    st_stream16(o + 2 * a, acc[v][a].x, acc[v][a].y, acc[v][a + 1].x, acc[v][a + 1].y);
             }
         }
         acc_bias = 0.0f;
 #pragma unroll
         for (int v = 0; v < V; ++v)
 #pragma unroll
-            for (int a = 0; a < NACC; ++a) acc[v][a] = 0.0f;
+            for (int a = 0; a < NACC / 2; ++a) acc[v][a] = make_float2(0.0f, 0.0f);
     };
 
     // ---- pipeline: the request side runs one stage ahead of the consuming side
