@@ -504,9 +504,11 @@ __device__ __forceinline__ void process_item(const FwdParams& p, const TableMeta
     const bool cols_full = __all_sync(0xffffffffu, my_cols);
     // this lane's slots: vector k of stage st is at my_rows[(st * kStageVecs + k) * 32]
     const uint4* my_rows = wbuf + lane;
-    const uint32_t my_rows_s = (uint32_t)__cvta_generic_to_shared(wbuf) + lane * 16;
+    uint32_t my_rows_s = (uint32_t)__cvta_generic_to_shared(wbuf) + lane * 16;
+    asm volatile("" : "+r"(my_rows_s));
     const float2* my_sb = sbbuf + grp;               // int8: scale/bias of row u at [(st*kStageVecs+u)*8]
-    const uint32_t my_sb_s = (uint32_t)__cvta_generic_to_shared(sbbuf) + grp * 8;
+    uint32_t my_sb_s = (uint32_t)__cvta_generic_to_shared(sbbuf) + grp * 8;
+    asm volatile("" : "+r"(my_sb_s));
     auto issue = [&](const IdChunk& c, int j0, int st) {
         if (c.clean && j0 + CR <= c.nmin) {          // full stage, nothing to check
 #pragma unroll
@@ -686,9 +688,10 @@ ebag_fwd_kernel(const FwdParams p) {
     __shared__ float total_bytes;
     __shared__ uint4 stage_buf[kWarps * kWarpSmemVecs];      // per warp: 4 KB ring + the item's bags
     __shared__ float2 sb_buf[DT == DT_INT8 ? kWarps * kStages * kStageVecs * 8 : 1];
-    uint4* wbuf = stage_buf + (threadIdx.x >> 5) * kWarpSmemVecs;
-    float2* sbbuf = sb_buf + (DT == DT_INT8 ? (threadIdx.x >> 5) * (kStages * kStageVecs * 8) : 0);
-    const int tid = threadIdx.x;
+    int tid;
+    asm volatile("mov.u32 %0, %%tid.x;" : "=r"(tid));      // read once: not re-read wherever a use is
+    uint4* wbuf = stage_buf + (tid >> 5) * kWarpSmemVecs;
+    float2* sbbuf = sb_buf + (DT == DT_INT8 ? (tid >> 5) * (kStages * kStageVecs * 8) : 0);
     const int lane = tid & 31;
 
     // This launch may have been made resident before the kernel ahead of it on the stream
@@ -811,9 +814,10 @@ ebag_parts_kernel(const FwdParams p) {
     __shared__ float2 sb_buf[DT == DT_INT8 ? kWarps * kStages * kStageVecs * 8 : 1];
     __shared__ unsigned part0_s[kMaxLongBags + 1];     // first part of every recorded bag
     __shared__ unsigned scan_warp_s[kWarps], scan_carry_s;
-    uint4* wbuf = stage_buf + (threadIdx.x >> 5) * kWarpSmemVecs;
-    float2* sbbuf = sb_buf + (DT == DT_INT8 ? (threadIdx.x >> 5) * (kStages * kStageVecs * 8) : 0);
-    const int tid = threadIdx.x;
+    int tid;
+    asm volatile("mov.u32 %0, %%tid.x;" : "=r"(tid));      // read once: not re-read wherever a use is
+    uint4* wbuf = stage_buf + (tid >> 5) * kWarpSmemVecs;
+    float2* sbbuf = sb_buf + (DT == DT_INT8 ? (tid >> 5) * (kStages * kStageVecs * 8) : 0);
     const int lane = tid & 31;
 
     // this launch may have been made resident before the forward kernel finished: wait for it
