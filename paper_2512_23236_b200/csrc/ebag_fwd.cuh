@@ -146,6 +146,23 @@ __device__ __forceinline__ void cp_async16(uint32_t smem, const void* gmem) {
 __device__ __forceinline__ void cp_async8(uint32_t smem, const void* gmem) {
     asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(smem), "l"(gmem));
 }
+// Loads from the shared window by its 32-bit address (no generic pointer to keep alongside it).
+__device__ __forceinline__ uint4 lds128(uint32_t a) {
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a));
+    return v;
+}
+__device__ __forceinline__ uint32_t lds32(uint32_t a) {
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(a));
+    return v;
+}
+__device__ __forceinline__ float2 lds64f(uint32_t a) {
+    float2 v;
+    asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(a));
+    return v;
+}
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;"); }
 template <int N>
 __device__ __forceinline__ void cp_async_wait() {
@@ -420,6 +437,10 @@ __device__ __forceinline__ void process_item(const FwdParams& p, const TableMeta
     bagw[32 + lane] = off_hi;
     bagw[64 + lane] = key;
     __syncwarp();
+    // this lane's slots in the ring, as addresses in the shared window: vector k of stage st is
+    // at my_rows_s + (st * kStageVecs + k) * 512 (kept opaque: not to be recomputed at every use)
+    uint32_t my_rows_s = (uint32_t)__cvta_generic_to_shared(wbuf) + lane * 16;
+    asm volatile("" : "+r"(my_rows_s));
     const int64_t* __restrict__ idx_base = p.indices + base;
     const float* __restrict__ w_base = WEIGHTED ? p.weights + base : nullptr;
 
@@ -433,7 +454,7 @@ __device__ __forceinline__ void process_item(const FwdParams& p, const TableMeta
     }
     const uint32_t stride = (uint32_t)m.stride;
     const uint32_t rows = (uint32_t)m.rows;          // tables have fewer than 2^31 rows
-    const char* sb_base = tbase + m.D;
+    const int sb_delta = m.D - vec0 * 16;            // int8, lane 0 of a group: from its row vector to the scale/bias pair
     const int nslots = (cnt + NG - 1) >> (5 - m.g_log2);
 
     const int64_t* __restrict__ map_ptr = MAPID ? p.mappings[t] : nullptr;
@@ -458,11 +479,12 @@ __device__ __forceinline__ void process_item(const FwdParams& p, const TableMeta
         }
     };
     auto slot_bag = [&](int pos_in_item, uint32_t& s, uint32_t& e, int& orig, bool& elsewhere) {
-        const uint32_t k = bagw[64 + (pos_in_item & 31)];
+        const uint32_t bag_s = my_rows_s - lane * 16 + kStages * kStageVecs * 512;   // after the ring
+        const uint32_t k = lds32(bag_s + 256 + (pos_in_item & 31) * 4);
         orig = (int)(k & 31u);
         elsewhere = (k & 32u) != 0;
-        s = bagw[orig];
-        e = bagw[32 + orig];
+        s = lds32(bag_s + orig * 4);
+        e = lds32(bag_s + 128 + orig * 4);
         if (pos_in_item >= cnt) s = e = 0;
     };
 
@@ -502,11 +524,6 @@ __device__ __forceinline__ void process_item(const FwdParams& p, const TableMeta
 #pragma unroll
     for (int v = 0; v < V; ++v) my_cols = my_cols && col_on[v];
     const bool cols_full = __all_sync(0xffffffffu, my_cols);
-    // this lane's slots: vector k of stage st is at my_rows[(st * kStageVecs + k) * 32]
-    const uint4* my_rows = wbuf + lane;
-    uint32_t my_rows_s = (uint32_t)__cvta_generic_to_shared(wbuf) + lane * 16;
-    asm volatile("" : "+r"(my_rows_s));
-    const float2* my_sb = sbbuf + grp;               // int8: scale/bias of row u at [(st*kStageVecs+u)*8]
     uint32_t my_sb_s = (uint32_t)__cvta_generic_to_shared(sbbuf) + grp * 8;
     asm volatile("" : "+r"(my_sb_s));
     auto issue = [&](const IdChunk& c, int j0, int st) {
@@ -519,7 +536,7 @@ __device__ __forceinline__ void process_item(const FwdParams& p, const TableMeta
                 for (int v = 0; v < V; ++v)
                     cp_async16(my_rows_s + (st * kStageVecs + u * V + v) * 512, lane_base[v] + roff);
                 if (DT == DT_INT8 && lig == 0)
-                    cp_async8(my_sb_s + (st * kStageVecs + u) * 64, sb_base + roff);
+                    cp_async8(my_sb_s + (st * kStageVecs + u) * 64, lane_base[0] + roff + sb_delta);
             }
             return;
         }
@@ -533,7 +550,7 @@ __device__ __forceinline__ void process_item(const FwdParams& p, const TableMeta
                     if (col_on[v])
                         cp_async16(my_rows_s + (st * kStageVecs + u * V + v) * 512, lane_base[v] + roff);
                 if (DT == DT_INT8 && lig == 0)
-                    cp_async8(my_sb_s + (st * kStageVecs + u) * 64, sb_base + roff);
+                    cp_async8(my_sb_s + (st * kStageVecs + u) * 64, lane_base[0] + roff + sb_delta);
             }
         }
     };
@@ -549,7 +566,7 @@ __device__ __forceinline__ void process_item(const FwdParams& p, const TableMeta
             for (int u = 0; u < CR; ++u) {
                 float wu = WEIGHTED ? __shfl_sync(0xffffffffu, c.w, j0 + u, G) : 1.0f;
                 if (DT == DT_INT8) {
-                    const float2 sb = my_sb[(st * kStageVecs + u) * 8];
+                    const float2 sb = lds64f(my_sb_s + (st * kStageVecs + u) * 64);
                     acc_bias = fmaf(wu, sb.y, acc_bias);
                     wu *= sb.x;
                     acc_bias = fmaf(wu, -128.0f, acc_bias);
@@ -557,7 +574,7 @@ __device__ __forceinline__ void process_item(const FwdParams& p, const TableMeta
                 }
 #pragma unroll
                 for (int v = 0; v < V; ++v) {
-                    const uint4 d = my_rows[(st * kStageVecs + u * V + v) * 32];
+                    const uint4 d = lds128(my_rows_s + (st * kStageVecs + u * V + v) * 512);
                     accumulate<DT, WEIGHTED || DT == DT_INT8>(acc[v], d, wu);
                 }
             }
@@ -569,7 +586,7 @@ __device__ __forceinline__ void process_item(const FwdParams& p, const TableMeta
             float wu = WEIGHTED ? __shfl_sync(0xffffffffu, c.w, j0 + u, G) : 1.0f;
             if (j0 + u < c.nmax && r != kInvalidRow) {
                 if (DT == DT_INT8) {
-                    const float2 sb = my_sb[(st * kStageVecs + u) * 8];
+                    const float2 sb = lds64f(my_sb_s + (st * kStageVecs + u) * 64);
                     acc_bias = fmaf(wu, sb.y, acc_bias);
                     wu *= sb.x;
                     acc_bias = fmaf(wu, -128.0f, acc_bias);
@@ -578,7 +595,7 @@ __device__ __forceinline__ void process_item(const FwdParams& p, const TableMeta
 #pragma unroll
                 for (int v = 0; v < V; ++v)
                     if (col_on[v]) {
-                        const uint4 d = my_rows[(st * kStageVecs + u * V + v) * 32];
+                        const uint4 d = lds128(my_rows_s + (st * kStageVecs + u * V + v) * 512);
                         accumulate<DT, WEIGHTED || DT == DT_INT8>(acc[v], d, wu);
                     }
             }
