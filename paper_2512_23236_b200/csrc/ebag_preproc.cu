@@ -104,10 +104,10 @@ extern "C" ebag_status ebag_mbdt(const float* values, int32_t F, int64_t B, cons
 // of a nested jagged batch, all features in a constant number of launches.  The kept events of a
 // user are a prefix of that user's events, so per feature a user's kept inner lengths and kept
 // values are each ONE contiguous range; only user-level prefix sums are needed:
-//   1. scan outer lengths            -> first event of every user, before and after (1 CTA)
-//   2. per (feature, user) sums      -> values held / kept by the user           (1 warp each)
-//   3. scan those per feature        -> first value of every user, before and after (1 CTA each)
-//   4. copy the two ranges per (feature, user)                                    (1 warp each)
+//   1. scan outer lengths            -> first event of every user, before and after (1 CTA per tile)
+//   2. per (feature, user) sums      -> values held / kept by the user   (a warp per 8 users)
+//   3. scan those per feature        -> first value of every user, before and after (1 CTA per tile)
+//   4. copy the two ranges per (feature, user)                            (a warp per 8 users)
 namespace {
 
 constexpr int kScanThreads = 1024;
@@ -133,140 +133,285 @@ __host__ __device__ inline BetWorkspace carve(void* ws, int F, int64_t U) {
     return w;
 }
 
-// exclusive prefix sums of a[0..n) and b[0..n) by one CTA, totals written at index n.
-// Every thread owns kScanItems consecutive entries per round (negative entries count as 0).
+// Exclusive prefix sums of a[0..n) and b[0..n), totals written at index n (negative entries count
+// as 0), by a grid of CTAs with no communication between them: the CTA of tile c first ADDS UP
+// everything before its tile (a plain reduction with many loads in flight, served by L2 once the
+// first CTA has touched the data; redundant, but a few hundred KB), then scans its own tile of
+// kScanThreads * kScanItems entries in one round.  CLAMP: b is not read, b[i] = min(a[i], clamp)
+// and is also written to b_out.  At 32,768 entries a single CTA walking the tiles one after the
+// other took 56-60 us per scan, a fifth of the whole truncation.
 constexpr int kScanItems = 4;
-__device__ void block_exscan2(const int64_t* __restrict__ a, const int64_t* __restrict__ b, int64_t n,
-                              int64_t* __restrict__ sa, int64_t* __restrict__ sb) {
-    __shared__ int64_t warp_a[32], warp_b[32], carry[2];
+constexpr int kScanTile = kScanThreads * kScanItems;
+__device__ __forceinline__ int64_t nonneg(int64_t x) { return x < 0 ? 0 : x; }
+
+template <bool CLAMP>
+__device__ void tile_exscan2(const int64_t* __restrict__ a, const int64_t* __restrict__ b, int64_t clamp,
+                             int64_t n, int64_t tile, int64_t* __restrict__ b_out,
+                             int64_t* __restrict__ sa, int64_t* __restrict__ sb) {
+    __shared__ int64_t warp_a[32], warp_b[32], base[2];
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
-    if (tid == 0) carry[0] = carry[1] = 0;
-    __syncthreads();
-    for (int64_t base = 0; base < n; base += (int64_t)kScanThreads * kScanItems) {
-        const int64_t i0 = base + (int64_t)tid * kScanItems;
-        int64_t xa[kScanItems], xb[kScanItems];
-        int64_t ta = 0, tb = 0;                      // this thread's totals
+    const int64_t t0 = tile * kScanTile;
+    auto bval = [&](int64_t av, int64_t i) -> int64_t {
+        if (CLAMP) return av < clamp ? av : clamp;
+        return nonneg(b[i]);
+    };
+    // ---- everything before the tile
+    int64_t pa = 0, pb = 0;
+    for (int64_t i0 = tid; i0 < t0; i0 += (int64_t)kScanThreads * 8) {
+        int64_t xa[8], xb[8];
 #pragma unroll
-        for (int k = 0; k < kScanItems; ++k) {
-            xa[k] = i0 + k < n ? a[i0 + k] : 0;
-            xb[k] = i0 + k < n ? b[i0 + k] : 0;
-            if (xa[k] < 0) xa[k] = 0;
-            if (xb[k] < 0) xb[k] = 0;
-            ta += xa[k];
-            tb += xb[k];
+        for (int k = 0; k < 8; ++k) {
+            const int64_t i = i0 + (int64_t)k * kScanThreads;
+            xa[k] = i < t0 ? nonneg(a[i]) : 0;
+            xb[k] = i < t0 ? bval(xa[k], i) : 0;
         }
-        int64_t ia = ta, ib = tb;                    // inclusive over the threads of the warp
+#pragma unroll
+        for (int k = 0; k < 8; ++k) { pa += xa[k]; pb += xb[k]; }
+    }
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) {
+        pa += __shfl_xor_sync(0xffffffffu, pa, d);
+        pb += __shfl_xor_sync(0xffffffffu, pb, d);
+    }
+    if (lane == 0) { warp_a[wid] = pa; warp_b[wid] = pb; }
+    __syncthreads();
+    if (wid == 0) {
+        int64_t wa = warp_a[lane], wb = warp_b[lane];
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) {
+            wa += __shfl_xor_sync(0xffffffffu, wa, d);
+            wb += __shfl_xor_sync(0xffffffffu, wb, d);
+        }
+        if (lane == 0) { base[0] = wa; base[1] = wb; }
+    }
+    __syncthreads();
+    // ---- the tile itself: every thread owns kScanItems consecutive entries
+    const int64_t i0 = t0 + (int64_t)tid * kScanItems;
+    int64_t xa[kScanItems], xb[kScanItems];
+    int64_t ta = 0, tb = 0;                          // this thread's totals
+#pragma unroll
+    for (int k = 0; k < kScanItems; ++k) {
+        xa[k] = i0 + k < n ? nonneg(a[i0 + k]) : 0;
+        xb[k] = i0 + k < n ? bval(xa[k], i0 + k) : 0;
+        ta += xa[k];
+        tb += xb[k];
+    }
+    int64_t ia = ta, ib = tb;                        // inclusive over the threads of the warp
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const int64_t ya = __shfl_up_sync(0xffffffffu, ia, d), yb = __shfl_up_sync(0xffffffffu, ib, d);
+        if (lane >= d) { ia += ya; ib += yb; }
+    }
+    __syncthreads();                                 // warp_a / warp_b are reused
+    if (lane == 31) { warp_a[wid] = ia; warp_b[wid] = ib; }
+    __syncthreads();
+    if (wid == 0) {
+        int64_t wa = warp_a[lane], wb = warp_b[lane];
 #pragma unroll
         for (int d = 1; d < 32; d <<= 1) {
-            const int64_t ya = __shfl_up_sync(0xffffffffu, ia, d), yb = __shfl_up_sync(0xffffffffu, ib, d);
-            if (lane >= d) { ia += ya; ib += yb; }
+            const int64_t ya = __shfl_up_sync(0xffffffffu, wa, d), yb = __shfl_up_sync(0xffffffffu, wb, d);
+            if (lane >= d) { wa += ya; wb += yb; }
         }
-        if (lane == 31) { warp_a[wid] = ia; warp_b[wid] = ib; }
-        __syncthreads();
-        if (wid == 0) {
-            int64_t wa = warp_a[lane], wb = warp_b[lane];
-#pragma unroll
-            for (int d = 1; d < 32; d <<= 1) {
-                const int64_t ya = __shfl_up_sync(0xffffffffu, wa, d), yb = __shfl_up_sync(0xffffffffu, wb, d);
-                if (lane >= d) { wa += ya; wb += yb; }
-            }
-            warp_a[lane] = wa; warp_b[lane] = wb;      // inclusive over warps
-        }
-        __syncthreads();
-        int64_t ra = carry[0] + (wid ? warp_a[wid - 1] : 0) + ia - ta;   // exclusive for this thread
-        int64_t rb = carry[1] + (wid ? warp_b[wid - 1] : 0) + ib - tb;
-#pragma unroll
-        for (int k = 0; k < kScanItems; ++k) {
-            if (i0 + k < n) { sa[i0 + k] = ra; sb[i0 + k] = rb; }
-            ra += xa[k];
-            rb += xb[k];
-        }
-        __syncthreads();
-        if (tid == 0) { carry[0] += warp_a[31]; carry[1] += warp_b[31]; }
-        __syncthreads();
+        warp_a[lane] = wa; warp_b[lane] = wb;          // inclusive over warps
     }
-    if (tid == 0) { sa[n] = carry[0]; sb[n] = carry[1]; }
+    __syncthreads();
+    int64_t ra = base[0] + (wid ? warp_a[wid - 1] : 0) + ia - ta;   // exclusive for this thread
+    int64_t rb = base[1] + (wid ? warp_b[wid - 1] : 0) + ib - tb;
+#pragma unroll
+    for (int k = 0; k < kScanItems; ++k) {
+        if (i0 + k < n) {
+            sa[i0 + k] = ra;
+            sb[i0 + k] = rb;
+            if (CLAMP) b_out[i0 + k] = xb[k];
+        }
+        ra += xa[k];
+        rb += xb[k];
+    }
+    if (t0 + kScanTile >= n && tid == kScanThreads - 1) {           // the last tile also leaves the totals
+        sa[n] = base[0] + warp_a[31];
+        sb[n] = base[1] + warp_b[31];
+    }
 }
 
 __global__ void __launch_bounds__(kScanThreads)
 bet_scan_outer(const int64_t* __restrict__ outer, int64_t U, int64_t N, int64_t* __restrict__ outer_out,
                BetWorkspace w, int64_t* __restrict__ counts_out) {
-    for (int64_t u = threadIdx.x; u < U; u += kScanThreads) {
-        int64_t n = outer[u];
-        if (n < 0) n = 0;
-        outer_out[u] = n < N ? n : N;
+    tile_exscan2<true>(outer, nullptr, N, U, blockIdx.x, outer_out, w.ev_in, w.ev_out);
+    if ((int64_t)(blockIdx.x + 1) * kScanTile >= U) {
+        __syncthreads();
+        if (threadIdx.x == 0) counts_out[0] = w.ev_out[U];
     }
-    __syncthreads();
-    block_exscan2(outer, outer_out, U, w.ev_in, w.ev_out);
-    __syncthreads();
-    if (threadIdx.x == 0) counts_out[0] = w.ev_out[U];
 }
 
-// one warp per (feature, user): how many values the user holds and how many its kept events hold
-__global__ void bet_user_sums(const int64_t* __restrict__ inner, int64_t E, int64_t U, BetWorkspace w) {
-    const int f = blockIdx.y;
+constexpr int kCopyBatch = 4;       // 8-byte loads a lane keeps in flight
+constexpr int kTaskUsers = 8;       // users per warp task
+constexpr int kSumBatch = 6;        // bet_user_sums: loads per lane requested one user ahead (192 inner lengths)
+
+// How many values every user holds in a feature and how many its kept events hold.  A warp takes
+// kTaskUsers consecutive users of a feature at a time: a lane each reads the event range of one
+// of them, then the warp adds up the users' inner lengths one user after the other.  The grid is
+// one wave of resident CTAs and the (feature, users) tasks are dealt round-robin to its warps.
+__global__ void __launch_bounds__(256)
+bet_user_sums(const int64_t* __restrict__ inner, int64_t E, int64_t U, int F, BetWorkspace w) {
     const int lane = threadIdx.x & 31;
-    const int64_t u = blockIdx.x * (int64_t)(blockDim.x >> 5) + (threadIdx.x >> 5);
-    if (u >= U) return;
-    int64_t e0 = w.ev_in[u], e1 = w.ev_in[u + 1];
-    const int64_t keep = w.ev_out[u + 1] - w.ev_out[u];
-    if (e1 > E) e1 = E;                               // never read past the caller's array
-    if (e0 > e1) e0 = e1;
-    const int64_t* __restrict__ row = inner + (int64_t)f * E;
-    int64_t all = 0, kept = 0;
-    for (int64_t j = lane; j < e1 - e0; j += 32) {
-        int64_t n = __ldcs(reinterpret_cast<const long long*>(row + e0 + j));
-        if (n < 0) n = 0;
-        all += n;
-        if (j < keep) kept += n;
-    }
+    const int64_t warps = (int64_t)gridDim.x * (blockDim.x >> 5);
+    const int64_t chunks = (U + kTaskUsers - 1) / kTaskUsers;       // per feature
+    for (int64_t task = blockIdx.x * (int64_t)(blockDim.x >> 5) + (threadIdx.x >> 5); task < chunks * F;
+         task += warps) {
+        const int f = (int)(task / chunks);
+        const int64_t u0 = (task - (int64_t)f * chunks) * kTaskUsers;
+        const int64_t* __restrict__ row = inner + (int64_t)f * E;
+        const int64_t u = u0 + lane;
+        int64_t e0 = 0, e1 = 0, keep = 0;
+        if (lane < kTaskUsers && u < U) {
+            e0 = w.ev_in[u];
+            e1 = w.ev_in[u + 1];
+            keep = w.ev_out[u + 1] - w.ev_out[u];
+            if (e1 > E) e1 = E;                       // never read past the caller's array
+            if (e0 > e1) e0 = e1;
+        }
+        const int users = U - u0 < kTaskUsers ? (int)(U - u0) : kTaskUsers;
+        int64_t my_all = 0, my_kept = 0;              // results of user u0 + lane
+        // the first kSumBatch * 32 inner lengths of the NEXT user are requested before the
+        // current user's are added up, so that a warp always has a user's worth of loads in flight
+        int64_t cur[kSumBatch], nxt[kSumBatch];
+        auto first_batch = [&](int k, int64_t (&x)[kSumBatch]) {
+            const int64_t ke0 = __shfl_sync(0xffffffffu, e0, k & 31);
+            const int64_t cnt = k < users ? __shfl_sync(0xffffffffu, e1, k & 31) - ke0 : 0;
 #pragma unroll
-    for (int d = 16; d > 0; d >>= 1) {
-        all += __shfl_xor_sync(0xffffffffu, all, d);
-        kept += __shfl_xor_sync(0xffffffffu, kept, d);
-    }
-    if (lane == 0) {
-        w.v_all[(int64_t)f * U + u] = all;
-        w.v_keep[(int64_t)f * U + u] = kept;
+            for (int q = 0; q < kSumBatch; ++q) {
+                const int64_t j = lane + 32 * q;
+                x[q] = j < cnt ? __ldcs(reinterpret_cast<const long long*>(row + ke0 + j)) : 0;
+            }
+        };
+        first_batch(0, cur);
+        for (int k = 0; k < users; ++k) {
+            first_batch(k + 1, nxt);
+            const int64_t ke0 = __shfl_sync(0xffffffffu, e0, k);
+            const int64_t cnt = __shfl_sync(0xffffffffu, e1, k) - ke0;
+            const int64_t kkeep = __shfl_sync(0xffffffffu, keep, k);
+            int64_t all = 0, kept = 0;
+#pragma unroll
+            for (int q = 0; q < kSumBatch; ++q) {
+                const int64_t n = nonneg(cur[q]);
+                all += n;
+                if (lane + 32 * q < kkeep) kept += n;
+            }
+            for (int64_t j0 = lane + 32 * kSumBatch; j0 < cnt; j0 += 32 * kCopyBatch) {   // the rest, if any
+                int64_t x[kCopyBatch];
+#pragma unroll
+                for (int q = 0; q < kCopyBatch; ++q) {
+                    const int64_t j = j0 + 32 * q;
+                    x[q] = j < cnt ? __ldcs(reinterpret_cast<const long long*>(row + ke0 + j)) : 0;
+                }
+#pragma unroll
+                for (int q = 0; q < kCopyBatch; ++q) {
+                    const int64_t n = nonneg(x[q]);
+                    all += n;
+                    if (j0 + 32 * q < kkeep) kept += n;
+                }
+            }
+#pragma unroll
+            for (int d = 16; d > 0; d >>= 1) {
+                all += __shfl_xor_sync(0xffffffffu, all, d);
+                kept += __shfl_xor_sync(0xffffffffu, kept, d);
+            }
+            if (lane == k) { my_all = all; my_kept = kept; }
+#pragma unroll
+            for (int q = 0; q < kSumBatch; ++q) cur[q] = nxt[q];
+        }
+        if (lane < users) {                            // coalesced
+            w.v_all[(int64_t)f * U + u] = my_all;
+            w.v_keep[(int64_t)f * U + u] = my_kept;
+        }
     }
 }
 
 __global__ void __launch_bounds__(kScanThreads)
 bet_scan_values(int64_t U, BetWorkspace w, int64_t* __restrict__ counts_out) {
-    const int f = blockIdx.x;
-    block_exscan2(w.v_all + (int64_t)f * U, w.v_keep + (int64_t)f * U, U, w.v_in + (int64_t)f * (U + 1),
-                  w.v_out + (int64_t)f * (U + 1));
-    __syncthreads();
-    if (threadIdx.x == 0) counts_out[1 + f] = w.v_out[(int64_t)f * (U + 1) + U];
+    const int f = blockIdx.y;
+    tile_exscan2<false>(w.v_all + (int64_t)f * U, w.v_keep + (int64_t)f * U, 0, U, blockIdx.x, nullptr,
+                        w.v_in + (int64_t)f * (U + 1), w.v_out + (int64_t)f * (U + 1));
+    if ((int64_t)(blockIdx.x + 1) * kScanTile >= U) {
+        __syncthreads();
+        if (threadIdx.x == 0) counts_out[1 + f] = w.v_out[(int64_t)f * (U + 1) + U];
+    }
 }
 
-// one warp per (feature, user): copy the kept inner lengths and the kept values, both contiguous
+// Copies `n` 8-byte words src -> dst with a warp, kCopyBatch loads in flight per lane.
+template <bool CLAMP>
+__device__ __forceinline__ void warp_copy64(const int64_t* __restrict__ src, int64_t* __restrict__ dst,
+                                            int64_t n, int lane) {
+    for (int64_t j0 = lane; j0 < n; j0 += 32 * kCopyBatch) {
+        long long x[kCopyBatch];
+#pragma unroll
+        for (int k = 0; k < kCopyBatch; ++k) {
+            const int64_t j = j0 + 32 * k;
+            x[k] = j < n ? __ldcs(reinterpret_cast<const long long*>(src + j)) : 0;
+        }
+#pragma unroll
+        for (int k = 0; k < kCopyBatch; ++k) {
+            const int64_t j = j0 + 32 * k;
+            if (j < n) __stcs(reinterpret_cast<long long*>(dst + j), CLAMP && x[k] < 0 ? 0 : x[k]);
+        }
+    }
+}
+
+// A warp takes kTaskUsers consecutive users of a feature at a time: a lane each reads the ranges
+// of one of them, then the warp copies the users' kept inner lengths and kept values, both
+// contiguous per user, one user after the other.  Same task dealing as bet_user_sums.
 __global__ void __launch_bounds__(256)
 bet_copy(const int64_t* __restrict__ inner, int64_t E, const int64_t* __restrict__ values,
-         const int64_t* __restrict__ value_offsets, int64_t U, BetWorkspace w,
+         const int64_t* __restrict__ value_offsets, int64_t U, int F, BetWorkspace w,
          int64_t* __restrict__ inner_out, int64_t* __restrict__ values_out) {
-    const int f = blockIdx.y;
     const int lane = threadIdx.x & 31;
     const int64_t warps = (int64_t)gridDim.x * (blockDim.x >> 5);
-    const int64_t vbase = value_offsets[f], vend = value_offsets[f + 1];
-    for (int64_t u = blockIdx.x * (int64_t)(blockDim.x >> 5) + (threadIdx.x >> 5); u < U; u += warps) {
-        const int64_t e_in = w.ev_in[u], e_out = w.ev_out[u];
-        int64_t keep = w.ev_out[u + 1] - e_out;
-        if (e_in + keep > E) keep = E > e_in ? E - e_in : 0;
-        const int64_t v_in = vbase + w.v_in[(int64_t)f * (U + 1) + u];
-        const int64_t v_out = vbase + w.v_out[(int64_t)f * (U + 1) + u];
-        int64_t nv = w.v_keep[(int64_t)f * U + u];
-        if (v_in + nv > vend) nv = vend > v_in ? vend - v_in : 0;      // stay inside the feature's values
-        const int64_t* __restrict__ src_i = inner + (int64_t)f * E + e_in;
-        int64_t* __restrict__ dst_i = inner_out + (int64_t)f * E + e_out;
-        for (int64_t j = lane; j < keep; j += 32) {
-            const int64_t n = __ldcs(reinterpret_cast<const long long*>(src_i + j));
-            __stcs(reinterpret_cast<long long*>(dst_i + j), (long long)(n < 0 ? 0 : n));
+    const int64_t chunks = (U + kTaskUsers - 1) / kTaskUsers;       // per feature
+    for (int64_t task = blockIdx.x * (int64_t)(blockDim.x >> 5) + (threadIdx.x >> 5); task < chunks * F;
+         task += warps) {
+        const int f = (int)(task / chunks);
+        const int64_t u0 = (task - (int64_t)f * chunks) * kTaskUsers;
+        const int64_t vbase = value_offsets[f], vend = value_offsets[f + 1];
+        const int64_t* __restrict__ src_row = inner + (int64_t)f * E;
+        int64_t* __restrict__ dst_row = inner_out + (int64_t)f * E;
+        const int64_t u = u0 + lane;
+        int64_t e_in = 0, e_out = 0, keep = 0, v_in = 0, v_out = 0, nv = 0;
+        if (lane < kTaskUsers && u < U) {
+            e_in = w.ev_in[u];
+            e_out = w.ev_out[u];
+            keep = w.ev_out[u + 1] - e_out;
+            if (e_in + keep > E) keep = E > e_in ? E - e_in : 0;
+            v_in = vbase + w.v_in[(int64_t)f * (U + 1) + u];
+            v_out = vbase + w.v_out[(int64_t)f * (U + 1) + u];
+            nv = w.v_keep[(int64_t)f * U + u];
+            if (v_in + nv > vend) nv = vend > v_in ? vend - v_in : 0;   // stay inside the feature's values
         }
-        for (int64_t j = lane; j < nv; j += 32)
-            __stcs(reinterpret_cast<long long*>(values_out + v_out + j),
-                   __ldcs(reinterpret_cast<const long long*>(values + v_in + j)));
+        const int users = U - u0 < kTaskUsers ? (int)(U - u0) : kTaskUsers;
+        for (int k = 0; k < users; ++k) {
+            const int64_t ke_in = __shfl_sync(0xffffffffu, e_in, k), ke_out = __shfl_sync(0xffffffffu, e_out, k);
+            const int64_t kkeep = __shfl_sync(0xffffffffu, keep, k);
+            const int64_t kv_in = __shfl_sync(0xffffffffu, v_in, k), kv_out = __shfl_sync(0xffffffffu, v_out, k);
+            const int64_t knv = __shfl_sync(0xffffffffu, nv, k);
+            warp_copy64<true>(src_row + ke_in, dst_row + ke_out, kkeep, lane);
+            warp_copy64<false>(values + kv_in, values_out + kv_out, knv, lane);
+        }
     }
+}
+
+// One wave of resident 256-thread CTAs, or fewer when there are fewer tasks than warps.
+template <typename K>
+unsigned bet_grid(K kernel, int F, int64_t U) {
+    int dev = 0, sms = 148, per_sm = 4;
+    if (cudaGetDevice(&dev) == cudaSuccess) {
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, 256, 0) != cudaSuccess || per_sm < 1)
+            per_sm = 4;
+    }
+    cudaGetLastError();
+    const int64_t tasks = ((U + kTaskUsers - 1) / kTaskUsers) * F;
+    const int64_t need = (tasks + 7) / 8;
+    const int64_t wave = (int64_t)sms * per_sm;
+    return (unsigned)(need < wave ? (need > 0 ? need : 1) : wave);
 }
 
 }  // namespace
@@ -291,19 +436,15 @@ extern "C" ebag_status ebag_batch_event_truncate(const int64_t* outer_lengths, i
         return EBAG_ERR_INVALID_ARG;
     cudaStream_t s = (cudaStream_t)stream;
     const BetWorkspace w = carve(workspace, F, U);
-    bet_scan_outer<<<1, kScanThreads, 0, s>>>(outer_lengths, U, N, outer_out, w, counts_out);
+    const unsigned tiles = (unsigned)(U > 0 ? (U + kScanTile - 1) / kScanTile : 1);
+    bet_scan_outer<<<tiles, kScanThreads, 0, s>>>(outer_lengths, U, N, outer_out, w, counts_out);
     if (F > 0 && U > 0) {
-        const int warps = 8;
-        bet_user_sums<<<dim3((unsigned)((U + warps - 1) / warps), (unsigned)F), warps * 32, 0, s>>>(
-            inner_lengths, E, U, w);
+        bet_user_sums<<<bet_grid(bet_user_sums, F, U), 256, 0, s>>>(inner_lengths, E, U, F, w);
     }
-    if (F > 0) bet_scan_values<<<F, kScanThreads, 0, s>>>(U, w, counts_out);
+    if (F > 0) bet_scan_values<<<dim3(tiles, (unsigned)F), kScanThreads, 0, s>>>(U, w, counts_out);
     if (F > 0 && U > 0) {
-        int64_t bx = (U + 7) / 8;
-        const int64_t cap = 148 * 8 * 4 / F + 1;           // a few waves of 8-warp CTAs
-        if (bx > cap) bx = cap;
-        bet_copy<<<dim3((unsigned)bx, (unsigned)F), 256, 0, s>>>(inner_lengths, E, values, value_offsets, U, w,
-                                                                 inner_out, values_out);
+        bet_copy<<<bet_grid(bet_copy, F, U), 256, 0, s>>>(inner_lengths, E, values, value_offsets, U, F, w,
+                                                          inner_out, values_out);
     }
     if (cudaGetLastError() != cudaSuccess) return EBAG_ERR_CUDA;
     return EBAG_OK;
