@@ -43,7 +43,7 @@ typedef void* ebag_stream;        /* a cudaStream_t */
 typedef enum {
     EBAG_OK = 0,
     EBAG_ERR_INVALID_ARG = 1, /* NULL where a pointer is required, T<=0, B<0, bad D, ... */
-    EBAG_ERR_UNSUPPORTED = 2, /* mean pooling with weights; sizes beyond the stated limits */
+    EBAG_ERR_UNSUPPORTED = 2, /* sizes beyond the stated limits */
     EBAG_ERR_CUDA = 3,        /* a CUDA runtime call failed (see ebag_last_cuda_error) */
     EBAG_ERR_INDEX_OOB = 4,   /* reported by ebag_last_status: ids outside [0, rows) were skipped */
     EBAG_ERR_BAD_OFFSETS = 5  /* reported by ebag_last_status: malformed bags were treated as empty */
@@ -92,7 +92,8 @@ ebag_status ebag_create_tbe(int32_t T, const int64_t* rows, const int32_t* D, eb
  *   n_indices  length of indices (and of per_sample_weights); bags reaching past it are malformed.
  *   offsets  device int64 [T*B + 1], non-decreasing, offsets[0] == 0: bag g = t*B + b owns
  *            indices[offsets[g] .. offsets[g+1]).
- *   per_sample_weights  device fp32 [n_indices] or NULL (must be NULL for EBAG_MEAN).
+ *   per_sample_weights  device fp32 [n_indices] or NULL.  With EBAG_MEAN the weighted sum is
+ *            divided by the bag length L (the lookup count), not by the sum of the weights.
  *   B        bags per table, B >= 0, T*B < 2^31.
  *   out      device fp32 [B, sum(D)] row-major, 16-byte aligned; every element is overwritten
  *            exactly once; must not alias an input.
@@ -106,6 +107,16 @@ ebag_status ebag_forward(ebag_tbe* h, const void* const* tables, const int32_t* 
                          const int64_t* indices, int64_t n_indices, const int64_t* offsets,
                          const float* per_sample_weights, int64_t B, ebag_mode mode, float* out,
                          ebag_stream stream);
+
+/*
+ * ebag_forward for 32-bit ids: `indices` is device int32 [n_indices] (4-byte aligned); everything
+ * else, the offsets included, is as in ebag_forward.  The paper's problem statement allows ids of
+ * either width (Sec. 2.2); negative ids are rejected like any id outside the table.
+ */
+ebag_status ebag_forward_i32(ebag_tbe* h, const void* const* tables, const int32_t* D,
+                             const int32_t* indices, int64_t n_indices, const int64_t* offsets,
+                             const float* per_sample_weights, int64_t B, ebag_mode mode, float* out,
+                             ebag_stream stream);
 
 /*
  * The same forward for callers whose per-step data lives in HOST memory: indices, offsets,

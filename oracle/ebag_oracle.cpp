@@ -14,7 +14,8 @@
 //   for every table t and bag b (bag id g = t*B + b):
 //       s = offsets[g], e = offsets[g+1], L = e - s
 //       out[b, Doff[t] + d] = pool_{i = s .. e-1} w_i * value(t, indices[i], d)
-//   pool = sum, or sum / L (mean; an empty bag stays +0.0f), w_i = weights[i] or 1.
+//   pool = sum, or sum / L (mean; an empty bag stays +0.0f), w_i = weights[i] or 1.  With weights
+//   the mean still divides by the lookup count L (not by the sum of the weights).
 //   value() widens the stored element to fp32: fp32 as is, fp16/bf16 exactly, rowwise int8 as
 //   scale[row] * (float)q + bias[row] (one fp32 multiply, then one fp32 add).
 //
@@ -100,7 +101,6 @@ int ebag_oracle_forward(int32_t T, const int64_t* rows, const int32_t* D, int32_
     if (T <= 0 || B < 0 || !rows || !D || !tables || !offsets || !out32) return 1;
     if (dtype < DT_F32 || dtype > DT_INT8_ROWWISE) return 1;
     if (mode != MODE_SUM && mode != MODE_MEAN) return 1;
-    if (mode == MODE_MEAN && weights) return 1;
     if (dtype == DT_INT8_ROWWISE && (!scales || !biases)) return 1;
     std::vector<int64_t> Doff(T + 1, 0);
     for (int32_t t = 0; t < T; ++t) {

@@ -28,6 +28,7 @@ SIGNATURES = {
     "ebag_row_stride": (_i64, [_int, _i32]),
     "ebag_create_tbe": (_int, [_i32, _vp, _vp, _int, _int, _vp]),
     "ebag_forward": (_int, [_vp, _vp, _vp, _vp, _i64, _vp, _vp, _i64, _int, _vp, _vp]),
+    "ebag_forward_i32": (_int, [_vp, _vp, _vp, _vp, _i64, _vp, _vp, _i64, _int, _vp, _vp]),
     "ebag_forward_host": (_int, [_vp, _vp, _vp, _vp, _i64, _vp, _vp, _i64, _int, _vp, _vp]),
     "ebag_forward_noalloc": (_int, [_i32, _vp, _vp, _int, _vp, _vp, _i64, _vp, _vp, _i64, _int, _vp,
                                     _vp, _vp]),
@@ -280,17 +281,23 @@ class TBE:
 
     def forward(self, tables: List, indices, offsets, B: int, mode: int = EBAG_SUM,
                 per_sample_weights=None, out=None, stream=None):
-        """Device tensors in, device tensor out ([B, sum D] float32).  Enqueues only."""
+        """Device tensors in, device tensor out ([B, sum D] float32).  Enqueues only.
+        ``indices`` may be int64 or int32 (the matching entry point is called)."""
         import torch
         if out is None:
             out = torch.empty((B, self.sumD), dtype=torch.float32, device=indices.device)
         if not hasattr(self, "_d_arr"):
             self._d_arr = (ctypes.c_int32 * self.T)(*self.D)
             self._d_ptr = ctypes.cast(self._d_arr, _vp)
-        st = lib().ebag_forward(self._h, self._table_array(tables), self._d_ptr, _ptr(indices),
-                                int(indices.numel()), _ptr(offsets), _ptr(per_sample_weights), B, mode,
-                                _ptr(out), _stream_ptr(stream))
-        _check(st, "ebag_forward")
+        if indices.dtype == torch.int32:
+            fn, name = lib().ebag_forward_i32, "ebag_forward_i32"
+        elif indices.dtype == torch.int64:
+            fn, name = lib().ebag_forward, "ebag_forward"
+        else:
+            raise TypeError("indices must be int64 or int32")
+        st = fn(self._h, self._table_array(tables), self._d_ptr, _ptr(indices), int(indices.numel()),
+                _ptr(offsets), _ptr(per_sample_weights), B, mode, _ptr(out), _stream_ptr(stream))
+        _check(st, name)
         return out
 
     def forward_mapid(self, tables: List, values, offsets, mappings: List, B: int,

@@ -153,7 +153,6 @@ ebag_status check_forward_args(ebag_tbe* h, const void* const* tables, const int
                                const float* weights, int64_t B, ebag_mode mode, float* out) {
     if (!h || !tables || !D || !offsets || B < 0 || n_indices < 0) return EBAG_ERR_INVALID_ARG;
     if (mode != EBAG_SUM && mode != EBAG_MEAN) return EBAG_ERR_INVALID_ARG;
-    if (mode == EBAG_MEAN && weights) return EBAG_ERR_UNSUPPORTED;
     if (n_indices > 0 && !indices) return EBAG_ERR_INVALID_ARG;
     if (B > 0 && !out) return EBAG_ERR_INVALID_ARG;
     if ((int64_t)h->T * B >= (1ll << 31)) return EBAG_ERR_UNSUPPORTED;
@@ -201,9 +200,9 @@ ebag_status forward_device(ebag_tbe* h, const void* const* tables, const int64_t
                            int64_t n_indices, const int64_t* offsets, const float* weights,
                            int64_t B, int64_t b0, int64_t b1, ebag_mode mode, float* out,
                            cudaStream_t stream, const int64_t* const* mappings = nullptr,
-                           const int64_t* mapping_len = nullptr) {
+                           const int64_t* mapping_len = nullptr, bool idx32 = false) {
     if (b1 <= b0) return EBAG_OK;
-    if (((uintptr_t)out & 15u) || ((uintptr_t)indices & 7u) || ((uintptr_t)offsets & 7u) ||
+    if (((uintptr_t)out & 15u) || ((uintptr_t)indices & (idx32 ? 3u : 7u)) || ((uintptr_t)offsets & 7u) ||
         ((uintptr_t)weights & 3u))
         return EBAG_ERR_INVALID_ARG;
     const void* const* d_tables = nullptr;
@@ -227,6 +226,7 @@ ebag_status forward_device(ebag_tbe* h, const void* const* tables, const int64_t
     p.T = h->T;
     p.sumD = h->sumD;
     p.mean = mode == EBAG_MEAN ? 1 : 0;
+    p.idx32 = idx32 ? 1 : 0;
     p.item_bytes = h->item_bytes;
     // Long bags.  The bytes this call can gather are at most n_indices * (widest row), so at most
     // that / long_bytes bags can reach long_bytes; with long_bytes = 4 * part_bytes (a power of two) and
@@ -536,6 +536,20 @@ ebag_status ebag_forward(ebag_tbe* h, const void* const* tables, const int32_t* 
     if (!guard.ok) return EBAG_ERR_CUDA;
     return forward_device(h, tables, indices, n_indices, offsets, per_sample_weights, B, 0, B, mode,
                           out, (cudaStream_t)stream);
+}
+
+ebag_status ebag_forward_i32(ebag_tbe* h, const void* const* tables, const int32_t* D,
+                             const int32_t* indices, int64_t n_indices, const int64_t* offsets,
+                             const float* per_sample_weights, int64_t B, ebag_mode mode, float* out,
+                             ebag_stream stream) {
+    const int64_t* ids = reinterpret_cast<const int64_t*>(indices);   // width travels in idx32
+    ebag_status st = check_forward_args(h, tables, D, ids, n_indices, offsets, per_sample_weights, B,
+                                        mode, out);
+    if (st != EBAG_OK) return st;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) return EBAG_ERR_CUDA;
+    return forward_device(h, tables, ids, n_indices, offsets, per_sample_weights, B, 0, B, mode, out,
+                          (cudaStream_t)stream, nullptr, nullptr, true);
 }
 
 ebag_status ebag_forward_host(ebag_tbe* h, const void* const* tables, const int32_t* D,

@@ -108,7 +108,7 @@ struct PartArgs {                        // one part of a long bag (parts kernel
 struct FwdParams {
     const void* const* tables;   // device [T]
     const TableMeta* meta;       // device [T]
-    const int64_t* indices;
+    const int64_t* indices;      // int32 ids instead when idx32 is set
     const int64_t* offsets;
     const float* weights;
     float* out;
@@ -123,6 +123,7 @@ struct FwdParams {
     int32_t T;
     int32_t sumD;
     int32_t mean;                // 1: divide by the bag length
+    int32_t idx32;               // 1: `indices` holds 32-bit ids
     uint32_t item_bytes;
     LongParams lg;
 };
@@ -441,7 +442,9 @@ __device__ __forceinline__ void process_item(const FwdParams& p, const TableMeta
     // at my_rows_s + (st * kStageVecs + k) * 512 (kept opaque: not to be recomputed at every use)
     uint32_t my_rows_s = (uint32_t)__cvta_generic_to_shared(wbuf) + lane * 16;
     asm volatile("" : "+r"(my_rows_s));
-    const int64_t* __restrict__ idx_base = p.indices + base;
+    // first id of the item (ids are 8 bytes wide, or 4 when p.idx32)
+    const char* __restrict__ idx_base =
+        reinterpret_cast<const char*>(p.indices) + base * (p.idx32 ? 4 : 8);
     const float* __restrict__ w_base = WEIGHTED ? p.weights + base : nullptr;
 
     bool col_on[V];
@@ -466,7 +469,9 @@ __device__ __forceinline__ void process_item(const FwdParams& p, const TableMeta
         w = 0.0f;
         const uint32_t i = pos + lig;
         if (i < end) {
-            int64_t r = ld_stream_i64(idx_base + i);
+            int64_t r;
+            if (p.idx32) r = __ldcs(reinterpret_cast<const int*>(idx_base) + i);
+            else r = ld_stream_i64(reinterpret_cast<const int64_t*>(idx_base) + i);
             float wl = 1.0f;
             if (WEIGHTED) wl = ld_stream_f32(w_base + i);
             if (MAPID) r = map_id(map_ptr, map_len, map_steps, r);     // raw id -> row

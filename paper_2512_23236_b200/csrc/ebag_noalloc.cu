@@ -137,7 +137,6 @@ extern "C" ebag_status ebag_forward_noalloc(int32_t T, const int64_t* rows, cons
         return EBAG_ERR_INVALID_ARG;
     if (dtype < EBAG_F32 || dtype > EBAG_INT8_ROWWISE) return EBAG_ERR_INVALID_ARG;
     if (mode != EBAG_SUM && mode != EBAG_MEAN) return EBAG_ERR_INVALID_ARG;
-    if (mode == EBAG_MEAN && per_sample_weights) return EBAG_ERR_UNSUPPORTED;
     if (T > kMaxTables) return EBAG_ERR_UNSUPPORTED;       // beyond the static scratch
     if ((int64_t)T * B >= (1ll << 31)) return EBAG_ERR_UNSUPPORTED;
     if (n_indices > 0 && !indices) return EBAG_ERR_INVALID_ARG;
@@ -201,6 +200,7 @@ extern "C" ebag_status ebag_forward_noalloc(int32_t T, const int64_t* rows, cons
     p.T = T;
     p.sumD = (int32_t)d_off;
     p.mean = mode == EBAG_MEAN ? 1 : 0;
+    p.idx32 = 0;
     p.item_bytes = 32768;
     p.lg = LongParams{};                     // no room for partial sums here: bags are not split
     const bool w = per_sample_weights != nullptr;

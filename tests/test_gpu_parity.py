@@ -108,7 +108,8 @@ def test_host_buffer_entry_point_with_malformed_offsets_falls_back():
     (wl.BF16, [8, 16, 72, 256, 512, 1032, 2056]),
     (wl.INT8_ROWWISE, [16, 48, 128, 512, 528, 1040, 2064]),
 ])
-@pytest.mark.parametrize("mode,weighted", [(wl.SUM, False), (wl.MEAN, False), (wl.SUM, True)])
+@pytest.mark.parametrize("mode,weighted", [(wl.SUM, False), (wl.MEAN, False), (wl.SUM, True),
+                                           (wl.MEAN, True)])
 def test_all_row_widths(dtype, Ds, mode, weighted):
     rng = np.random.default_rng(42 + dtype)
     T, B = len(Ds), 77                      # ragged tail: 77 is not a multiple of any item size
@@ -122,6 +123,31 @@ def test_all_row_widths(dtype, Ds, mode, weighted):
     gpu, status, ref = _both(dtype, rows, Ds, tabs, idx, off, B, mode, w)
     assert status == (0, 0, 0)
     pu.compare(gpu, ref, dtype, lengths, T, B, Ds)
+
+
+# ------------------------------------------------------------------ 32-bit ids
+@pytest.mark.parametrize("dtype,Ds", [(wl.F32, [8, 64, 260]), (wl.BF16, [16, 128, 1032]),
+                                      (wl.INT8_ROWWISE, [16, 128, 528])])
+@pytest.mark.parametrize("mode,weighted", [(wl.SUM, False), (wl.MEAN, True)])
+def test_int32_ids(dtype, Ds, mode, weighted):
+    """ebag_forward_i32: parity with the oracle, the same bits as the 64-bit entry point on the
+    same ids, and ids outside the table (negative ones too) skipped and counted."""
+    rng = np.random.default_rng(77 + dtype)
+    T, B = len(Ds), 130
+    rows = [int(rng.integers(20, 500)) for _ in Ds]
+    lens = [rng.integers(0, 50, size=B) for _ in Ds]
+    idx, off, lengths = _jagged_from_lengths(rng, lens, rows)
+    bad = rng.choice(idx.shape[0], size=25, replace=False)
+    idx[bad[:10]] = -1 - rng.integers(0, 1000, size=10)
+    idx[bad[10:]] = 2**31 - 1 - rng.integers(0, 1000, size=15)
+    w = (rng.random(idx.shape[0]).astype(np.float32) - 0.25) if weighted else None
+    tabs = _rand_tables(rng, dtype, rows, Ds)
+    gpu64, st64, ref = _both(dtype, rows, Ds, tabs, idx, off, B, mode, w)
+    gpu32, st32, _ = _both(dtype, rows, Ds, tabs, idx.astype(np.int32), off, B, mode, w)
+    assert ref["n_oob"] == 25
+    assert st32 == st64 == (eb.EBAG_ERR_INDEX_OOB, 25, 0)
+    pu.compare(gpu32, ref, dtype)
+    assert np.array_equal(gpu32.view(np.uint32), gpu64.view(np.uint32))
 
 
 # ------------------------------------------------------------------ degenerate and extreme bags
@@ -237,10 +263,6 @@ def test_host_side_argument_errors():
     tab = torch.zeros(10, 16, device="cuda")
     idx = torch.zeros(4, dtype=torch.int64, device="cuda")
     off = torch.tensor([0, 4], dtype=torch.int64, device="cuda")
-    w = torch.ones(4, device="cuda")
-    with pytest.raises(eb.EbagError) as e:
-        tbe.forward([tab], idx, off, 1, eb.EBAG_MEAN, w)
-    assert e.value.status == eb.EBAG_ERR_UNSUPPORTED
     with pytest.raises(eb.EbagError) as e:
         eb.ebag_forward(tbe._h, [tab.data_ptr()], [32], idx.data_ptr(), 4, off.data_ptr(), None, 1, 0,
                         tab.data_ptr(), 0)

@@ -330,10 +330,32 @@ def test_bad_offsets_make_empty_bags_and_are_counted():
     assert r["n_bad_offsets"] == 1 and np.all(r["out32"][1] == 0)
 
 
-def test_rejects_mean_with_weights_and_bad_shapes():
+def test_weighted_mean_divides_the_weighted_sum_by_the_lookup_count():
+    """mean with per-sample weights = (sum of w*x) / L, L the number of lookups of the bag (the
+    divisor is not the sum of the weights).  Pinned against the weighted sum, which has its own
+    pins above, and against a brute-force evaluation in fp64."""
+    rng = np.random.default_rng(21)
+    rows, D, B = 50, 8, 40
+    tab = rng.standard_normal((rows, D)).astype(np.float32)
+    lengths = rng.integers(0, 9, size=B)
+    off = np.zeros(B + 1, np.int64)
+    np.cumsum(lengths, out=off[1:])
+    idx = rng.integers(0, rows, size=int(off[-1])).astype(np.int64)
+    w = rng.uniform(-2, 2, size=idx.size).astype(np.float32)
+    s = orc.forward([tab], orc.F32, idx, off, B, orc.SUM, weights=w)
+    m = orc.forward([tab], orc.F32, idx, off, B, orc.MEAN, weights=w)
+    for b in range(B):
+        L = lengths[b]
+        if L == 0:
+            assert np.all(m["out32"][b].view(np.uint32) == 0)
+            continue
+        assert np.array_equal(m["out32"][b], s["out32"][b] / np.float32(L))
+        brute = sum(np.float64(w[i]) * tab[idx[i]].astype(np.float64) for i in range(off[b], off[b + 1])) / L
+        assert np.allclose(m["out64"][b], brute, rtol=1e-12, atol=1e-12)
+        assert np.allclose(m["S"][b], s["S"][b] / L, rtol=1e-12)
+
+
+def test_rejects_bad_shapes():
     tab = np.zeros((4, 4), np.float32)
-    with pytest.raises(ValueError):
-        orc.forward([tab], orc.F32, np.zeros(1, np.int64), np.array([0, 1]), 1, orc.MEAN,
-                    weights=np.ones(1, np.float32))
     with pytest.raises(ValueError):
         orc.forward([tab], orc.F32, np.zeros(1, np.int64), np.array([0, 1, 1]), 1, orc.SUM)
