@@ -119,6 +119,27 @@ ebag_status ebag_forward_i32(ebag_tbe* h, const void* const* tables, const int32
                              ebag_stream stream);
 
 /*
+ * Backward of the pooled forward with respect to the tables (the training half; the operator is
+ * linear in the tables, so this is its transpose):
+ *     grad_tables[t][indices[i], d] += w_i * grad_out[b, Doff[t] + d]      (EBAG_MEAN: / L)
+ * for every lookup i of every bag (t, b).
+ *   grad_out     device fp32 [B, sum(D)], 16-byte aligned: gradient of the loss with respect to `out`.
+ *   indices      device int64 or int32 ids (index_bits = 64 or 32), as given to the forward.
+ *   offsets, per_sample_weights, B, mode   as given to the forward.
+ *   grad_tables  host array [T] of DEVICE pointers to dense fp32 [rows[t], D[t]] arrays (whatever
+ *                the storage type of the tables), 16-byte aligned, owned and zeroed by the caller:
+ *                the call ADDS into them.  Needs D[t] % 4 == 0 (else UNSUPPORTED).
+ * One kernel launch on `stream`, no allocation after the first call (which builds a few KB of
+ * metadata), no synchronisation.  Contributions are added with floating-point reductions in
+ * memory whose order is not fixed: two runs agree up to fp32 rounding, not bit for bit.  Ids
+ * outside the table and malformed bags are skipped and counted as in the forward
+ * (ebag_last_status).  The gradient with respect to per_sample_weights is not computed.
+ */
+ebag_status ebag_backward(ebag_tbe* h, const float* grad_out, const void* indices, int32_t index_bits,
+                          int64_t n_indices, const int64_t* offsets, const float* per_sample_weights,
+                          int64_t B, ebag_mode mode, float* const* grad_tables, ebag_stream stream);
+
+/*
  * The same forward for callers whose per-step data lives in HOST memory: indices, offsets,
  * per_sample_weights and out are host pointers (pinned memory makes the copies asynchronous);
  * tables stay device pointers (they are model state, loaded once).  The call copies the inputs

@@ -29,6 +29,7 @@ SIGNATURES = {
     "ebag_create_tbe": (_int, [_i32, _vp, _vp, _int, _int, _vp]),
     "ebag_forward": (_int, [_vp, _vp, _vp, _vp, _i64, _vp, _vp, _i64, _int, _vp, _vp]),
     "ebag_forward_i32": (_int, [_vp, _vp, _vp, _vp, _i64, _vp, _vp, _i64, _int, _vp, _vp]),
+    "ebag_backward": (_int, [_vp, _vp, _vp, _i32, _i64, _vp, _vp, _i64, _int, _vp, _vp]),
     "ebag_forward_host": (_int, [_vp, _vp, _vp, _vp, _i64, _vp, _vp, _i64, _int, _vp, _vp]),
     "ebag_forward_noalloc": (_int, [_i32, _vp, _vp, _int, _vp, _vp, _i64, _vp, _vp, _i64, _int, _vp,
                                     _vp, _vp]),
@@ -299,6 +300,23 @@ class TBE:
                 _ptr(offsets), _ptr(per_sample_weights), B, mode, _ptr(out), _stream_ptr(stream))
         _check(st, name)
         return out
+
+    def backward(self, grad_out, indices, offsets, B: int, grad_tables: List, mode: int = EBAG_SUM,
+                 per_sample_weights=None, stream=None):
+        """Adds the gradient of the forward with respect to the tables into ``grad_tables`` (a
+        list of T dense float32 CUDA tensors [rows_t, D_t]).  Enqueues only."""
+        import torch
+        bits = 32 if indices.dtype == torch.int32 else 64
+        if indices.dtype not in (torch.int32, torch.int64):
+            raise TypeError("indices must be int64 or int32")
+        for g in grad_tables:
+            if g.dtype != torch.float32 or not g.is_contiguous():
+                raise TypeError("gradient tables must be contiguous float32")
+        arr = (ctypes.c_void_p * self.T)(*[g.data_ptr() if g.numel() else None for g in grad_tables])
+        st = lib().ebag_backward(self._h, _ptr(grad_out), _ptr(indices), bits, int(indices.numel()),
+                                 _ptr(offsets), _ptr(per_sample_weights), B, mode,
+                                 ctypes.cast(arr, _vp), _stream_ptr(stream))
+        _check(st, "ebag_backward")
 
     def forward_mapid(self, tables: List, values, offsets, mappings: List, B: int,
                       mode: int = EBAG_SUM, per_sample_weights=None, out=None, stream=None):

@@ -9,6 +9,7 @@
 #include <vector>
 
 #include "ebag.h"
+#include "ebag_bwd.cuh"
 #include "ebag_fwd.cuh"
 
 using namespace ebag;
@@ -44,6 +45,8 @@ struct ebag_tbe {
     std::vector<int64_t> rows;
     std::vector<int32_t> D;
     TableMeta* d_meta = nullptr;
+    BwdTableMeta* d_bwd_meta = nullptr;            // built by the first ebag_backward
+    int bwd_occupancy[2] = {};
     Queue* d_queue = nullptr;
     Status* d_status = nullptr;
     // per-call pointer block [tables T][mappings T][mapping lengths T]: cached on the device,
@@ -94,6 +97,7 @@ ebag_status cuda_fail(ebag_tbe* h, cudaError_t e) {
 void free_handle(ebag_tbe* h) {
     if (!h) return;
     cudaFree(h->d_meta);
+    cudaFree(h->d_bwd_meta);
     cudaFree(h->d_queue);
     cudaFree(h->d_status);
     cudaFree(h->d_long);
@@ -550,6 +554,74 @@ ebag_status ebag_forward_i32(ebag_tbe* h, const void* const* tables, const int32
     if (!guard.ok) return EBAG_ERR_CUDA;
     return forward_device(h, tables, ids, n_indices, offsets, per_sample_weights, B, 0, B, mode, out,
                           (cudaStream_t)stream, nullptr, nullptr, true);
+}
+
+ebag_status ebag_backward(ebag_tbe* h, const float* grad_out, const void* indices, int32_t index_bits,
+                          int64_t n_indices, const int64_t* offsets, const float* per_sample_weights,
+                          int64_t B, ebag_mode mode, float* const* grad_tables, ebag_stream stream) {
+    if (!h || !offsets || !grad_tables || B < 0 || n_indices < 0) return EBAG_ERR_INVALID_ARG;
+    if (index_bits != 32 && index_bits != 64) return EBAG_ERR_INVALID_ARG;
+    if (mode != EBAG_SUM && mode != EBAG_MEAN) return EBAG_ERR_INVALID_ARG;
+    if (n_indices > 0 && !indices) return EBAG_ERR_INVALID_ARG;
+    if (B > 0 && !grad_out) return EBAG_ERR_INVALID_ARG;
+    if ((int64_t)h->T * B >= (1ll << 31)) return EBAG_ERR_UNSUPPORTED;
+    if (((uintptr_t)grad_out & 15u) || ((uintptr_t)indices & (index_bits == 32 ? 3u : 7u)) ||
+        ((uintptr_t)offsets & 7u) || ((uintptr_t)per_sample_weights & 3u))
+        return EBAG_ERR_INVALID_ARG;
+    for (int t = 0; t < h->T; ++t) {
+        if (h->D[t] % 4 != 0) return EBAG_ERR_UNSUPPORTED;          // fp32 gradient rows in 16-byte vectors
+        if (!grad_tables[t] && h->rows[t] > 0) return EBAG_ERR_INVALID_ARG;
+        if ((uintptr_t)grad_tables[t] & 15u) return EBAG_ERR_INVALID_ARG;
+    }
+    if (B == 0 || n_indices == 0) return EBAG_OK;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) return EBAG_ERR_CUDA;
+    cudaStream_t s = (cudaStream_t)stream;
+    if (!h->d_bwd_meta) {                       // first call: per-table metadata and launch geometry
+        std::vector<BwdTableMeta> meta(h->T);
+        int32_t d_off = 0;
+        for (int t = 0; t < h->T; ++t) {
+            BwdTableMeta& m = meta[t];
+            m.rows = h->rows[t];
+            m.D = h->D[t];
+            m.D_off = d_off;
+            m.nvec = h->D[t] / 4;
+            int g = 0;
+            while ((1 << g) < m.nvec && g < 5) ++g;
+            m.g_log2 = g;
+            d_off += h->D[t];
+        }
+        EBAG_CUDA(h, cudaMalloc((void**)&h->d_bwd_meta, sizeof(BwdTableMeta) * h->T));
+        EBAG_CUDA(h, cudaMemcpy(h->d_bwd_meta, meta.data(), sizeof(BwdTableMeta) * h->T,
+                                cudaMemcpyHostToDevice));
+        for (int w = 0; w < 2; ++w) {
+            EBAG_CUDA(h, occupancy_bwd(w != 0, h->T, &h->bwd_occupancy[w]));
+            if (h->bwd_occupancy[w] < 1) h->bwd_occupancy[w] = 1;
+        }
+    }
+    const void* const* d_ptrs = nullptr;
+    ebag_status st = stage_tables(h, reinterpret_cast<const void* const*>(grad_tables), nullptr, nullptr,
+                                  s, &d_ptrs);
+    if (st != EBAG_OK) return st;
+    BwdParams p;
+    p.grad_tables = reinterpret_cast<float* const*>(const_cast<void* const*>(d_ptrs));
+    p.meta = h->d_bwd_meta;
+    p.indices = indices;
+    p.offsets = offsets;
+    p.weights = per_sample_weights;
+    p.grad_out = grad_out;
+    p.status = h->d_status;
+    p.n_indices = n_indices;
+    p.B = B;
+    p.T = h->T;
+    p.sumD = h->sumD;
+    p.mean = mode == EBAG_MEAN ? 1 : 0;
+    p.idx32 = index_bits == 32 ? 1 : 0;
+    const bool w = per_sample_weights != nullptr;
+    const int grid = h->num_sms * h->bwd_occupancy[w ? 1 : 0];
+    EBAG_CUDA(h, launch_bwd(p, w, grid, s));
+    ++h->launches;
+    return EBAG_OK;
 }
 
 ebag_status ebag_forward_host(ebag_tbe* h, const void* const* tables, const int32_t* D,

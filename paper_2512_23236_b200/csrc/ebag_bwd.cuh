@@ -1,0 +1,38 @@
+// Parameters of the backward kernel (see ebag_bwd.cu).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "ebag_fwd.cuh"     // Status
+
+namespace ebag {
+
+struct BwdTableMeta {        // per table; gradient tables are dense fp32 [rows, D]
+    int64_t rows;
+    int32_t D;
+    int32_t D_off;           // first column of this table in grad_out
+    int32_t nvec;            // 16-byte vectors per gradient row (D / 4)
+    int32_t g_log2;          // log2 of the lanes that cover a row (or one column tile of it)
+};
+
+struct BwdParams {
+    float* const* grad_tables;   // device [T]
+    const BwdTableMeta* meta;    // device [T]
+    const void* indices;         // int64 ids, or int32 when idx32
+    const int64_t* offsets;
+    const float* weights;
+    const float* grad_out;       // [B, sumD]
+    Status* status;
+    int64_t n_indices;
+    int64_t B;
+    int32_t T;
+    int32_t sumD;
+    int32_t mean;
+    int32_t idx32;
+};
+
+cudaError_t launch_bwd(const BwdParams& p, bool weighted, int grid, cudaStream_t s);
+cudaError_t occupancy_bwd(bool weighted, int T, int* ctas_per_sm);
+
+}  // namespace ebag
