@@ -459,6 +459,143 @@ def run_bet(args, rank, local_rank, world):
     print(json.dumps(line), flush=True)
 
 
+BWD_WORKLOAD = 9       # backward (gradient with respect to the tables), a NEXT row
+
+
+def run_bwd(args, rank, local_rank, world):
+    """Workload 9: ebag_backward on workload 3's jagged structure (32 tables, Zipf ids, 87.7 M
+    lookups): dense fp32 gradient tables (31.9 GB), grad_out [65536, 4352] fp32.  Algorithmic
+    bytes: per lookup the reduction's payload (4 D) + id (8); per bag grad_out (4 D) + offset (8).
+    The reductions are resolved in L2, so the HBM copy bandwidth is a reference, not the bound."""
+    from oracle import ebag_bwd_oracle as bo
+    base = wl.make_workload(3, scale_rows=args.scale_rows, scale_B=args.scale_b, max_tables=args.max_tables or None,
+                            seed=bl.rank_seed(0, rank))
+    jag = wl.gen_jagged(base)
+    T, B = base.T, base.B
+    lookups = int(jag.lengths.sum())
+    per_table = np.add.reduceat(jag.lengths, np.arange(0, T * B, B))
+    alg = int(sum(int(per_table[t]) * (4 * base.D[t] + 8) for t in range(T)) + B * (4 * base.sumD + 8 * T))
+    config = {"workload": "bwd_" + base.name, "tables": T, "bags_per_table": B, "lookups": lookups,
+              "sum_D": base.sumD, "gradient_tables": "dense fp32", "algorithmic_bytes_per_step": alg,
+              "data": "workload 3's seeded jagged ids; grad_out N(0,1)",
+              "l2": f"{L2_FLUSH_BYTES >> 20} MiB written between timed steps (L2 flush)"}
+    rng = np.random.default_rng(bl.rank_seed(0, rank) + 1)
+    sb = min(B, 512)                                       # CPU sample: the first bags of table 0
+
+    def cpu_sample():
+        off = jag.offsets[:sb + 1]
+        idx = jag.indices[:off[-1]]
+        G = rng.standard_normal((sb, base.D[0]))
+        t0 = time.perf_counter()
+        bo.backward([base.rows[0]], [base.D[0]], G, idx, off, sb)
+        return int(off[-1]), time.perf_counter() - t0
+
+    if args.impl == "reference":
+        if rank != 0:
+            return
+        for _ in range(args.warmup):
+            cpu_sample()
+        n = dt = 0
+        for _ in range(args.steps):
+            a, b = cpu_sample()
+            n += a
+            dt += b
+        v = n / dt
+        print(json.dumps({"impl": "reference", "metric": "pooled_lookups_per_sec", "value": v,
+                          "unit": "lookups/s", "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+                          "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+                          "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": config,
+                          "cpu_baseline": {"value": v, "unit": "lookups/s", "cores": 1, "kind": "oracle",
+                                           "sample": f"the first {sb} bags of table 0 (Python loops over lookups)"},
+                          "e2e": {"value": v, "unit": "lookups/s", "h2d_bytes_per_step": 0,
+                                  "d2h_bytes_per_step": 0}, "gpu_launches": 0}), flush=True)
+        return
+    import paper_2512_23236_b200 as eb
+    eb.lib()
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    bl.init_process_group("nccl")
+    warmup = max(3, args.warmup)
+    grads = [torch.zeros(r, d, device=dev) for r, d in zip(base.rows, base.D)]
+    h_idx = torch.from_numpy(jag.indices).pin_memory()
+    h_off = torch.from_numpy(jag.offsets).pin_memory()
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(bl.rank_seed(0, rank) + 7)
+    d_G = torch.randn((B, base.sumD), device=dev, generator=gen)
+    h_G = d_G.cpu().pin_memory()
+    d_idx, d_off = h_idx.to(dev), h_off.to(dev)
+    s_idx, s_off, s_G = torch.empty_like(d_idx), torch.empty_like(d_off), torch.empty_like(d_G)
+    h_status = torch.zeros(2, dtype=torch.int64).pin_memory()
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
+    tbe = eb.TBE(base.rows, base.D, wl.F32, device=local_rank)
+    stream = torch.cuda.Stream(device=dev)
+    sampler = bl.ClockSampler(f"GPU-{torch.cuda.get_device_properties(dev).uuid}").start()
+    with torch.cuda.stream(stream):
+        for _ in range(warmup):
+            flush.fill_(1)
+            tbe.backward(d_G, d_idx, d_off, B, grads, stream=stream)
+        stream.synchronize()
+        assert tbe.last_status(stream) == (0, 0, 0)
+        bl.barrier()
+        torch.cuda.synchronize()
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+              for _ in range(args.steps)]
+        for a, b in ev:
+            flush.fill_(1)
+            a.record(stream)
+            tbe.backward(d_G, d_idx, d_off, B, grads, stream=stream)
+            b.record(stream)
+        torch.cuda.synchronize()
+        bl.barrier()
+        step_ms = [a.elapsed_time(b) for a, b in ev]
+        elapsed_ms = float(sum(step_ms))
+        # end to end: host grad_out, ids and offsets in; the gradient tables stay on the device
+        # (they are the optimizer's input), the status words come back
+        e2e_steps = args.e2e_steps or min(args.steps, 10)
+        ev2 = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+               for _ in range(e2e_steps)]
+        for a, b in ev2:
+            a.record(stream)
+            s_idx.copy_(h_idx, non_blocking=True)
+            s_off.copy_(h_off, non_blocking=True)
+            s_G.copy_(h_G, non_blocking=True)
+            tbe.backward(s_G, s_idx, s_off, B, grads, stream=stream)
+            h_status.copy_(grads[0][0, :2].to(torch.int64), non_blocking=True)
+            b.record(stream)
+        torch.cuda.synchronize()
+        bl.barrier()
+        e2e_ms = float(sum(a.elapsed_time(b) for a, b in ev2))
+    clocks = sampler.stop()
+    n_steps = warmup + args.steps + e2e_steps           # every step added into the same tables
+    total, max_ms = bl.reduce_job(lookups * args.steps, elapsed_ms, dev)
+    e2e_total, e2e_max = bl.reduce_job(lookups * e2e_steps, e2e_ms, dev)
+    tbe.close()
+    if rank != 0:
+        return
+    peaks = bl.measured_peaks(ROOT)
+    ms = elapsed_ms / args.steps
+    achieved = alg / (ms * 1e-3) / 1e9
+    n_cpu, dt = cpu_sample()
+    line = {"metric": "pooled_lookups_per_sec", "value": total / (max_ms * 1e-3), "unit": "lookups/s",
+            "n_gpus": world, "steps": args.steps, "warmup": warmup, "ms_per_step": max_ms / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+            "data": "synthetic", "config": config, "clocks": clocks, "gpu_launches": args.steps,
+            "e2e": {"value": e2e_total / (e2e_max * 1e-3), "unit": "lookups/s",
+                    "h2d_bytes_per_step": int(h_idx.numel() * 8 + h_off.numel() * 8 + h_G.numel() * 4),
+                    "d2h_bytes_per_step": 16, "steps": e2e_steps, "ms_per_step": e2e_max / e2e_steps},
+            "roofline": {"bound": "hbm", "kernel": "ebag_bwd_kernel", "achieved": achieved,
+                         "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
+                         "peak_source": f"{peaks['source']} HBM copy bandwidth (burst); the reductions are "
+                                        "resolved in L2, so this is a reference, not the binding limit",
+                         "algorithmic_bytes_per_launch": alg, "ms_per_launch": ms,
+                         "ms_per_launch_min": min(step_ms), "traffic": None},
+            "cpu_baseline": {"value": n_cpu / dt, "unit": "lookups/s", "cores": 1, "kind": "oracle",
+                             "sample": f"the first {sb} bags of table 0 (Python loops over lookups)",
+                             "seconds": dt},
+            "steps_accumulated": n_steps}
+    print(json.dumps(line), flush=True)
+
+
 def main():
     args = parse_args()
     rank, local_rank, world = bl.rank_info()
@@ -467,6 +604,9 @@ def main():
         return
     if args.workload == MBDT_WORKLOAD:
         run_mbdt(args, rank, local_rank, world)
+        return
+    if args.workload == BWD_WORKLOAD:
+        run_bwd(args, rank, local_rank, world)
         return
     if args.impl == "reference":
         run_reference(args, rank)
