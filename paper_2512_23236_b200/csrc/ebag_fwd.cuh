@@ -36,6 +36,8 @@ namespace ebag {
 
 enum : int { DT_F32 = 0, DT_F16 = 1, DT_BF16 = 2, DT_INT8 = 3 };
 
+constexpr int kMaxTablesAny = 2048;      // EBAG_MAX_TABLES
+constexpr size_t kMaxItemTableBytes = (2 * kMaxTablesAny + 1) * sizeof(int);   // the kernel's dynamic shared memory at most
 constexpr int kThreads = 256;            // 8 warps per CTA
 constexpr int kWarps = kThreads / 32;
 constexpr int kMaxItemBags = 32;         // an item's offsets live in one register per lane
@@ -1047,6 +1049,12 @@ EBAG_DECLARE_LAUNCHERS(int8)
                                           : (const void*)ebag_fwd_kernel<DT, false, true>)        \
                               : (weighted ? (const void*)ebag_fwd_kernel<DT, true, false>         \
                                           : (const void*)ebag_fwd_kernel<DT, false, false>);      \
+        /* static + dynamic shared memory passes 48 KB when there are many tables: opt in, once   \
+           and for the most tables any handle may have (the attribute belongs to the kernel, not  \
+           to the handle) */                                                                     \
+        cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize,      \
+                                             (int)(smem > kMaxItemTableBytes ? smem : kMaxItemTableBytes)); \
+        if (e != cudaSuccess) return e;                                                          \
         return cudaOccupancyMaxActiveBlocksPerMultiprocessor(n, k, kThreads, smem);              \
     }
 

@@ -258,6 +258,34 @@ def test_bad_offsets_treated_as_empty_and_counted():
     pu.compare(gpu, ref, wl.F32)
 
 
+def test_maximum_number_of_tables():
+    """EBAG_MAX_TABLES tables in one launch (the item table of the kernel lives in shared memory
+    and grows with T); one more table is refused at create time."""
+    rng = np.random.default_rng(31)
+    T, B = 2048, 5
+    Ds = [int(4 * rng.integers(1, 9)) for _ in range(T)]
+    rows = [int(rng.integers(1, 30)) for _ in range(T)]
+    lens = [rng.integers(0, 6, size=B) for _ in range(T)]
+    idx, off, lengths = _jagged_from_lengths(rng, lens, rows)
+    tabs = _rand_tables(rng, wl.F32, rows, Ds)
+    gpu, status, ref = _both(wl.F32, rows, Ds, tabs, idx, off, B, wl.MEAN)
+    assert status == (0, 0, 0)
+    pu.compare(gpu, ref, wl.F32, lengths, T, B, Ds)
+    with pytest.raises(eb.EbagError) as e:
+        eb.TBE([4] * 2049, [4] * 2049, eb.EBAG_F32)
+    assert e.value.status == eb.EBAG_ERR_UNSUPPORTED
+    tbe = eb.TBE([4] * 2048, [4] * 2048, eb.EBAG_F32)
+    try:
+        z = torch.zeros(4, 4, device="cuda")
+        off = torch.zeros(1, dtype=torch.int64, device="cuda")
+        with pytest.raises(eb.EbagError) as e:                 # T * B must stay below 2^31
+            eb.ebag_forward(tbe._h, [z.data_ptr()] * 2048, [4] * 2048, None, 0, off.data_ptr(), None,
+                            1 << 20, 0, z.data_ptr(), 0)
+        assert e.value.status == eb.EBAG_ERR_UNSUPPORTED
+    finally:
+        tbe.close()
+
+
 def test_host_side_argument_errors():
     tbe = eb.TBE([10], [16], eb.EBAG_F32, device=torch.cuda.current_device())
     tab = torch.zeros(10, 16, device="cuda")
