@@ -538,6 +538,7 @@ def run_bwd(args, rank, local_rank, world):
         assert tbe.last_status(stream) == (0, 0, 0)
         bl.barrier()
         torch.cuda.synchronize()
+        launches0 = tbe.launch_count()
         ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
               for _ in range(args.steps)]
         for a, b in ev:
@@ -547,6 +548,7 @@ def run_bwd(args, rank, local_rank, world):
             b.record(stream)
         torch.cuda.synchronize()
         bl.barrier()
+        launches = tbe.launch_count() - launches0
         step_ms = [a.elapsed_time(b) for a, b in ev]
         elapsed_ms = float(sum(step_ms))
         # end to end: host grad_out, ids and offsets in; the gradient tables stay on the device
@@ -579,7 +581,7 @@ def run_bwd(args, rank, local_rank, world):
     line = {"metric": "pooled_lookups_per_sec", "value": total / (max_ms * 1e-3), "unit": "lookups/s",
             "n_gpus": world, "steps": args.steps, "warmup": warmup, "ms_per_step": max_ms / args.steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
-            "data": "synthetic", "config": config, "clocks": clocks, "gpu_launches": args.steps,
+            "data": "synthetic", "config": config, "clocks": clocks, "gpu_launches": launches,
             "e2e": {"value": e2e_total / (e2e_max * 1e-3), "unit": "lookups/s",
                     "h2d_bytes_per_step": int(h_idx.numel() * 8 + h_off.numel() * 8 + h_G.numel() * 4),
                     "d2h_bytes_per_step": 16, "steps": e2e_steps, "ms_per_step": e2e_max / e2e_steps},

@@ -46,6 +46,7 @@ struct ebag_tbe {
     std::vector<int32_t> D;
     TableMeta* d_meta = nullptr;
     BwdTableMeta* d_bwd_meta = nullptr;            // built by the first ebag_backward
+    int32_t* d_bwd_hot = nullptr;                  // [T, kHotSlots] sampled hot rows of the current call
     int bwd_occupancy[2] = {};
     Queue* d_queue = nullptr;
     Status* d_status = nullptr;
@@ -98,6 +99,7 @@ void free_handle(ebag_tbe* h) {
     if (!h) return;
     cudaFree(h->d_meta);
     cudaFree(h->d_bwd_meta);
+    cudaFree(h->d_bwd_hot);
     cudaFree(h->d_queue);
     cudaFree(h->d_status);
     cudaFree(h->d_long);
@@ -594,6 +596,7 @@ ebag_status ebag_backward(ebag_tbe* h, const float* grad_out, const void* indice
         EBAG_CUDA(h, cudaMalloc((void**)&h->d_bwd_meta, sizeof(BwdTableMeta) * h->T));
         EBAG_CUDA(h, cudaMemcpy(h->d_bwd_meta, meta.data(), sizeof(BwdTableMeta) * h->T,
                                 cudaMemcpyHostToDevice));
+        EBAG_CUDA(h, cudaMalloc((void**)&h->d_bwd_hot, sizeof(int32_t) * kHotSlots * h->T));
         for (int w = 0; w < 2; ++w) {
             EBAG_CUDA(h, occupancy_bwd(w != 0, h->T, &h->bwd_occupancy[w]));
             if (h->bwd_occupancy[w] < 1) h->bwd_occupancy[w] = 1;
@@ -617,10 +620,12 @@ ebag_status ebag_backward(ebag_tbe* h, const float* grad_out, const void* indice
     p.sumD = h->sumD;
     p.mean = mode == EBAG_MEAN ? 1 : 0;
     p.idx32 = index_bits == 32 ? 1 : 0;
+    p.hot = h->d_bwd_hot;
+    p.use_cache = 1;
     const bool w = per_sample_weights != nullptr;
     const int grid = h->num_sms * h->bwd_occupancy[w ? 1 : 0];
     EBAG_CUDA(h, launch_bwd(p, w, grid, s));
-    ++h->launches;
+    h->launches += 2;                           // the hot-row sampler, then the backward kernel
     return EBAG_OK;
 }
 

@@ -13,6 +13,14 @@
 // 32/G consecutive bags numbered w, w + W, ... in table-major order; the ids of a bag are read
 // four at a time (every lane of a group reads the same id, one transaction).
 //
+// Hot rows.  Reductions to one address are applied one after the other in L2, and with skewed
+// (Zipf) ids a handful of rows per table take a large share of its lookups: the whole grid then
+// queues on them (measured: 13 times slower than uniform ids).  So a first, small kernel samples
+// the ids of every table and puts its most frequent rows into a small hashed table of K slots
+// (K = 2048 / D, at most 32); every warp of the main kernel sums the contributions to those
+// rows in its own 8 KB of shared memory and sends each sum to L2 once per table it passes
+// through.
+//
 // The order in which the contributions to a row arrive is not fixed, so results are
 // reproducible only up to fp32 rounding.  Ids outside the table and malformed bags are skipped
 // and counted, as in the forward.
@@ -26,18 +34,104 @@ namespace ebag {
 namespace {
 
 constexpr int kBwdThreads = 256;
+constexpr int kBwdWarps = kBwdThreads / 32;
 constexpr int kTileVecs = 2;          // 16-byte vectors of grad_out a lane holds per column tile
 constexpr int kIdBatch = 4;           // ids of a bag fetched together
+#ifndef EBAG_HOT_USE
+#define EBAG_HOT_USE 32
+#endif
+constexpr int kHotUse = EBAG_HOT_USE;   // slots in use at most (<= kHotSlots)
+constexpr int kSampleIds = 2048;      // ids of a table the hot-row kernel looks at
+constexpr int kSampleSlots = 4096;    // its hash table (32 KB of shared memory)
 
 __device__ __forceinline__ void red_add_v4(float* addr, float a, float b, float c, float d) {
     asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(addr), "f"(a), "f"(b), "f"(c), "f"(d)
                  : "memory");
 }
 
+__device__ __forceinline__ int64_t load_id(const void* indices, int idx32, int64_t i) {
+    return idx32 ? (int64_t)__ldg(reinterpret_cast<const int*>(indices) + i)
+                 : (int64_t)__ldg(reinterpret_cast<const long long*>(indices) + i);
+}
+
+// ---- the most frequent rows of every table, from an evenly spaced sample of its ids.  One CTA
+// per table: the sampled ids are counted in a shared-memory hash table (linear probing), then
+// the kHotRows largest counts are picked one after the other.  A row must show up at least
+// three times in the sample to be named.
+__global__ void __launch_bounds__(kBwdThreads) bwd_hot_rows_kernel(const BwdParams p) {
+    __shared__ int keys[kSampleSlots];
+    __shared__ int counts[kSampleSlots];
+    __shared__ unsigned long long best;
+    const int t = blockIdx.x, tid = threadIdx.x;
+    for (int i = tid; i < kSampleSlots; i += kBwdThreads) {
+        keys[i] = -1;
+        counts[i] = 0;
+    }
+    __syncthreads();
+    int64_t o0 = p.offsets[(int64_t)t * p.B], o1 = p.offsets[(int64_t)(t + 1) * p.B];
+    if (o0 < 0) o0 = 0;
+    if (o1 > p.n_indices) o1 = p.n_indices;
+    const int64_t n = o1 > o0 ? o1 - o0 : 0;
+    const int64_t S = n < kSampleIds ? n : kSampleIds;
+    const int64_t rows = p.meta[t].rows;
+    for (int64_t i = tid; i < S; i += kBwdThreads) {
+        const int64_t r = load_id(p.indices, p.idx32, o0 + i * n / S);
+        if ((uint64_t)r >= (uint64_t)rows) continue;
+        unsigned slot = ((unsigned)r * 2654435761u) >> 20;                 // 12 bits
+        for (int probe = 0; probe < kSampleSlots; ++probe) {
+            const int old = atomicCAS(&keys[slot], -1, (int)r);
+            if (old == -1 || old == (int)r) {
+                atomicAdd(&counts[slot], 1);
+                break;
+            }
+            slot = (slot + 1) & (kSampleSlots - 1);
+        }
+    }
+    __syncthreads();
+    // candidates by decreasing count; each goes to the first of its two hash slots that is still free
+    const int D = p.meta[t].D;
+    int K = 1;
+    while (K * 2 <= kHotUse && K * 2 * D <= kCacheFloats) K *= 2;
+    if (D > kCacheFloats) K = 0;
+    if (tid < kHotSlots) p.hot[t * kHotSlots + tid] = -1;
+    __syncthreads();
+    for (int k = 0; k < 2 * K; ++k) {
+        if (tid == 0) best = 0;
+        __syncthreads();
+        unsigned long long mine = 0;
+        for (int i = tid; i < kSampleSlots; i += kBwdThreads)
+            if (counts[i] >= 3) {
+                const unsigned long long v = ((unsigned long long)counts[i] << 32) | (unsigned)i;
+                if (v > mine) mine = v;
+            }
+        if (mine) atomicMax(&best, mine);
+        __syncthreads();
+        const unsigned long long got = best;
+        if (got == 0) break;                                               // uniform: no candidates left
+        if (tid == 0) {
+            const int slot = (int)(got & 0xffffffffu);
+            const int row = keys[slot];
+            counts[slot] = 0;                                              // taken
+            int* d1 = p.hot + t * kHotSlots + hot_slot((uint32_t)row, K);
+            int* d2 = p.hot + t * kHotSlots + hot_slot2((uint32_t)row, K);
+            if (*d1 < 0) *d1 = row;
+            else if (*d2 < 0) *d2 = row;
+        }
+        __syncthreads();
+    }
+}
+
 template <bool WEIGHTED>
 __global__ void __launch_bounds__(kBwdThreads) ebag_bwd_kernel(const BwdParams p) {
-    extern __shared__ int item_base[];                        // [T+1] first item of each table
-    const int tid = threadIdx.x, lane = tid & 31;
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    // per warp: kCacheFloats floats of sums, then kHotSlots ids and kHotSlots flags; after all
+    // warps: item_base[T+1]
+    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    float* cache = reinterpret_cast<float*>(smem_raw) + (size_t)wid * kCacheFloats;
+    int* hot_s = reinterpret_cast<int*>(smem_raw + (size_t)kBwdWarps * kCacheFloats * sizeof(float)) +
+                 wid * 2 * kHotSlots;                                     // [ids | touched]
+    int* item_base = reinterpret_cast<int*>(smem_raw + (size_t)kBwdWarps * kCacheFloats * sizeof(float)) +
+                     kBwdWarps * 2 * kHotSlots;                           // [T+1] first item of each table
     // ---- items: groups of 32/G consecutive bags of a table
     for (int t = tid; t < p.T; t += kBwdThreads) {
         const int ng = 32 >> p.meta[t].g_log2;
@@ -50,10 +144,26 @@ __global__ void __launch_bounds__(kBwdThreads) ebag_bwd_kernel(const BwdParams p
     }
     __syncthreads();
     const int64_t total = item_base[p.T];
-    const int64_t warps = (int64_t)gridDim.x * (kBwdThreads / 32);
+    const int64_t warps = (int64_t)gridDim.x * kBwdWarps;
     unsigned n_oob = 0, n_bad = 0;
+    int cur_t = -1;                       // table whose hot rows this warp holds (-1: none)
+    int cur_K = 0;                        // its slots in use (0: not cached)
 
-    for (int64_t item = (int64_t)blockIdx.x * (kBwdThreads / 32) + (tid >> 5); item < total; item += warps) {
+    // sends the warp's cached sums of table `t` to the gradient table
+    auto flush = [&](int t, int K) {
+        const BwdTableMeta m = p.meta[t];
+        float* __restrict__ gt = p.grad_tables[t];
+        for (int k = 0; k < K; ++k) {
+            const int row = hot_s[k];
+            if (row < 0 || !hot_s[kHotSlots + k]) continue;
+            for (int vec = lane; vec < m.nvec; vec += 32) {
+                const float4 x = *reinterpret_cast<const float4*>(cache + (size_t)k * m.D + vec * 4);
+                red_add_v4(gt + row * (int64_t)m.D + vec * 4, x.x, x.y, x.z, x.w);
+            }
+        }
+    };
+
+    for (int64_t item = (int64_t)blockIdx.x * kBwdWarps + wid; item < total; item += warps) {
         int lo_t = 0, hi_t = p.T;
         while (hi_t - lo_t > 1) {
             const int mid = (lo_t + hi_t) >> 1;
@@ -61,6 +171,22 @@ __global__ void __launch_bounds__(kBwdThreads) ebag_bwd_kernel(const BwdParams p
         }
         const int t = lo_t;
         const BwdTableMeta m = p.meta[t];
+        if (t != cur_t) {                 // a new table: hand in the old sums, learn the new hot rows
+            __syncwarp();
+            if (cur_t >= 0 && cur_K > 0) flush(cur_t, cur_K);
+            __syncwarp();
+            cur_t = t;
+            cur_K = 0;
+            if (p.use_cache && m.D <= kCacheFloats) {
+                cur_K = 1;
+                while (cur_K * 2 <= kHotUse && cur_K * 2 * m.D <= kCacheFloats) cur_K *= 2;
+                hot_s[lane] = p.hot[t * kHotSlots + lane];                 // kHotSlots == 32 lanes
+                hot_s[kHotSlots + lane] = 0;
+                for (int i = lane; i < cur_K * m.D / 4; i += 32)
+                    reinterpret_cast<float4*>(cache)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+            __syncwarp();
+        }
         const int G = 1 << m.g_log2, ng = 32 >> m.g_log2;
         const int lig = lane & (G - 1), grp = lane >> m.g_log2;
         const int64_t b = (item - item_base[t]) * ng + grp;
@@ -105,8 +231,7 @@ __global__ void __launch_bounds__(kBwdThreads) ebag_bwd_kernel(const BwdParams p
                     r[k] = -1;
                     w[k] = 1.0f;
                     if (j0 + k < L) {
-                        r[k] = p.idx32 ? (int64_t)__ldg(reinterpret_cast<const int*>(p.indices) + i)
-                                       : __ldg(reinterpret_cast<const long long*>(p.indices) + i);
+                        r[k] = load_id(p.indices, p.idx32, i);
                         if (WEIGHTED) w[k] = __ldg(p.weights + i);
                     }
                 }
@@ -115,6 +240,29 @@ __global__ void __launch_bounds__(kBwdThreads) ebag_bwd_kernel(const BwdParams p
                     if (j0 + k >= L) continue;
                     if ((uint64_t)r[k] >= (uint64_t)m.rows) {
                         if (lig == 0 && c0 == 0) ++n_oob;
+                        continue;
+                    }
+                    int slot = -1;
+                    if (cur_K > 0) {
+                        const int h1 = hot_slot((uint32_t)r[k], cur_K), h2 = hot_slot2((uint32_t)r[k], cur_K);
+                        if (hot_s[h1] == (int)r[k]) slot = h1;
+                        else if (hot_s[h2] == (int)r[k]) slot = h2;
+                    }
+                    if (slot >= 0) {
+                        // a hot row: summed here, in this warp's shared memory (several groups of
+                        // the warp may hit the same row at once, hence the atomics)
+                        if (lig == 0) hot_s[kHotSlots + slot] = 1;
+                        float* crow = cache + (size_t)slot * m.D;
+#pragma unroll
+                        for (int v = 0; v < kTileVecs; ++v)
+                            if (on[v]) {
+                                float* a = crow + (size_t)(c0 + v * G + lig) * 4;
+                                const float ww = WEIGHTED ? w[k] : 1.0f;
+                                atomicAdd(a + 0, ww * gv[v].x);
+                                atomicAdd(a + 1, ww * gv[v].y);
+                                atomicAdd(a + 2, ww * gv[v].z);
+                                atomicAdd(a + 3, ww * gv[v].w);
+                            }
                         continue;
                     }
                     float* row = gt + r[k] * (int64_t)m.D;
@@ -129,6 +277,8 @@ __global__ void __launch_bounds__(kBwdThreads) ebag_bwd_kernel(const BwdParams p
             }
         }
     }
+    __syncwarp();
+    if (cur_t >= 0 && cur_K > 0) flush(cur_t, cur_K);
     n_oob = __reduce_add_sync(0xffffffffu, n_oob);
     n_bad = __reduce_add_sync(0xffffffffu, n_bad);
     if (lane == 0) {
@@ -137,17 +287,36 @@ __global__ void __launch_bounds__(kBwdThreads) ebag_bwd_kernel(const BwdParams p
     }
 }
 
+template <typename K>
+cudaError_t allow_smem(K kernel, size_t bytes) {
+    return cudaFuncSetAttribute(reinterpret_cast<const void*>(kernel),
+                                cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+}
+
 }  // namespace
 
+size_t bwd_smem_bytes(int T) {
+    return (size_t)kBwdWarps * kCacheFloats * sizeof(float) + (size_t)kBwdWarps * 2 * kHotSlots * sizeof(int) +
+           (size_t)(T + 1) * sizeof(int);
+}
+
 cudaError_t launch_bwd(const BwdParams& p, bool weighted, int grid, cudaStream_t s) {
-    const size_t smem = (size_t)(p.T + 1) * sizeof(int);
+    if (p.use_cache) {
+        bwd_hot_rows_kernel<<<p.T, kBwdThreads, 0, s>>>(p);
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+    }
+    const size_t smem = bwd_smem_bytes(p.T);
     if (weighted) ebag_bwd_kernel<true><<<grid, kBwdThreads, smem, s>>>(p);
     else ebag_bwd_kernel<false><<<grid, kBwdThreads, smem, s>>>(p);
     return cudaGetLastError();
 }
 
 cudaError_t occupancy_bwd(bool weighted, int T, int* ctas_per_sm) {
-    const size_t smem = (size_t)(T + 1) * sizeof(int);
+    const size_t smem = bwd_smem_bytes(T);
+    cudaError_t e = weighted ? allow_smem(ebag_bwd_kernel<true>, bwd_smem_bytes(2048))
+                             : allow_smem(ebag_bwd_kernel<false>, bwd_smem_bytes(2048));
+    if (e != cudaSuccess) return e;
     return weighted ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(ctas_per_sm, ebag_bwd_kernel<true>,
                                                                      kBwdThreads, smem)
                     : cudaOccupancyMaxActiveBlocksPerMultiprocessor(ctas_per_sm, ebag_bwd_kernel<false>,

@@ -16,6 +16,13 @@ struct BwdTableMeta {        // per table; gradient tables are dense fp32 [rows,
     int32_t g_log2;          // log2 of the lanes that cover a row (or one column tile of it)
 };
 
+constexpr int kHotSlots = 32;        // hot-row slots per table (a table of width D uses the first K = min(32, 2048 / D))
+constexpr int kCacheFloats = 2048;   // floats of shared memory per warp for the sums of hot rows (8 KB)
+
+// the two slots row r may sit in among K slots (K a power of two)
+__host__ __device__ inline int hot_slot(uint32_t r, int K) { return (int)((r * 2654435761u) >> 27) & (K - 1); }
+__host__ __device__ inline int hot_slot2(uint32_t r, int K) { return (int)((r * 0x85EBCA6Bu) >> 27) & (K - 1); }
+
 struct BwdParams {
     float* const* grad_tables;   // device [T]
     const BwdTableMeta* meta;    // device [T]
@@ -30,8 +37,11 @@ struct BwdParams {
     int32_t sumD;
     int32_t mean;
     int32_t idx32;
+    int32_t* hot;                // [T, kHotSlots] frequent rows of every table by a sample, at their hash slot (-1: none)
+    int32_t use_cache;           // 0: hot rows are not looked for
 };
 
+size_t bwd_smem_bytes(int T);
 cudaError_t launch_bwd(const BwdParams& p, bool weighted, int grid, cudaStream_t s);
 cudaError_t occupancy_bwd(bool weighted, int T, int* ctas_per_sm);
 
