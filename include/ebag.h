@@ -129,8 +129,10 @@ ebag_status ebag_forward_i32(ebag_tbe* h, const void* const* tables, const int32
  *   grad_tables  host array [T] of DEVICE pointers to dense fp32 [rows[t], D[t]] arrays (whatever
  *                the storage type of the tables), 16-byte aligned, owned and zeroed by the caller:
  *                the call ADDS into them.  Needs D[t] % 4 == 0 (else UNSUPPORTED).
- * One kernel launch on `stream`, no allocation after the first call (which builds a few KB of
- * metadata), no synchronisation.  Contributions are added with floating-point reductions in
+ * Two kernel launches on `stream` (a short one that samples the ids of every table for its most
+ * frequent rows, whose contributions are then summed in shared memory before they reach the
+ * gradient table, and the backward proper), no allocation after the first call (which builds a
+ * few KB of metadata), no synchronisation.  Contributions are added with floating-point reductions in
  * memory whose order is not fixed: two runs agree up to fp32 rounding, not bit for bit.  Ids
  * outside the table and malformed bags are skipped and counted as in the forward
  * (ebag_last_status).  The gradient with respect to per_sample_weights is not computed.
