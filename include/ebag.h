@@ -49,7 +49,8 @@ typedef enum {
     EBAG_ERR_BAD_OFFSETS = 5  /* reported by ebag_last_status: malformed bags were treated as empty */
 } ebag_status;
 
-typedef enum { EBAG_F32 = 0, EBAG_F16 = 1, EBAG_BF16 = 2, EBAG_INT8_ROWWISE = 3 } ebag_dtype;
+typedef enum { EBAG_F32 = 0, EBAG_F16 = 1, EBAG_BF16 = 2, EBAG_INT8_ROWWISE = 3,
+               EBAG_UINT8_ROWWISE = 4 } ebag_dtype;
 
 /* weighted sum = EBAG_SUM with per_sample_weights != NULL */
 typedef enum { EBAG_SUM = 0, EBAG_MEAN = 1 } ebag_mode;
@@ -57,12 +58,14 @@ typedef enum { EBAG_SUM = 0, EBAG_MEAN = 1 } ebag_mode;
 #define EBAG_MAX_TABLES 2048
 
 /*
- * Bytes from one stored row to the next.  F32/F16/BF16: D * element size.  INT8_ROWWISE: the
- * packed row [D codes, each stored as q + 128 in one byte][fp32 scale][fp32 bias][8 bytes pad]
+ * Bytes from one stored row to the next.  F32/F16/BF16: D * element size.  INT8_ROWWISE and
+ * UINT8_ROWWISE (value = scale[row] * code + bias[row], code signed or unsigned 8-bit): the
+ * packed row [D codes, one byte each: q + 128 for signed codes, the code itself for unsigned
+ * ones][fp32 scale][fp32 bias][8 bytes pad]
  * = D + 16 (one gather fetches codes and dequantisation constants together; build it with
- * ebag_pack_int8_rowwise).  Returns -1 if D is not allowed for the dtype:
+ * ebag_pack_int8_rowwise or ebag_pack_uint8_rowwise).  Returns -1 if D is not allowed for the dtype:
  * D > 0 and D * element size must be a multiple of 16 bytes (D%4==0 for F32, D%8==0 for
- * F16/BF16, D%16==0 for INT8_ROWWISE), so that rows can be gathered with 128-bit loads.
+ * F16/BF16, D%16==0 for the rowwise types), so that rows can be gathered with 128-bit loads.
  */
 int64_t ebag_row_stride(ebag_dtype dtype, int32_t D);
 
@@ -177,6 +180,10 @@ ebag_status ebag_last_status(ebag_tbe* h, ebag_stream stream, int64_t* n_oob,
  */
 ebag_status ebag_pack_int8_rowwise(const int8_t* q, const float* scale, const float* bias,
                                    int64_t rows, int32_t D, void* dst, ebag_stream stream);
+
+/* The same for UINT8_ROWWISE tables: q [rows, D] holds unsigned codes. */
+ebag_status ebag_pack_uint8_rowwise(const uint8_t* q, const float* scale, const float* bias,
+                                    int64_t rows, int32_t D, void* dst, ebag_stream stream);
 
 /*
  * MapId transform (paper Sec. 5.4.1 "MapId Transform"): `mapping` is a sorted (strictly

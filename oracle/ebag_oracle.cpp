@@ -47,7 +47,7 @@
 
 namespace {
 
-enum { DT_F32 = 0, DT_F16 = 1, DT_BF16 = 2, DT_INT8_ROWWISE = 3 };
+enum { DT_F32 = 0, DT_F16 = 1, DT_BF16 = 2, DT_INT8_ROWWISE = 3, DT_UINT8_ROWWISE = 4 };
 enum { MODE_SUM = 0, MODE_MEAN = 1 };
 
 inline float bits_to_float(uint32_t u) {
@@ -85,8 +85,8 @@ int ebag_oracle_max_threads(void) {
 
 // Returns 0 on success, 1 on an invalid argument.  All pointers are HOST pointers.
 //   tables[t]  : dense row-major [rows[t], D[t]] of float (F32), uint16_t bit patterns (F16, BF16)
-//                or int8_t codes (INT8_ROWWISE)
-//   scales[t], biases[t] : [rows[t]] fp32, INT8_ROWWISE only (else the arrays may be NULL)
+//                or int8_t codes (INT8_ROWWISE) or uint8_t codes (UINT8_ROWWISE)
+//   scales[t], biases[t] : [rows[t]] fp32, the two rowwise types only (else the arrays may be NULL)
 //   indices    : [n_indices] int64;  weights : [n_indices] fp32 or NULL
 //   offsets    : [T*B + 1] int64
 //   out32      : [B, sum(D)] fp32, fully overwritten
@@ -99,9 +99,9 @@ int ebag_oracle_forward(int32_t T, const int64_t* rows, const int32_t* D, int32_
                         float* out32, double* out64, double* S, int64_t* n_oob,
                         int64_t* n_bad_offsets, int32_t nthreads) {
     if (T <= 0 || B < 0 || !rows || !D || !tables || !offsets || !out32) return 1;
-    if (dtype < DT_F32 || dtype > DT_INT8_ROWWISE) return 1;
+    if (dtype < DT_F32 || dtype > DT_UINT8_ROWWISE) return 1;
     if (mode != MODE_SUM && mode != MODE_MEAN) return 1;
-    if (dtype == DT_INT8_ROWWISE && (!scales || !biases)) return 1;
+    if ((dtype == DT_INT8_ROWWISE || dtype == DT_UINT8_ROWWISE) && (!scales || !biases)) return 1;
     std::vector<int64_t> Doff(T + 1, 0);
     for (int32_t t = 0; t < T; ++t) {
         if (D[t] <= 0 || rows[t] < 0) return 1;
@@ -146,7 +146,9 @@ int ebag_oracle_forward(int32_t T, const int64_t* rows, const int32_t* D, int32_
                         case DT_F16:  x = half_to_float(((const uint16_t*)tables[t])[at]); break;
                         case DT_BF16: x = bf16_to_float(((const uint16_t*)tables[t])[at]); break;
                         default: {
-                            const float q = (float)((const int8_t*)tables[t])[at];
+                            const float q = dtype == DT_UINT8_ROWWISE
+                                                ? (float)((const uint8_t*)tables[t])[at]
+                                                : (float)((const int8_t*)tables[t])[at];
                             const float sq = scales[t][r] * q;      // rounded product
                             x = sq + biases[t][r];                  // rounded sum
                         }

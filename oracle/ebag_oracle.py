@@ -17,7 +17,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "ebag_oracle.cpp")
 _LIB = os.path.join(_HERE, "libebag_oracle.so")
 
-F32, F16, BF16, INT8_ROWWISE = 0, 1, 2, 3
+F32, F16, BF16, INT8_ROWWISE, UINT8_ROWWISE = 0, 1, 2, 3, 4
 SUM, MEAN = 0, 1
 
 _lib = None
@@ -50,7 +50,8 @@ def max_threads() -> int:
     return int(_load().ebag_oracle_max_threads())
 
 
-_TABLE_NP = {F32: np.float32, F16: np.uint16, BF16: np.uint16, INT8_ROWWISE: np.int8}
+_TABLE_NP = {F32: np.float32, F16: np.uint16, BF16: np.uint16, INT8_ROWWISE: np.int8,
+             UINT8_ROWWISE: np.uint8}
 
 
 def _ptr_array(arrs):
@@ -62,7 +63,8 @@ def forward(tables, dtype, indices, offsets, B, mode=SUM, weights=None, scales=N
     """Run the oracle.
 
     tables : list of T numpy arrays [rows_t, D_t]; float32 (F32), uint16 bit patterns (F16/BF16)
-             or int8 codes (INT8_ROWWISE, with ``scales``/``biases`` lists of float32 [rows_t]).
+             or int8 / uint8 codes (INT8_ROWWISE / UINT8_ROWWISE, with ``scales``/``biases`` lists of
+             float32 [rows_t]: value = scale * code + bias).
     Returns dict(out32 [B, sumD] f32, out64, S (f64 or None), n_oob, n_bad_offsets).
     """
     lib = _load()
@@ -83,7 +85,7 @@ def forward(tables, dtype, indices, offsets, B, mode=SUM, weights=None, scales=N
     if w is not None and w.shape[0] != indices.shape[0]:
         raise ValueError("weights must pair with indices")
     sc = bi = None
-    if dtype == INT8_ROWWISE:
+    if dtype in (INT8_ROWWISE, UINT8_ROWWISE):
         sc = [np.ascontiguousarray(s, dtype=np.float32) for s in scales]
         bi = [np.ascontiguousarray(s, dtype=np.float32) for s in biases]
     sumD = int(D.sum())

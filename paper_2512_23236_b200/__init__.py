@@ -12,7 +12,7 @@ import ctypes
 import os
 from typing import List, Optional, Sequence
 
-EBAG_F32, EBAG_F16, EBAG_BF16, EBAG_INT8_ROWWISE = 0, 1, 2, 3
+EBAG_F32, EBAG_F16, EBAG_BF16, EBAG_INT8_ROWWISE, EBAG_UINT8_ROWWISE = 0, 1, 2, 3, 4
 EBAG_SUM, EBAG_MEAN = 0, 1
 EBAG_OK, EBAG_ERR_INVALID_ARG, EBAG_ERR_UNSUPPORTED, EBAG_ERR_CUDA = 0, 1, 2, 3
 EBAG_ERR_INDEX_OOB, EBAG_ERR_BAD_OFFSETS = 4, 5
@@ -43,6 +43,7 @@ SIGNATURES = {
                                   _vp]),
     "ebag_last_status": (_int, [_vp, _vp, _vp, _vp]),
     "ebag_pack_int8_rowwise": (_int, [_vp, _vp, _vp, _i64, _i32, _vp, _vp]),
+    "ebag_pack_uint8_rowwise": (_int, [_vp, _vp, _vp, _i64, _i32, _vp, _vp]),
     "ebag_set_param": (_int, [_vp, ctypes.c_char_p, _i64]),
     "ebag_launch_count": (_i64, [_vp]),
     "ebag_last_cuda_error": (ctypes.c_char_p, [_vp]),
@@ -215,8 +216,11 @@ def ebag_destroy(h: int) -> None:
 
 
 def ebag_pack_int8_rowwise(q, scale, bias, stream=None):
-    """torch int8 [rows, D], fp32 [rows], fp32 [rows] (device) -> packed uint8 [rows, D+16]."""
+    """torch int8 (or uint8, for EBAG_UINT8_ROWWISE tables) [rows, D], fp32 [rows], fp32 [rows]
+    (device) -> packed uint8 [rows, D+16]."""
     import torch
+    if q.dtype not in (torch.int8, torch.uint8):
+        raise TypeError("codes must be int8 or uint8")
     rows, D = q.shape
     stride = ebag_row_stride(EBAG_INT8_ROWWISE, D)
     if stride < 0:
@@ -226,10 +230,13 @@ def ebag_pack_int8_rowwise(q, scale, bias, stream=None):
     bias = bias.contiguous().float()
     dst = torch.empty((rows, stride), dtype=torch.uint8, device=q.device)
     with torch.cuda.device(q.device):
-        st = lib().ebag_pack_int8_rowwise(_ptr(q), _ptr(scale), _ptr(bias), rows, D, _ptr(dst),
-                                          _stream_ptr(stream))
+        fn = lib().ebag_pack_uint8_rowwise if q.dtype == torch.uint8 else lib().ebag_pack_int8_rowwise
+        st = fn(_ptr(q), _ptr(scale), _ptr(bias), rows, D, _ptr(dst), _stream_ptr(stream))
     _check(st, "ebag_pack_int8_rowwise")
     return dst
+
+
+ebag_pack_uint8_rowwise = ebag_pack_int8_rowwise     # the code type of `q` selects the entry point
 
 
 # ---------------------------------------------------------------- convenience wrapper

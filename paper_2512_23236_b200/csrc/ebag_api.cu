@@ -36,7 +36,8 @@ struct DeviceGuard {             // make the handle's device current for the dur
     }
 };
 
-int elem_bytes(int dtype) { return dtype == EBAG_F32 ? 4 : (dtype == EBAG_INT8_ROWWISE ? 1 : 2); }
+bool is_rowwise8(int dtype) { return dtype == EBAG_INT8_ROWWISE || dtype == EBAG_UINT8_ROWWISE; }
+int elem_bytes(int dtype) { return dtype == EBAG_F32 ? 4 : (is_rowwise8(dtype) ? 1 : 2); }
 
 }  // namespace
 
@@ -233,6 +234,7 @@ ebag_status forward_device(ebag_tbe* h, const void* const* tables, const int64_t
     p.sumD = h->sumD;
     p.mean = mode == EBAG_MEAN ? 1 : 0;
     p.idx32 = idx32 ? 1 : 0;
+    p.code_zero = h->dtype == EBAG_UINT8_ROWWISE ? 0.0f : 128.0f;
     p.item_bytes = h->item_bytes;
     // Long bags.  The bytes this call can gather are at most n_indices * (widest row), so at most
     // that / long_bytes bags can reach long_bytes; with long_bytes = 4 * part_bytes (a power of two) and
@@ -279,7 +281,7 @@ ebag_status grow(ebag_tbe* h, T** buf, int64_t* cap, int64_t need) {
 
 __global__ void pack_int8_rowwise_kernel(const int8_t* __restrict__ q, const float* __restrict__ scale,
                                          const float* __restrict__ bias, int64_t rows, int D,
-                                         uint4* __restrict__ dst) {
+                                         uint4* __restrict__ dst, uint32_t flip) {
     // one thread per 16-byte vector of the packed row: D/16 vectors of codes, stored biased by
     // +128 (sign bit flipped) so that the forward kernel widens them without a sign fix-up, then
     // one vector holding scale, bias and 8 bytes of zero padding
@@ -292,10 +294,10 @@ __global__ void pack_int8_rowwise_kernel(const int8_t* __restrict__ q, const flo
         uint4 x;
         if (v < vecs - 1) {
             x = *reinterpret_cast<const uint4*>(q + r * D + v * 16);
-            x.x ^= 0x80808080u;
-            x.y ^= 0x80808080u;
-            x.z ^= 0x80808080u;
-            x.w ^= 0x80808080u;
+            x.x ^= flip;                  // 0x80808080 for signed codes, 0 for unsigned ones
+            x.y ^= flip;
+            x.z ^= flip;
+            x.w ^= flip;
         } else {
             x = make_uint4(__float_as_uint(scale[r]), __float_as_uint(bias[r]), 0u, 0u);
         }
@@ -420,17 +422,17 @@ ebag_status ebag_forward_mapid(ebag_tbe* h, const void* const* tables, const int
 }
 
 int64_t ebag_row_stride(ebag_dtype dtype, int32_t D) {
-    if (D <= 0 || dtype < EBAG_F32 || dtype > EBAG_INT8_ROWWISE) return -1;
+    if (D <= 0 || dtype < EBAG_F32 || dtype > EBAG_UINT8_ROWWISE) return -1;
     const int64_t payload = (int64_t)D * elem_bytes(dtype);
     if (payload % 16 != 0) return -1;
-    return dtype == EBAG_INT8_ROWWISE ? payload + 16 : payload;
+    return (dtype == EBAG_INT8_ROWWISE || dtype == EBAG_UINT8_ROWWISE) ? payload + 16 : payload;
 }
 
 ebag_status ebag_create_tbe(int32_t T, const int64_t* rows, const int32_t* D, ebag_dtype dtype,
                             int device, ebag_tbe** out) {
     if (!out) return EBAG_ERR_INVALID_ARG;
     *out = nullptr;
-    if (T <= 0 || !rows || !D || dtype < EBAG_F32 || dtype > EBAG_INT8_ROWWISE)
+    if (T <= 0 || !rows || !D || dtype < EBAG_F32 || dtype > EBAG_UINT8_ROWWISE)
         return EBAG_ERR_INVALID_ARG;
     if (T > EBAG_MAX_TABLES) return EBAG_ERR_UNSUPPORTED;
     std::vector<TableMeta> meta(T);
@@ -734,8 +736,9 @@ ebag_status ebag_last_status(ebag_tbe* h, ebag_stream stream, int64_t* n_oob, in
     return EBAG_OK;
 }
 
-ebag_status ebag_pack_int8_rowwise(const int8_t* q, const float* scale, const float* bias,
-                                   int64_t rows, int32_t D, void* dst, ebag_stream stream) {
+namespace {
+ebag_status pack_rowwise8(const void* q, const float* scale, const float* bias, int64_t rows, int32_t D,
+                          void* dst, uint32_t flip, ebag_stream stream) {
     if (rows < 0 || ebag_row_stride(EBAG_INT8_ROWWISE, D) < 0) return EBAG_ERR_INVALID_ARG;
     if (rows == 0) return EBAG_OK;
     if (!q || !scale || !bias || !dst) return EBAG_ERR_INVALID_ARG;
@@ -744,10 +747,21 @@ ebag_status ebag_pack_int8_rowwise(const int8_t* q, const float* scale, const fl
     int64_t blocks = (total + 255) / 256;
     if (blocks > 148 * 32) blocks = 148 * 32;
     pack_int8_rowwise_kernel<<<(int)blocks, 256, 0, (cudaStream_t)stream>>>(
-        q, scale, bias, rows, D, static_cast<uint4*>(dst));
+        static_cast<const int8_t*>(q), scale, bias, rows, D, static_cast<uint4*>(dst), flip);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(nullptr, e);
     return EBAG_OK;
+}
+}  // namespace
+
+ebag_status ebag_pack_int8_rowwise(const int8_t* q, const float* scale, const float* bias,
+                                   int64_t rows, int32_t D, void* dst, ebag_stream stream) {
+    return pack_rowwise8(q, scale, bias, rows, D, dst, 0x80808080u, stream);
+}
+
+ebag_status ebag_pack_uint8_rowwise(const uint8_t* q, const float* scale, const float* bias,
+                                    int64_t rows, int32_t D, void* dst, ebag_stream stream) {
+    return pack_rowwise8(q, scale, bias, rows, D, dst, 0u, stream);
 }
 
 ebag_status ebag_set_param(ebag_tbe* h, const char* name, int64_t value) {

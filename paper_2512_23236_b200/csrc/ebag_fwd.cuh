@@ -126,6 +126,7 @@ struct FwdParams {
     int32_t sumD;
     int32_t mean;                // 1: divide by the bag length
     int32_t idx32;               // 1: `indices` holds 32-bit ids
+    float code_zero;             // rowwise 8-bit tables: the stored byte that means code 0 (128 signed, 0 unsigned)
     uint32_t item_bytes;
     LongParams lg;
 };
@@ -576,7 +577,7 @@ __device__ __forceinline__ void process_item(const FwdParams& p, const TableMeta
                     const float2 sb = lds64f(my_sb_s + (st * kStageVecs + u) * 64);
                     acc_bias = fmaf(wu, sb.y, acc_bias);
                     wu *= sb.x;
-                    acc_bias = fmaf(wu, -128.0f, acc_bias);
+                    acc_bias = fmaf(wu, -p.code_zero, acc_bias);
                     wu *= kInt8Up;
                 }
 #pragma unroll
@@ -596,7 +597,7 @@ __device__ __forceinline__ void process_item(const FwdParams& p, const TableMeta
                     const float2 sb = lds64f(my_sb_s + (st * kStageVecs + u) * 64);
                     acc_bias = fmaf(wu, sb.y, acc_bias);
                     wu *= sb.x;
-                    acc_bias = fmaf(wu, -128.0f, acc_bias);
+                    acc_bias = fmaf(wu, -p.code_zero, acc_bias);
                     wu *= kInt8Up;
                 }
 #pragma unroll

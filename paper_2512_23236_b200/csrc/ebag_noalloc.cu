@@ -69,7 +69,7 @@ struct DeviceState {
 DeviceState g_state[kMaxDevices];
 std::mutex g_mutex;
 
-int elem_bytes(int dtype) { return dtype == EBAG_F32 ? 4 : (dtype == EBAG_INT8_ROWWISE ? 1 : 2); }
+int elem_bytes(int dtype) { return dtype == EBAG_F32 ? 4 : (dtype >= EBAG_INT8_ROWWISE ? 1 : 2); }
 
 size_t fwd_smem_bytes(int T) { return (size_t)(2 * T + 1) * sizeof(int); }
 
@@ -135,7 +135,7 @@ extern "C" ebag_status ebag_forward_noalloc(int32_t T, const int64_t* rows, cons
                                             ebag_stream stream) {
     if (T <= 0 || !rows || !D || !tables || !offsets || B < 0 || n_indices < 0)
         return EBAG_ERR_INVALID_ARG;
-    if (dtype < EBAG_F32 || dtype > EBAG_INT8_ROWWISE) return EBAG_ERR_INVALID_ARG;
+    if (dtype < EBAG_F32 || dtype > EBAG_UINT8_ROWWISE) return EBAG_ERR_INVALID_ARG;
     if (mode != EBAG_SUM && mode != EBAG_MEAN) return EBAG_ERR_INVALID_ARG;
     if (T > kMaxTables) return EBAG_ERR_UNSUPPORTED;       // beyond the static scratch
     if ((int64_t)T * B >= (1ll << 31)) return EBAG_ERR_UNSUPPORTED;
@@ -201,10 +201,12 @@ extern "C" ebag_status ebag_forward_noalloc(int32_t T, const int64_t* rows, cons
     p.sumD = (int32_t)d_off;
     p.mean = mode == EBAG_MEAN ? 1 : 0;
     p.idx32 = 0;
+    p.code_zero = dtype == EBAG_UINT8_ROWWISE ? 0.0f : 128.0f;
     p.item_bytes = 32768;
     p.lg = LongParams{};                     // no room for partial sums here: bags are not split
     const bool w = per_sample_weights != nullptr;
-    const int grid = st->num_sms * st->occupancy[dtype][w ? 1 : 0];
+    const int kernel_of = dtype > EBAG_INT8_ROWWISE ? EBAG_INT8_ROWWISE : dtype;   // both 8-bit types share kernels
+    const int grid = st->num_sms * st->occupancy[kernel_of][w ? 1 : 0];
     if (launch(dtype, p, w, grid, fwd_smem_bytes(T), s) != cudaSuccess) {
         cudaGetLastError();
         return EBAG_ERR_CUDA;

@@ -37,12 +37,13 @@ from typing import List, Optional
 import numpy as np
 import torch
 
-F32, F16, BF16, INT8_ROWWISE = 0, 1, 2, 3
+F32, F16, BF16, INT8_ROWWISE, UINT8_ROWWISE = 0, 1, 2, 3, 4
 SUM, MEAN = 0, 1
 
-DTYPE_NAMES = {F32: "f32", F16: "f16", BF16: "bf16", INT8_ROWWISE: "int8_rowwise"}
+DTYPE_NAMES = {F32: "f32", F16: "f16", BF16: "bf16", INT8_ROWWISE: "int8_rowwise",
+               UINT8_ROWWISE: "uint8_rowwise"}
 _TORCH_DT = {F32: torch.float32, F16: torch.float16, BF16: torch.bfloat16,
-             INT8_ROWWISE: torch.int8}
+             INT8_ROWWISE: torch.int8, UINT8_ROWWISE: torch.uint8}
 
 
 @dataclasses.dataclass
@@ -175,14 +176,17 @@ def gen_jagged(w: Workload) -> Jagged:
 def gen_table(w: Workload, t: int, device="cpu"):
     """Values of table ``t`` as torch tensors on ``device``.
 
-    F32/F16/BF16: one tensor [rows, D] of that dtype.  INT8_ROWWISE: (codes int8 [rows, D],
-    scale float32 [rows], bias float32 [rows])."""
+    F32/F16/BF16: one tensor [rows, D] of that dtype.  INT8_ROWWISE / UINT8_ROWWISE: (codes int8 /
+    uint8 [rows, D], scale float32 [rows], bias float32 [rows])."""
     dev = torch.device(device)
     g = torch.Generator(device=dev)
     g.manual_seed((w.seed * 1_000_003 + w.number) * 4099 + t)
     rows, D = w.rows[t], w.D[t]
-    if w.dtype == INT8_ROWWISE:
-        q = torch.randint(-128, 128, (rows, D), dtype=torch.int8, device=dev, generator=g)
+    if w.dtype in (INT8_ROWWISE, UINT8_ROWWISE):
+        if w.dtype == INT8_ROWWISE:
+            q = torch.randint(-128, 128, (rows, D), dtype=torch.int8, device=dev, generator=g)
+        else:
+            q = torch.randint(0, 256, (rows, D), dtype=torch.uint8, device=dev, generator=g)
         scale = torch.empty(rows, dtype=torch.float32, device=dev).uniform_(0.01, 0.03,
                                                                             generator=g)
         bias = torch.empty(rows, dtype=torch.float32, device=dev).normal_(0.0, 0.1, generator=g)
@@ -231,8 +235,8 @@ def algorithmic_bytes(w: Workload, lengths: np.ndarray) -> dict:
     """Bytes the operator itself must move for this input: per lookup the stored row
     (D*elem, plus 8 for rowwise int8 scale+bias), the int64 id and, if weighted, the fp32
     weight; per bag one int64 offset and the fp32 output row."""
-    elem = {F32: 4, F16: 2, BF16: 2, INT8_ROWWISE: 1}[w.dtype]
-    extra = 8 if w.dtype == INT8_ROWWISE else 0
+    elem = {F32: 4, F16: 2, BF16: 2, INT8_ROWWISE: 1, UINT8_ROWWISE: 1}[w.dtype]
+    extra = 8 if w.dtype in (INT8_ROWWISE, UINT8_ROWWISE) else 0
     gathered = 0
     n = 0
     for t in range(w.T):

@@ -15,14 +15,15 @@ import paper_2512_23236_b200 as eb
 from oracle import ebag_oracle as orc
 from paper_2512_23236_b200 import workloads as wl
 
-TOL = {wl.F32: 1e-5, wl.F16: 2e-3, wl.BF16: 2e-3, wl.INT8_ROWWISE: 2e-3}
+TOL = {wl.F32: 1e-5, wl.F16: 2e-3, wl.BF16: 2e-3, wl.INT8_ROWWISE: 2e-3, wl.UINT8_ROWWISE: 2e-3}
+ROWWISE8 = (wl.INT8_ROWWISE, wl.UINT8_ROWWISE)
 
 
 def device_tables(dtype, tables):
     """torch tables (any device) -> list of CUDA tensors in the library's layout."""
     out = []
     for t in tables:
-        if dtype == wl.INT8_ROWWISE:
+        if dtype in ROWWISE8:
             q, s, b = (x.cuda() for x in t)
             out.append(eb.ebag_pack_int8_rowwise(q, s, b))
         else:
@@ -31,7 +32,7 @@ def device_tables(dtype, tables):
 
 
 def oracle_tables(dtype, tables):
-    if dtype == wl.INT8_ROWWISE:
+    if dtype in ROWWISE8:
         return ([wl.raw_numpy(t[0]) for t in tables], [wl.raw_numpy(t[1]) for t in tables],
                 [wl.raw_numpy(t[2]) for t in tables])
     return [wl.raw_numpy(t) for t in tables], None, None
@@ -129,7 +130,7 @@ def sampled_check(w, jag, dev_tables_raw, gpu_out, bags_per_table, seed=0):
             uniq = np.zeros(1, np.int64)
         sel = torch.from_numpy(uniq).cuda()
         tab = dev_tables_raw[t]
-        if w.dtype == wl.INT8_ROWWISE:
+        if w.dtype in ROWWISE8:
             c_tables.append(wl.raw_numpy(tab[0].index_select(0, sel)))
             c_sc.append(wl.raw_numpy(tab[1].index_select(0, sel)))
             c_bi.append(wl.raw_numpy(tab[2].index_select(0, sel)))

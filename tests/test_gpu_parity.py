@@ -27,8 +27,11 @@ def _jagged_from_lengths(rng, lengths_per_table, rows):
 def _rand_tables(rng, dtype, rows, D, small_ints=False):
     tabs = []
     for r, d in zip(rows, D):
-        if dtype == wl.INT8_ROWWISE:
-            q = torch.from_numpy(rng.integers(-128, 128, size=(r, d)).astype(np.int8))
+        if dtype in (wl.INT8_ROWWISE, wl.UINT8_ROWWISE):
+            if dtype == wl.INT8_ROWWISE:
+                q = torch.from_numpy(rng.integers(-128, 128, size=(r, d)).astype(np.int8))
+            else:
+                q = torch.from_numpy(rng.integers(0, 256, size=(r, d)).astype(np.uint8))
             if small_ints:
                 s, b = torch.ones(r), torch.zeros(r)
             else:
@@ -107,6 +110,7 @@ def test_host_buffer_entry_point_with_malformed_offsets_falls_back():
     (wl.F16, [8, 24, 64, 128, 264, 520, 1032]),
     (wl.BF16, [8, 16, 72, 256, 512, 1032, 2056]),
     (wl.INT8_ROWWISE, [16, 48, 128, 512, 528, 1040, 2064]),
+    (wl.UINT8_ROWWISE, [16, 64, 128, 528, 2064]),
 ])
 @pytest.mark.parametrize("mode,weighted", [(wl.SUM, False), (wl.MEAN, False), (wl.SUM, True),
                                            (wl.MEAN, True)])
@@ -194,7 +198,7 @@ def test_single_bag_single_lookup():
 
 
 # ------------------------------------------------------------------ integer-exact cases, bit for bit
-@pytest.mark.parametrize("dtype", [wl.F32, wl.F16, wl.BF16, wl.INT8_ROWWISE])
+@pytest.mark.parametrize("dtype", [wl.F32, wl.F16, wl.BF16, wl.INT8_ROWWISE, wl.UINT8_ROWWISE])
 def test_integer_valued_tables_match_bit_for_bit(dtype):
     """Products and partial sums are integers below 2^24, so every summation order gives the same
     fp32 result: the GPU must equal the oracle exactly."""

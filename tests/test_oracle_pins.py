@@ -330,6 +330,31 @@ def test_bad_offsets_make_empty_bags_and_are_counted():
     assert r["n_bad_offsets"] == 1 and np.all(r["out32"][1] == 0)
 
 
+def test_uint8_rowwise_is_scale_times_unsigned_code_plus_bias():
+    """UINT8_ROWWISE: value = scale * u + bias with u the unsigned byte.  Pinned against the F32
+    path (pinned above) on the dequantised table, where the two must agree bit for bit: scale a
+    power of two and bias a small integer make scale*u + bias exact in fp32."""
+    rng = np.random.default_rng(33)
+    rows, D, B = 40, 16, 25
+    u = rng.integers(0, 256, size=(rows, D)).astype(np.uint8)
+    scale = (2.0 ** rng.integers(-3, 3, size=rows)).astype(np.float32)
+    bias = rng.integers(-5, 6, size=rows).astype(np.float32)
+    lengths = rng.integers(0, 7, size=B)
+    off = np.zeros(B + 1, np.int64)
+    np.cumsum(lengths, out=off[1:])
+    idx = rng.integers(0, rows, size=int(off[-1])).astype(np.int64)
+    w = rng.integers(-2, 3, size=idx.size).astype(np.float32)
+    deq = (scale[:, None] * u.astype(np.float32) + bias[:, None]).astype(np.float32)
+    for mode, ww in ((orc.SUM, None), (orc.SUM, w), (orc.MEAN, None)):
+        a = orc.forward([u], orc.UINT8_ROWWISE, idx, off, B, mode, weights=ww, scales=[scale], biases=[bias])
+        b = orc.forward([deq], orc.F32, idx, off, B, mode, weights=ww)
+        assert np.array_equal(a["out32"].view(np.uint32), b["out32"].view(np.uint32))
+    # and it differs from reading the same bytes as signed codes
+    u_sum = orc.forward([u], orc.UINT8_ROWWISE, idx, off, B, orc.SUM, scales=[scale], biases=[bias])
+    s8 = orc.forward([u.view(np.int8)], orc.INT8_ROWWISE, idx, off, B, orc.SUM, scales=[scale], biases=[bias])
+    assert not np.array_equal(s8["out32"], u_sum["out32"])
+
+
 def test_weighted_mean_divides_the_weighted_sum_by_the_lookup_count():
     """mean with per-sample weights = (sum of w*x) / L, L the number of lookups of the bag (the
     divisor is not the sum of the weights).  Pinned against the weighted sum, which has its own
