@@ -14,6 +14,7 @@ constexpr int kIlp = 8;              // values per thread in flight (8 x 4 B x 2
 // blockIdx.y is the feature.  "Below" is written !(x <= b) so that NaN lands in the last bin,
 // like the library routine the paper's pseudocode calls.  Short lists are counted linearly
 // (the vectorised counting the paper's kernel uses), long ones by a branch-free halving search.
+template <bool VEC>       // VEC: B is a multiple of 4 and both arrays are 16-byte aligned
 __global__ void __launch_bounds__(kThreads)
 mbdt_kernel(const float* __restrict__ values, int64_t B, const float* __restrict__ borders,
             const int64_t* __restrict__ border_offsets, const int64_t* __restrict__ out_offsets,
@@ -32,6 +33,58 @@ mbdt_kernel(const float* __restrict__ values, int64_t B, const float* __restrict
     const float* __restrict__ vf = values + (int64_t)f * B;
     int64_t* __restrict__ of = out + (int64_t)f * B;
     const int64_t stride = (int64_t)gridDim.x * kThreads;
+    // bin of one value
+    auto bin = [&](float x) -> int {
+        if (K <= kSmemBorders) {
+            int n = 0;
+            for (int j = 0; j < K; ++j) n += !(x <= sb[j]);
+            return n;
+        }
+        int lo = 0, hi = K;
+        const int steps = 32 - __clz(K);
+        for (int s = 0; s < steps; ++s) {
+            const int mid = (lo + hi) >> 1;
+            const float b = __ldg(bf + (mid < K ? mid : K - 1));
+            const bool active = lo < hi;
+            const bool right = !(x <= b);
+            lo = (active && right) ? mid + 1 : lo;
+            hi = (active && !right) ? mid : hi;
+        }
+        return lo;
+    };
+    if (VEC) {
+        // four consecutive values per thread and step: one 16-byte load, two 16-byte stores
+        const int64_t B4 = B >> 2;
+        const float4* __restrict__ v4 = reinterpret_cast<const float4*>(vf);
+        longlong2* __restrict__ o2 = reinterpret_cast<longlong2*>(of);
+        for (int64_t i = blockIdx.x * (int64_t)kThreads + threadIdx.x; i < B4; i += 2 * stride) {
+            const bool second = i + stride < B4;
+            const float4 a = __ldcs(v4 + i);
+            float4 c = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (second) c = __ldcs(v4 + i + stride);
+            const float x[8] = {a.x, a.y, a.z, a.w, c.x, c.y, c.z, c.w};
+            int n[8];
+            if (K <= kSmemBorders) {
+#pragma unroll
+                for (int k = 0; k < 8; ++k) n[k] = 0;
+                for (int j = 0; j < K; ++j) {
+                    const float b = sb[j];
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) n[k] += !(x[k] <= b);
+                }
+            } else {
+#pragma unroll
+                for (int k = 0; k < 8; ++k) n[k] = bin(x[k]);
+            }
+            __stcs(o2 + 2 * i, make_longlong2(n[0] + add, n[1] + add));
+            __stcs(o2 + 2 * i + 1, make_longlong2(n[2] + add, n[3] + add));
+            if (second) {
+                __stcs(o2 + 2 * (i + stride), make_longlong2(n[4] + add, n[5] + add));
+                __stcs(o2 + 2 * (i + stride) + 1, make_longlong2(n[6] + add, n[7] + add));
+            }
+        }
+        return;
+    }
     for (int64_t i = blockIdx.x * (int64_t)kThreads + threadIdx.x; i < B; i += kIlp * stride) {
         float x[kIlp];
         int n[kIlp];
@@ -46,26 +99,8 @@ mbdt_kernel(const float* __restrict__ values, int64_t B, const float* __restrict
                 for (int k = 0; k < kIlp; ++k) n[k] += !(x[k] <= b);
             }
         } else {
-            const int steps = 32 - __clz(K);
-            int lo[kIlp], hi[kIlp];
 #pragma unroll
-            for (int k = 0; k < kIlp; ++k) {
-                lo[k] = 0;
-                hi[k] = K;
-            }
-            for (int s = 0; s < steps; ++s) {
-#pragma unroll
-                for (int k = 0; k < kIlp; ++k) {
-                    const int mid = (lo[k] + hi[k]) >> 1;
-                    const float b = __ldg(bf + (mid < K ? mid : K - 1));
-                    const bool active = lo[k] < hi[k];
-                    const bool right = !(x[k] <= b);
-                    lo[k] = (active && right) ? mid + 1 : lo[k];
-                    hi[k] = (active && !right) ? mid : hi[k];
-                }
-            }
-#pragma unroll
-            for (int k = 0; k < kIlp; ++k) n[k] = lo[k];
+            for (int k = 0; k < kIlp; ++k) n[k] = bin(x[k]);
         }
 #pragma unroll
         for (int k = 0; k < kIlp; ++k)
@@ -85,7 +120,7 @@ extern "C" ebag_status ebag_mbdt(const float* values, int32_t F, int64_t B, cons
     int dev = 0, sms = 0, per_sm = 0;
     if (cudaGetDevice(&dev) != cudaSuccess ||
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
-        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, mbdt_kernel, kThreads, 0) != cudaSuccess) {
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, mbdt_kernel<true>, kThreads, 0) != cudaSuccess) {
         cudaGetLastError();
         return EBAG_ERR_CUDA;
     }
@@ -93,8 +128,13 @@ extern "C" ebag_status ebag_mbdt(const float* values, int32_t F, int64_t B, cons
     int64_t cap = (int64_t)sms * per_sm / F;
     if (cap < 1) cap = 1;
     if (bx > cap) bx = cap;
-    mbdt_kernel<<<dim3((unsigned)bx, (unsigned)F), kThreads, 0, (cudaStream_t)stream>>>(
-        values, B, borders, border_offsets, out_offsets, out);
+    const bool vec = (B & 3) == 0 && !((uintptr_t)values & 15u) && !((uintptr_t)out & 15u);
+    if (vec)
+        mbdt_kernel<true><<<dim3((unsigned)bx, (unsigned)F), kThreads, 0, (cudaStream_t)stream>>>(
+            values, B, borders, border_offsets, out_offsets, out);
+    else
+        mbdt_kernel<false><<<dim3((unsigned)bx, (unsigned)F), kThreads, 0, (cudaStream_t)stream>>>(
+            values, B, borders, border_offsets, out_offsets, out);
     if (cudaGetLastError() != cudaSuccess) return EBAG_ERR_CUDA;
     return EBAG_OK;
 }
