@@ -42,7 +42,8 @@ constexpr int kThreads = 256;            // 8 warps per CTA
 constexpr int kWarps = kThreads / 32;
 constexpr int kMaxItemBags = 32;         // an item's offsets live in one register per lane
 constexpr int kItemsPerWarp = 4;         // small calls: aim for at least this many items per warp
-constexpr float kSortedItemFactor = 4.0f; // item size multiplier for tables with several bags per warp
+constexpr float kSortedItemFactor = 8.0f; // item size multiplier for tables whose rows take one vector per lane
+constexpr float kSmallCallFactor = 4.0f;  // the same in a call so small that the items are shrunk
 constexpr uint32_t kInvalidRow = 0xFFFFFFFFu;
 
 struct TableMeta {       // per table, built at create, lives in device memory
@@ -747,7 +748,11 @@ ebag_fwd_kernel(const FwdParams p) {
         const int ng = 32 >> p.meta[t].g_log2;
         // bags that run side by side are matched by length inside an item: more bags per item,
         // better matches (measured: cfg 5 6.70 -> 5.75 ms, cfg 3 2.35 -> 2.12 ms)
-        const float want = (ng > 1 ? kSortedItemFactor * item_bytes : item_bytes) / bag_bytes[t];
+        // (also: fewer item start-ups, each of which leaves the warp's pipeline empty for a while;
+        // rows of two vectors per lane gather enough per bag and balance better with small items)
+        const float target = p.meta[t].V == 1 ? fminf(kSortedItemFactor * (float)p.item_bytes, kSmallCallFactor * spread)
+                                              : item_bytes;
+        const float want = target / bag_bytes[t];
         int ib = want >= (float)kMaxItemBags ? kMaxItemBags : (int)want;
         ib = (ib / ng) * ng;
         if (ib < ng) ib = ng;
