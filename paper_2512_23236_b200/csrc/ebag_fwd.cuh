@@ -44,6 +44,7 @@ constexpr int kMaxItemBags = 32;         // an item's offsets live in one regist
 constexpr int kItemsPerWarp = 4;         // small calls: aim for at least this many items per warp
 constexpr float kSortedItemFactor = 8.0f; // item size multiplier for tables whose rows take one vector per lane
 constexpr float kSmallCallFactor = 4.0f;  // the same in a call so small that the items are shrunk
+constexpr float kTailItemFactor = 2.0f;   // the same for the last tables of a call (1 / 2 / 4 measured: 2 is best)
 constexpr uint32_t kInvalidRow = 0xFFFFFFFFu;
 
 struct TableMeta {       // per table, built at create, lives in device memory
@@ -711,7 +712,7 @@ ebag_fwd_kernel(const FwdParams p) {
     int* item_base = smem_i;                                   // [T+1] first item of each table
     int* item_bags = smem_i + p.T + 1;                         // [T]   bags per item of each table
     float* bag_bytes = reinterpret_cast<float*>(item_bags);    // [T]   (first pass) bytes per bag
-    __shared__ float total_bytes;
+    __shared__ unsigned long long total_bytes_u;
     __shared__ uint4 stage_buf[kWarps * kWarpSmemVecs];      // per warp: 4 KB ring + the item's bags
     __shared__ float2 sb_buf[DT == DT_INT8 ? kWarps * kStages * kStageVecs * 8 : 1];
     int tid;
@@ -727,7 +728,9 @@ ebag_fwd_kernel(const FwdParams p) {
     asm volatile("griddepcontrol.launch_dependents;");
 
     // ---- size the items of every table from its share of the offsets prefix sum
-    if (tid == 0) total_bytes = 0.0f;
+    // (summed as integers: every CTA must arrive at the same item tables, bit for bit, and a
+    // floating-point sum would depend on the order of the additions)
+    if (tid == 0) total_bytes_u = 0ull;
     __syncthreads();
     for (int t = tid; t < p.T; t += kThreads) {
         const int64_t n0 = p.offsets[(int64_t)t * p.off_stride];
@@ -737,12 +740,26 @@ ebag_fwd_kernel(const FwdParams p) {
         if (nt > p.n_indices) nt = p.n_indices;
         const float bytes = (float)nt * (float)p.meta[t].stride;
         bag_bytes[t] = fmaxf(bytes / (float)p.B, 1.0f);
-        atomicAdd(&total_bytes, bytes);
+        atomicAdd(&total_bytes_u, (unsigned long long)nt * (unsigned long long)p.meta[t].stride);
     }
     __syncthreads();
+    const float total_bytes = (float)total_bytes_u;
     // small calls: shrink the items so that every warp of the grid gets a few of them
     const float spread = total_bytes / (float)(gridDim.x * kWarps * kItemsPerWarp);
     const float item_bytes = fminf((float)p.item_bytes, spread);
+    const float big_item = fminf(kSortedItemFactor * (float)p.item_bytes, kSmallCallFactor * spread);
+    // The queue hands items out in table order, so the last tables decide how long the slowest
+    // warp runs after the others are done: the tables that make up the last big item's worth of
+    // work per warp get plain (small) items.  Marked by a negative bag size.
+    if (tid == 0) {
+        const float budget = big_item * (float)(gridDim.x * kWarps);
+        float after = 0.0f;
+        for (int t = p.T - 1; t >= 0; --t) {
+            after += bag_bytes[t] * (float)p.B;
+            if (after > budget) break;
+            bag_bytes[t] = -bag_bytes[t];
+        }
+    }
     __syncthreads();
     for (int t = tid; t < p.T; t += kThreads) {
         const int ng = 32 >> p.meta[t].g_log2;
@@ -750,9 +767,9 @@ ebag_fwd_kernel(const FwdParams p) {
         // better matches (measured: cfg 5 6.70 -> 5.75 ms, cfg 3 2.35 -> 2.12 ms)
         // (also: fewer item start-ups, each of which leaves the warp's pipeline empty for a while;
         // rows of two vectors per lane gather enough per bag and balance better with small items)
-        const float target = p.meta[t].V == 1 ? fminf(kSortedItemFactor * (float)p.item_bytes, kSmallCallFactor * spread)
-                                              : item_bytes;
-        const float want = target / bag_bytes[t];
+        const bool tail = bag_bytes[t] < 0.0f;
+        const float target = p.meta[t].V != 1 ? item_bytes : (tail ? fminf(kTailItemFactor * item_bytes, big_item) : big_item);
+        const float want = target / fabsf(bag_bytes[t]);
         int ib = want >= (float)kMaxItemBags ? kMaxItemBags : (int)want;
         ib = (ib / ng) * ng;
         if (ib < ng) ib = ng;
