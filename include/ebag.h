@@ -306,6 +306,11 @@ ebag_status ebag_forward_noalloc(int32_t T, const int64_t* rows, const int32_t* 
  *   "item_bytes"   target bytes of gathered rows per work item (default 32768)
  *   "ctas_per_sm"  resident CTAs per SM of the persistent grid (default: occupancy limit)
  *   "host_chunks"  bag ranges per ebag_forward_host call, 1..16 (default 0: from the size)
+ *   "out_dtype"    element type of `out` in ebag_forward, ebag_forward_i32 and
+ *                  ebag_forward_mapid: EBAG_F32 (default), EBAG_F16 or EBAG_BF16.  Sums are still
+ *                  accumulated in fp32 and rounded to nearest-even once, when the bag is written;
+ *                  `out` then points at [B, sum(D)] 16-bit elements (same alignment rule).
+ *                  ebag_forward_host returns UNSUPPORTED unless it is EBAG_F32.
  *   "split_bytes"  a bag whose rows add up to this many bytes or more (rows narrower than 256
  *                  bytes count as 256) is pooled in parts by many warps instead of by one, the
  *                  partial sums added in lookup order by a second, short kernel launched after

@@ -270,6 +270,13 @@ class TBE:
 
     def set_param(self, name: str, value: int):
         _check(lib().ebag_set_param(self._h, name.encode(), int(value)), "ebag_set_param")
+        if name == "out_dtype":
+            self._out_dtype = int(value)
+
+    def _out_torch_dtype(self):
+        import torch
+        return {EBAG_F32: torch.float32, EBAG_F16: torch.float16,
+                EBAG_BF16: torch.bfloat16}[getattr(self, "_out_dtype", EBAG_F32)]
 
     def launch_count(self) -> int:
         return int(lib().ebag_launch_count(self._h))
@@ -293,7 +300,9 @@ class TBE:
         ``indices`` may be int64 or int32 (the matching entry point is called)."""
         import torch
         if out is None:
-            out = torch.empty((B, self.sumD), dtype=torch.float32, device=indices.device)
+            out = torch.empty((B, self.sumD), dtype=self._out_torch_dtype(), device=indices.device)
+        elif out.dtype != self._out_torch_dtype():
+            raise TypeError("out must have the handle's out_dtype")
         if not hasattr(self, "_d_arr"):
             self._d_arr = (ctypes.c_int32 * self.T)(*self.D)
             self._d_ptr = ctypes.cast(self._d_arr, _vp)
@@ -330,7 +339,7 @@ class TBE:
         """Raw ids in: table t maps them through the sorted device tensor mappings[t] first."""
         import torch
         if out is None:
-            out = torch.empty((B, self.sumD), dtype=torch.float32, device=values.device)
+            out = torch.empty((B, self.sumD), dtype=self._out_torch_dtype(), device=values.device)
         ebag_forward_mapid(self._h, [t.data_ptr() for t in tables], self.D, _ptr(values),
                            int(values.numel()), _ptr(offsets), _ptr(per_sample_weights),
                            [m.data_ptr() for m in mappings], [int(m.numel()) for m in mappings], B,

@@ -66,6 +66,7 @@ struct ebag_tbe {
     void* d_long = nullptr;
     LongParams lg = {};
     uint32_t max_stride = 0;
+    int out_dtype = EBAG_F32;                      // element type of `out` (F32, F16 or BF16)
     uint32_t split_bytes = 65536;                  // a bag gathering this much or more is split; 0: never
     int64_t launches = 0;
     std::string cuda_error;
@@ -222,7 +223,10 @@ ebag_status forward_device(ebag_tbe* h, const void* const* tables, const int64_t
     p.indices = indices;
     p.offsets = offsets + b0;
     p.weights = weights;
-    p.out = out + b0 * (int64_t)h->sumD;
+    p.out16 = h->out_dtype == EBAG_F16 ? 1 : (h->out_dtype == EBAG_BF16 ? 2 : 0);
+    // (a 16-bit `out` is addressed in elements inside the kernel; the range offset is applied here in bytes)
+    p.out = reinterpret_cast<float*>(reinterpret_cast<char*>(out) +
+                                     b0 * (int64_t)h->sumD * (p.out16 ? 2 : 4));
     p.queue = h->d_queue;
     p.status = h->d_status;
     p.mappings = reinterpret_cast<const int64_t* const*>(d_tables + h->T);
@@ -638,6 +642,7 @@ ebag_status ebag_forward_host(ebag_tbe* h, const void* const* tables, const int3
     ebag_status st = check_forward_args(h, tables, D, indices, n_indices, offsets,
                                         per_sample_weights, B, mode, out);
     if (st != EBAG_OK) return st;
+    if (h->out_dtype != EBAG_F32) return EBAG_ERR_UNSUPPORTED;      // the host path stages and returns fp32
     if (B == 0) return EBAG_OK;
     DeviceGuard guard(h->device);
     if (!guard.ok) return EBAG_ERR_CUDA;
@@ -774,6 +779,11 @@ ebag_status ebag_set_param(ebag_tbe* h, const char* name, int64_t value) {
     if (std::strcmp(name, "split_bytes") == 0) {
         if (value != 0 && (value < 1024 || value > (1ll << 31) - 1)) return EBAG_ERR_INVALID_ARG;
         h->split_bytes = (uint32_t)value;
+        return EBAG_OK;
+    }
+    if (std::strcmp(name, "out_dtype") == 0) {
+        if (value != EBAG_F32 && value != EBAG_F16 && value != EBAG_BF16) return EBAG_ERR_INVALID_ARG;
+        h->out_dtype = (int)value;
         return EBAG_OK;
     }
     if (std::strcmp(name, "host_chunks") == 0) {

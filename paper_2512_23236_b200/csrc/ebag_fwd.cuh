@@ -115,7 +115,7 @@ struct FwdParams {
     const int64_t* indices;      // int32 ids instead when idx32 is set
     const int64_t* offsets;
     const float* weights;
-    float* out;
+    float* out;                  // [B, sumD] fp32, or 16-bit elements when out16 is set
     Queue* queue;
     Status* status;
     const int64_t* const* mappings;   // MapId variant: device [T] sorted id lists (else unused)
@@ -128,6 +128,7 @@ struct FwdParams {
     int32_t sumD;
     int32_t mean;                // 1: divide by the bag length
     int32_t idx32;               // 1: `indices` holds 32-bit ids
+    int32_t out16;               // 0: fp32 output; 1: fp16; 2: bf16 (rounded to nearest-even once, at the store)
     float code_zero;             // rowwise 8-bit tables: the stored byte that means code 0 (128 signed, 0 unsigned)
     uint32_t item_bytes;
     LongParams lg;
@@ -139,6 +140,13 @@ __device__ __forceinline__ int64_t ld_stream_i64(const int64_t* p) {
     return __ldcs(reinterpret_cast<const long long*>(p));
 }
 __device__ __forceinline__ float ld_stream_f32(const float* p) { return __ldcs(p); }
+// two fp32 values rounded to nearest-even into one 32-bit word of fp16 (kind 1) or bf16 (kind 2)
+__device__ __forceinline__ uint32_t pack16(float lo, float hi, int kind) {
+    uint32_t r;
+    if (kind == 1) asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    else asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
 __device__ __forceinline__ void st_stream16(float* p, float a, float b, float c, float d) {
     __stcs(reinterpret_cast<float4*>(p), make_float4(a, b, c, d));
 }
@@ -639,9 +647,26 @@ __device__ __forceinline__ void process_item(const FwdParams& p, const TableMeta
                     }
                     acc[v][a] = x;
                 }
+                if (PART || p.out16 == 0) {
 #pragma unroll
-                for (int a = 0; a < NACC / 2; a += 2)
-                    st_stream16(o + 2 * a, acc[v][a].x, acc[v][a].y, acc[v][a + 1].x, acc[v][a + 1].y);
+                    for (int a = 0; a < NACC / 2; a += 2)
+                        st_stream16(o + 2 * a, acc[v][a].x, acc[v][a].y, acc[v][a + 1].x, acc[v][a + 1].y);
+                } else {
+                    // 16-bit output: the same elements, half the bytes
+                    uint32_t* o16 = reinterpret_cast<uint32_t*>(p.out) +
+                                    (((bag0 + orig) * (int64_t)p.sumD + m.D_off +
+                                      (int64_t)(vec0 + v * G + lig) * NACC) >> 1);
+                    uint32_t wd[NACC / 2];
+#pragma unroll
+                    for (int a = 0; a < NACC / 2; ++a) wd[a] = pack16(acc[v][a].x, acc[v][a].y, p.out16);
+                    if constexpr (NACC == 4) {
+                        __stcs(reinterpret_cast<uint2*>(o16), make_uint2(wd[0], wd[1]));
+                    } else {
+#pragma unroll
+                        for (int a = 0; a < NACC / 2; a += 4)
+                            __stcs(reinterpret_cast<uint4*>(o16 + a), make_uint4(wd[a], wd[a + 1], wd[a + 2], wd[a + 3]));
+                    }
+                }
             }
         }
         acc_bias = 0.0f;
@@ -992,7 +1017,14 @@ ebag_parts_kernel(const FwdParams p) {
                     acc.x = __fdiv_rn(acc.x, fl); acc.y = __fdiv_rn(acc.y, fl);
                     acc.z = __fdiv_rn(acc.z, fl); acc.w = __fdiv_rn(acc.w, fl);
                 }
-                st_stream16(orow + c, acc.x, acc.y, acc.z, acc.w);
+                if (p.out16 == 0) {
+                    st_stream16(orow + c, acc.x, acc.y, acc.z, acc.w);
+                } else {
+                    uint32_t* o16 = reinterpret_cast<uint32_t*>(p.out) +
+                                    ((rec.bag * (int64_t)p.sumD + m.D_off + c) >> 1);
+                    __stcs(reinterpret_cast<uint2*>(o16),
+                           make_uint2(pack16(acc.x, acc.y, p.out16), pack16(acc.z, acc.w, p.out16)));
+                }
             }
             if (lane == 0) p.lg.arrivals[bi] = 0;       // ready for the next launch
         }

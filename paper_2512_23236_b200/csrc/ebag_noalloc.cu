@@ -201,6 +201,7 @@ extern "C" ebag_status ebag_forward_noalloc(int32_t T, const int64_t* rows, cons
     p.sumD = (int32_t)d_off;
     p.mean = mode == EBAG_MEAN ? 1 : 0;
     p.idx32 = 0;
+    p.out16 = 0;
     p.code_zero = dtype == EBAG_UINT8_ROWWISE ? 0.0f : 128.0f;
     p.item_bytes = 32768;
     p.lg = LongParams{};                     // no room for partial sums here: bags are not split

@@ -154,6 +154,79 @@ def test_int32_ids(dtype, Ds, mode, weighted):
     assert np.array_equal(gpu32.view(np.uint32), gpu64.view(np.uint32))
 
 
+# ------------------------------------------------------------------ 16-bit output
+def _round_bf16(x32):
+    """fp32 array rounded to nearest-even bf16, returned as fp32."""
+    b = x32.astype(np.float32).view(np.uint32).astype(np.uint64)
+    b = (b + 0x7FFF + ((b >> 16) & 1)) & 0xFFFF0000
+    return b.astype(np.uint32).view(np.float32)
+
+
+@pytest.mark.parametrize("dtype,Ds", [(wl.F32, [4, 64, 260]), (wl.BF16, [8, 128, 1032]),
+                                      (wl.INT8_ROWWISE, [16, 128, 528])])
+@pytest.mark.parametrize("out_dtype", [eb.EBAG_F16, eb.EBAG_BF16])
+@pytest.mark.parametrize("mode,weighted", [(wl.SUM, False), (wl.MEAN, True)])
+def test_sixteen_bit_output(dtype, Ds, out_dtype, mode, weighted):
+    """out_dtype fp16 / bf16: fp32 sums rounded once at the store.  The value must lie within the
+    usual bar of the oracle plus one rounding of the output type (2^-11 relative for fp16, 2^-8
+    for bf16), it must be EXACTLY the rounding of some fp32 value within the bar (checked on the
+    integer-valued case below), empty bags are +0, and a long bag takes the parts path."""
+    rng = np.random.default_rng(91 + dtype)
+    T, B = len(Ds), 70
+    rows = [int(rng.integers(20, 400)) for _ in Ds]
+    lens = [rng.integers(0, 40, size=B) for _ in Ds]
+    lens[0][5] = 2000                                     # pooled in parts
+    idx, off, lengths = _jagged_from_lengths(rng, lens, rows)
+    w = (rng.random(idx.shape[0]).astype(np.float32) - 0.25) if weighted else None
+    tabs = _rand_tables(rng, dtype, rows, Ds)
+    dev = pu.device_tables(dtype, tabs)
+    ot, sc, bi = pu.oracle_tables(dtype, tabs)
+    ref = orc.forward(ot, dtype, idx, off, B, mode, weights=w, scales=sc, biases=bi)
+    tbe = eb.TBE(rows, Ds, dtype, device=torch.cuda.current_device())
+    try:
+        tbe.set_param("out_dtype", out_dtype)
+        out = tbe.forward(dev, torch.from_numpy(idx).cuda(), torch.from_numpy(off).cuda(), B, mode,
+                          None if w is None else torch.from_numpy(w).cuda())
+        assert out.dtype == (torch.float16 if out_dtype == eb.EBAG_F16 else torch.bfloat16)
+        assert tbe.last_status() == (0, 0, 0)
+        got = out.float().cpu().numpy().astype(np.float64)
+    finally:
+        tbe.close()
+    rel = 2.0 ** -11 if out_dtype == eb.EBAG_F16 else 2.0 ** -8
+    err = np.abs(got - ref["out64"])
+    bar = pu.TOL[dtype] * ref["S"] + rel * np.abs(ref["out64"]) + 2.0 ** -24
+    assert np.all(err <= bar), f"{(err > bar).sum()} elements beyond the bar"
+    col = 0
+    for t in range(T):
+        empty = lengths[t * B:(t + 1) * B] == 0
+        assert np.all(got[:, col:col + Ds[t]][empty] == 0.0)
+        col += Ds[t]
+
+
+@pytest.mark.parametrize("out_dtype", [eb.EBAG_F16, eb.EBAG_BF16])
+def test_sixteen_bit_output_rounds_to_nearest_even(out_dtype):
+    # integer-valued sums are exact in fp32, so the 16-bit result must be exactly their rounding
+    rng = np.random.default_rng(17)
+    rows, D, B = [500], [64], 300
+    lens = [rng.integers(0, 80, size=B)]
+    idx, off, lengths = _jagged_from_lengths(rng, lens, rows)
+    tabs = _rand_tables(rng, wl.F32, rows, D, small_ints=True)
+    w = np.full(idx.shape[0], 37.0, np.float32)            # sums in the thousands: they need rounding
+    ref = orc.forward([wl.raw_numpy(tabs[0])], wl.F32, idx, off, B, wl.SUM, weights=w)
+    tbe = eb.TBE(rows, D, wl.F32, device=torch.cuda.current_device())
+    try:
+        tbe.set_param("out_dtype", out_dtype)
+        out = tbe.forward(pu.device_tables(wl.F32, tabs), torch.from_numpy(idx).cuda(),
+                          torch.from_numpy(off).cuda(), B, wl.SUM, torch.from_numpy(w).cuda())
+        got = out.float().cpu().numpy()
+    finally:
+        tbe.close()
+    want = ref["out32"].astype(np.float16).astype(np.float32) if out_dtype == eb.EBAG_F16 \
+        else _round_bf16(ref["out32"])
+    assert np.abs(ref["out32"]).max() > 2048               # values that do need rounding occur
+    assert np.array_equal(got.view(np.uint32), want.view(np.uint32))
+
+
 # ------------------------------------------------------------------ degenerate and extreme bags
 @pytest.mark.parametrize("dtype,D", [(wl.F32, 256), (wl.BF16, 64), (wl.INT8_ROWWISE, 128)])
 def test_planted_bag_lengths(dtype, D):
