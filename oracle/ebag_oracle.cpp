@@ -14,7 +14,8 @@
 //   for every table t and bag b (bag id g = t*B + b):
 //       s = offsets[g], e = offsets[g+1], L = e - s
 //       out[b, Doff[t] + d] = pool_{i = s .. e-1} w_i * value(t, indices[i], d)
-//   pool = sum, or sum / L (mean; an empty bag stays +0.0f), w_i = weights[i] or 1.  With weights
+//   pool = sum, or sum / L (mean; an empty bag stays +0.0f), or max (the largest value among the
+//   lookups that were not skipped; +0.0f if there is none; no weights), w_i = weights[i] or 1.  With weights
 //   the mean still divides by the lookup count L (not by the sum of the weights).
 //   value() widens the stored element to fp32: fp32 as is, fp16/bf16 exactly, rowwise int8 as
 //   scale[row] * (float)q + bias[row] (one fp32 multiply, then one fp32 add).
@@ -48,7 +49,7 @@
 namespace {
 
 enum { DT_F32 = 0, DT_F16 = 1, DT_BF16 = 2, DT_INT8_ROWWISE = 3, DT_UINT8_ROWWISE = 4 };
-enum { MODE_SUM = 0, MODE_MEAN = 1 };
+enum { MODE_SUM = 0, MODE_MEAN = 1, MODE_MAX = 2 };
 
 inline float bits_to_float(uint32_t u) {
     float f;
@@ -100,7 +101,8 @@ int ebag_oracle_forward(int32_t T, const int64_t* rows, const int32_t* D, int32_
                         int64_t* n_bad_offsets, int32_t nthreads) {
     if (T <= 0 || B < 0 || !rows || !D || !tables || !offsets || !out32) return 1;
     if (dtype < DT_F32 || dtype > DT_UINT8_ROWWISE) return 1;
-    if (mode != MODE_SUM && mode != MODE_MEAN) return 1;
+    if (mode != MODE_SUM && mode != MODE_MEAN && mode != MODE_MAX) return 1;
+    if (mode == MODE_MAX && weights) return 1;
     if ((dtype == DT_INT8_ROWWISE || dtype == DT_UINT8_ROWWISE) && (!scales || !biases)) return 1;
     std::vector<int64_t> Doff(T + 1, 0);
     for (int32_t t = 0; t < T; ++t) {
@@ -134,6 +136,7 @@ int ebag_oracle_forward(int32_t T, const int64_t* rows, const int32_t* D, int32_
             acc32.assign(Dt, 0.0f);
             acc64.assign(Dt, 0.0);
             accS.assign(Dt, 0.0);
+            int64_t seen = 0;                              // lookups that were not skipped
             for (int64_t i = s; i < e; ++i) {              // ascending, sequential
                 const int64_t r = indices[i];
                 if (r < 0 || r >= rows[t]) { ++oob_total; continue; }
@@ -153,12 +156,21 @@ int ebag_oracle_forward(int32_t T, const int64_t* rows, const int32_t* D, int32_
                             x = sq + biases[t][r];                  // rounded sum
                         }
                     }
+                    if (mode == MODE_MAX) {
+                        // max pooling: the largest value among the bag's (valid) lookups; the
+                        // scale the tolerance refers to is the largest magnitude seen
+                        if (seen == 0 || x > acc32[d]) acc32[d] = x;
+                        if (seen == 0 || (double)x > acc64[d]) acc64[d] = (double)x;
+                        accS[d] = std::fmax(accS[d], std::fabs((double)x));
+                        continue;
+                    }
                     const float p = w * x;                          // rounded product
                     acc32[d] = acc32[d] + p;                        // rounded sum
                     const double pd = (double)w * (double)x;
                     acc64[d] += pd;
                     accS[d] += std::fabs(pd);
                 }
+                ++seen;
             }
             float* o32 = out32 + b * sumD + Doff[t];
             double* o64 = out64 ? out64 + b * sumD + Doff[t] : nullptr;

@@ -18,7 +18,7 @@ _SRC = os.path.join(_HERE, "ebag_oracle.cpp")
 _LIB = os.path.join(_HERE, "libebag_oracle.so")
 
 F32, F16, BF16, INT8_ROWWISE, UINT8_ROWWISE = 0, 1, 2, 3, 4
-SUM, MEAN = 0, 1
+SUM, MEAN, MAX = 0, 1, 2
 
 _lib = None
 

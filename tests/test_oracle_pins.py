@@ -355,6 +355,40 @@ def test_uint8_rowwise_is_scale_times_unsigned_code_plus_bias():
     assert not np.array_equal(s8["out32"], u_sum["out32"])
 
 
+@pytest.mark.parametrize("dtype", [orc.F32, orc.BF16, orc.INT8_ROWWISE])
+def test_max_pooling_against_numpy(dtype):
+    """MAX: element-wise maximum over the looked-up rows, by brute force with numpy; skipped ids
+    take no part, a bag with no valid lookup is +0, weights are refused."""
+    rng = np.random.default_rng(55 + dtype)
+    rows, D, B = 60, 12, 50
+    kw = {}
+    if dtype == orc.F32:
+        tab = rng.standard_normal((rows, D)).astype(np.float32)
+        val = tab
+    elif dtype == orc.BF16:
+        f = rng.standard_normal((rows, D)).astype(np.float32)
+        tab = (f.view(np.uint32) >> 16).astype(np.uint16)
+        val = (tab.astype(np.uint32) << 16).view(np.float32)
+    else:
+        tab = rng.integers(-128, 128, size=(rows, D)).astype(np.int8)
+        sc = rng.uniform(0.5, 2.0, rows).astype(np.float32)
+        bi = rng.normal(0, 1, rows).astype(np.float32)
+        kw = dict(scales=[sc], biases=[bi])
+        val = (sc[:, None] * tab.astype(np.float32)).astype(np.float32) + bi[:, None]
+    lengths = rng.integers(0, 9, size=B)
+    off = np.zeros(B + 1, np.int64)
+    np.cumsum(lengths, out=off[1:])
+    idx = rng.integers(0, rows, size=int(off[-1])).astype(np.int64)
+    idx[rng.random(idx.size) < 0.1] = -1                  # skipped
+    r = orc.forward([tab], dtype, idx, off, B, orc.MAX, **kw)
+    for b in range(B):
+        ids = [i for i in idx[off[b]:off[b + 1]] if 0 <= i < rows]
+        want = np.max(val[ids], axis=0) if ids else np.zeros(D, np.float32)
+        assert np.array_equal(r["out32"][b], want.astype(np.float32)), b
+    with pytest.raises(ValueError):
+        orc.forward([tab], dtype, idx, off, B, orc.MAX, weights=np.ones(idx.size, np.float32), **kw)
+
+
 def test_weighted_mean_divides_the_weighted_sum_by_the_lookup_count():
     """mean with per-sample weights = (sum of w*x) / L, L the number of lookups of the bag (the
     divisor is not the sum of the weights).  Pinned against the weighted sum, which has its own
