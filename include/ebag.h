@@ -52,8 +52,11 @@ typedef enum {
 typedef enum { EBAG_F32 = 0, EBAG_F16 = 1, EBAG_BF16 = 2, EBAG_INT8_ROWWISE = 3,
                EBAG_UINT8_ROWWISE = 4 } ebag_dtype;
 
-/* weighted sum = EBAG_SUM with per_sample_weights != NULL */
-typedef enum { EBAG_SUM = 0, EBAG_MEAN = 1 } ebag_mode;
+/* weighted sum = EBAG_SUM with per_sample_weights != NULL.  EBAG_MAX: element-wise maximum over
+ * the bag's lookups (ids that are skipped take no part; a bag with no valid lookup gives +0.0f);
+ * no weights, not for ebag_forward_mapid nor ebag_forward_noalloc (UNSUPPORTED), long bags are
+ * not split.  A maximum is exact, so EBAG_MAX results do not depend on the order of the lookups. */
+typedef enum { EBAG_SUM = 0, EBAG_MEAN = 1, EBAG_MAX = 2 } ebag_mode;
 
 #define EBAG_MAX_TABLES 2048
 

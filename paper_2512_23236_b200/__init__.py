@@ -13,7 +13,7 @@ import os
 from typing import List, Optional, Sequence
 
 EBAG_F32, EBAG_F16, EBAG_BF16, EBAG_INT8_ROWWISE, EBAG_UINT8_ROWWISE = 0, 1, 2, 3, 4
-EBAG_SUM, EBAG_MEAN = 0, 1
+EBAG_SUM, EBAG_MEAN, EBAG_MAX = 0, 1, 2
 EBAG_OK, EBAG_ERR_INVALID_ARG, EBAG_ERR_UNSUPPORTED, EBAG_ERR_CUDA = 0, 1, 2, 3
 EBAG_ERR_INDEX_OOB, EBAG_ERR_BAD_OFFSETS = 4, 5
 EBAG_NOALLOC_MAX_TABLES = 64

@@ -137,6 +137,15 @@ cudaError_t launch_fwd(int dtype, const FwdParams& p, bool w, bool mapid, int gr
     }
 }
 
+cudaError_t launch_fwdmax(int dtype, const FwdParams& p, int grid, size_t smem, cudaStream_t s) {
+    switch (dtype) {
+        case EBAG_F32: return launch_fwdmax_f32(p, grid, smem, s);
+        case EBAG_F16: return launch_fwdmax_f16(p, grid, smem, s);
+        case EBAG_BF16: return launch_fwdmax_bf16(p, grid, smem, s);
+        default: return launch_fwdmax_int8(p, grid, smem, s);
+    }
+}
+
 cudaError_t launch_parts(int dtype, const FwdParams& p, bool w, bool mapid, int grid, cudaStream_t s) {
     switch (dtype) {
         case EBAG_F32: return launch_parts_f32(p, w, mapid, grid, s);
@@ -160,7 +169,8 @@ ebag_status check_forward_args(ebag_tbe* h, const void* const* tables, const int
                                const int64_t* indices, int64_t n_indices, const int64_t* offsets,
                                const float* weights, int64_t B, ebag_mode mode, float* out) {
     if (!h || !tables || !D || !offsets || B < 0 || n_indices < 0) return EBAG_ERR_INVALID_ARG;
-    if (mode != EBAG_SUM && mode != EBAG_MEAN) return EBAG_ERR_INVALID_ARG;
+    if (mode != EBAG_SUM && mode != EBAG_MEAN && mode != EBAG_MAX) return EBAG_ERR_INVALID_ARG;
+    if (mode == EBAG_MAX && weights) return EBAG_ERR_UNSUPPORTED;
     if (n_indices > 0 && !indices) return EBAG_ERR_INVALID_ARG;
     if (B > 0 && !out) return EBAG_ERR_INVALID_ARG;
     if ((int64_t)h->T * B >= (1ll << 31)) return EBAG_ERR_UNSUPPORTED;
@@ -262,6 +272,13 @@ ebag_status forward_device(ebag_tbe* h, const void* const* tables, const int64_t
     int per_sm = h->occupancy[mapid ? 1 : 0][w ? 1 : 0];
     if (h->ctas_per_sm > 0 && h->ctas_per_sm < per_sm) per_sm = h->ctas_per_sm;
     const int grid = h->num_sms * per_sm;
+    if (mode == EBAG_MAX) {                        // its own kernel; bags are never split
+        if (mapid) return EBAG_ERR_UNSUPPORTED;
+        p.lg.ctl = nullptr;
+        EBAG_CUDA(h, launch_fwdmax(h->dtype, p, grid, fwd_smem_bytes(h->T), stream));
+        ++h->launches;
+        return EBAG_OK;
+    }
     EBAG_CUDA(h, launch_fwd(h->dtype, p, w, mapid, grid, fwd_smem_bytes(h->T), stream));
     ++h->launches;
     if (p.lg.ctl) {

@@ -267,6 +267,45 @@ __device__ __forceinline__ void accumulate(float2* acc, const uint4& d, float w)
 constexpr float kInt8Up = 0x1p64f;       // weight * scale travels as weight * scale * 2^64
 constexpr float kInt8Down = 0x1p69f;     // 2^(133 - 64)
 
+// acc[0..kAcc) = max(acc, widen(d))      (max pooling; rowwise 8-bit: scale * (code - zero) + bias,
+// product and sum rounded separately, as the definition is written)
+template <int DT>
+__device__ __forceinline__ void accumulate_max(float2* acc, const uint4& d, float scale, float bias,
+                                               float code_zero) {
+    const uint32_t r[4] = {d.x, d.y, d.z, d.w};
+    if constexpr (DT == DT_F32) {
+        acc[0].x = fmaxf(acc[0].x, __uint_as_float(r[0]));
+        acc[0].y = fmaxf(acc[0].y, __uint_as_float(r[1]));
+        acc[1].x = fmaxf(acc[1].x, __uint_as_float(r[2]));
+        acc[1].y = fmaxf(acc[1].y, __uint_as_float(r[3]));
+    } else if constexpr (DT == DT_BF16) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            acc[i].x = fmaxf(acc[i].x, __uint_as_float(r[i] << 16));
+            acc[i].y = fmaxf(acc[i].y, __uint_as_float(r[i] & 0xffff0000u));
+        }
+    } else if constexpr (DT == DT_F16) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&r[i]));
+            acc[i].x = fmaxf(acc[i].x, f.x);
+            acc[i].y = fmaxf(acc[i].y, f.y);
+        }
+    } else {
+        const float zero = 8388608.0f + code_zero;       // 2^23 + the byte that means code 0
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const float q = __uint_as_float(__byte_perm(r[i], 0x4B000000u, 0x7440 + k)) - zero;   // exact
+                const float x = __fadd_rn(__fmul_rn(scale, q), bias);
+                float& a = (k & 1) ? acc[2 * i + k / 2].y : acc[2 * i + k / 2].x;
+                a = fmaxf(a, x);
+            }
+        }
+    }
+}
+
 // Sort 32 keys, one per lane, in descending order (bitonic network, 15 exchange steps).
 __device__ __forceinline__ uint32_t warp_sort_desc(uint32_t v, int lane) {
 #pragma unroll
@@ -380,9 +419,10 @@ __device__ __forceinline__ void load_bag_range(const FwdParams& p, int64_t g0, i
 
 // PART: the "item" is one part of a long bag (`pa`): its lookups are shared out among the row
 // groups as if they were NG bags, and the rows of sums go to the part's slot, never divided.
+// POOL: 0 sums (sum, mean, weighted), 1 takes the element-wise maximum.
 // `skip` (forward kernel, splitting on): bit i set = bag i of the item is pooled elsewhere; the
 // call for the first column tile of an item works it out, the calls for the other tiles reuse it.
-template <int DT, bool WEIGHTED, bool MAPID, int V, bool PART = false>
+template <int DT, bool WEIGHTED, bool MAPID, int V, bool PART = false, int POOL = 0>
 __device__ __forceinline__ void process_item(const FwdParams& p, const TableMeta& m,
                                                    const char* __restrict__ tbase, int t,
                                                    int64_t bag0, int cnt, int vec0, int lane,
@@ -574,26 +614,31 @@ __device__ __forceinline__ void process_item(const FwdParams& p, const TableMeta
     };
     float2 acc[V][NACC / 2];                         // pairs: two fp32 operations per instruction
     float acc_bias = 0.0f;
+    const float acc0 = POOL == 1 ? __int_as_float(0xff800000) : 0.0f;     // -inf for max pooling
 #pragma unroll
     for (int v = 0; v < V; ++v)
 #pragma unroll
-        for (int a = 0; a < NACC / 2; ++a) acc[v][a] = make_float2(0.0f, 0.0f);
+        for (int a = 0; a < NACC / 2; ++a) acc[v][a] = make_float2(acc0, acc0);
     auto consume = [&](const IdChunk& c, int j0, int st) {
         if (c.clean && j0 + CR <= c.nmin) {
 #pragma unroll
             for (int u = 0; u < CR; ++u) {
                 float wu = WEIGHTED ? __shfl_sync(0xffffffffu, c.w, j0 + u, G) : 1.0f;
+                float2 sb = make_float2(1.0f, 0.0f);
                 if (DT == DT_INT8) {
-                    const float2 sb = lds64f(my_sb_s + (st * kStageVecs + u) * 64);
-                    acc_bias = fmaf(wu, sb.y, acc_bias);
-                    wu *= sb.x;
-                    acc_bias = fmaf(wu, -p.code_zero, acc_bias);
-                    wu *= kInt8Up;
+                    sb = lds64f(my_sb_s + (st * kStageVecs + u) * 64);
+                    if (POOL == 0) {
+                        acc_bias = fmaf(wu, sb.y, acc_bias);
+                        wu *= sb.x;
+                        acc_bias = fmaf(wu, -p.code_zero, acc_bias);
+                        wu *= kInt8Up;
+                    }
                 }
 #pragma unroll
                 for (int v = 0; v < V; ++v) {
                     const uint4 d = lds128(my_rows_s + (st * kStageVecs + u * V + v) * 512);
-                    accumulate<DT, WEIGHTED || DT == DT_INT8>(acc[v], d, wu);
+                    if constexpr (POOL == 1) accumulate_max<DT>(acc[v], d, sb.x, sb.y, p.code_zero);
+                    else accumulate<DT, WEIGHTED || DT == DT_INT8>(acc[v], d, wu);
                 }
             }
             return;
@@ -603,18 +648,22 @@ __device__ __forceinline__ void process_item(const FwdParams& p, const TableMeta
             const uint32_t r = __shfl_sync(0xffffffffu, c.r, j0 + u, G);
             float wu = WEIGHTED ? __shfl_sync(0xffffffffu, c.w, j0 + u, G) : 1.0f;
             if (j0 + u < c.nmax && r != kInvalidRow) {
+                float2 sb = make_float2(1.0f, 0.0f);
                 if (DT == DT_INT8) {
-                    const float2 sb = lds64f(my_sb_s + (st * kStageVecs + u) * 64);
-                    acc_bias = fmaf(wu, sb.y, acc_bias);
-                    wu *= sb.x;
-                    acc_bias = fmaf(wu, -p.code_zero, acc_bias);
-                    wu *= kInt8Up;
+                    sb = lds64f(my_sb_s + (st * kStageVecs + u) * 64);
+                    if (POOL == 0) {
+                        acc_bias = fmaf(wu, sb.y, acc_bias);
+                        wu *= sb.x;
+                        acc_bias = fmaf(wu, -p.code_zero, acc_bias);
+                        wu *= kInt8Up;
+                    }
                 }
 #pragma unroll
                 for (int v = 0; v < V; ++v)
                     if (col_on[v]) {
                         const uint4 d = lds128(my_rows_s + (st * kStageVecs + u * V + v) * 512);
-                        accumulate<DT, WEIGHTED || DT == DT_INT8>(acc[v], d, wu);
+                        if constexpr (POOL == 1) accumulate_max<DT>(acc[v], d, sb.x, sb.y, p.code_zero);
+                        else accumulate<DT, WEIGHTED || DT == DT_INT8>(acc[v], d, wu);
                     }
             }
         }
@@ -637,11 +686,14 @@ __device__ __forceinline__ void process_item(const FwdParams& p, const TableMeta
 #pragma unroll
                 for (int a = 0; a < NACC / 2; ++a) {
                     float2 x = acc[v][a];
-                    if (DT == DT_INT8) {
+                    if (POOL == 1) {                 // a bag with no valid lookup reads +0
+                        if (x.x == acc0) x.x = 0.0f;
+                        if (x.y == acc0) x.y = 0.0f;
+                    } else if (DT == DT_INT8) {
                         x.x = fmaf(x.x, kInt8Down, acc_bias);
                         x.y = fmaf(x.y, kInt8Down, acc_bias);
                     }
-                    if (!PART && p.mean && L > 0) {
+                    if (POOL == 0 && !PART && p.mean && L > 0) {
                         x.x = __fdiv_rn(x.x, (float)L);
                         x.y = __fdiv_rn(x.y, (float)L);
                     }
@@ -673,7 +725,7 @@ __device__ __forceinline__ void process_item(const FwdParams& p, const TableMeta
 #pragma unroll
         for (int v = 0; v < V; ++v)
 #pragma unroll
-            for (int a = 0; a < NACC / 2; ++a) acc[v][a] = make_float2(0.0f, 0.0f);
+            for (int a = 0; a < NACC / 2; ++a) acc[v][a] = make_float2(acc0, acc0);
     };
 
     // ---- pipeline: the request side runs one stage ahead of the consuming side
@@ -730,7 +782,7 @@ __device__ __forceinline__ void process_item(const FwdParams& p, const TableMeta
 }
 
 // ------------------------------------------------------------------ the kernel
-template <int DT, bool WEIGHTED, bool MAPID>
+template <int DT, bool WEIGHTED, bool MAPID, int POOL = 0>
 __global__ void __launch_bounds__(kThreads, EBAG_MIN_BLOCKS)
 ebag_fwd_kernel(const FwdParams p) {
     extern __shared__ int smem_i[];
@@ -846,13 +898,13 @@ ebag_fwd_kernel(const FwdParams p) {
         const PartArgs no_part{};
         unsigned skip = 0;
         if (m.V == 1) {
-            process_item<DT, WEIGHTED, MAPID, 1>(p, m, tbase, t, bag0, cnt, 0, lane, n_oob, n_bad, wbuf,
-                                                 sbbuf, skip, no_part);
+            process_item<DT, WEIGHTED, MAPID, 1, false, POOL>(p, m, tbase, t, bag0, cnt, 0, lane, n_oob, n_bad,
+                                                              wbuf, sbbuf, skip, no_part);
         } else {
             // rows above 512 bytes: two vectors per lane, 1 KB column tiles
             for (int vec0 = 0; vec0 < m.nvec; vec0 += 64)
-                process_item<DT, WEIGHTED, MAPID, 2>(p, m, tbase, t, bag0, cnt, vec0, lane, n_oob, n_bad,
-                                                     wbuf, sbbuf, skip, no_part);
+                process_item<DT, WEIGHTED, MAPID, 2, false, POOL>(p, m, tbase, t, bag0, cnt, vec0, lane, n_oob,
+                                                                  n_bad, wbuf, sbbuf, skip, no_part);
         }
         q = __shfl_sync(0xffffffffu, q_next, 0);
     }
@@ -1050,6 +1102,7 @@ ebag_parts_kernel(const FwdParams p) {
     cudaError_t launch_fwd_##NAME(const FwdParams& p, bool weighted, bool mapid, int grid,        \
                                   size_t smem, cudaStream_t s);                                  \
     cudaError_t occupancy_fwd_##NAME(bool weighted, bool mapid, size_t smem, int* ctas_per_sm);  \
+    cudaError_t launch_fwdmax_##NAME(const FwdParams& p, int grid, size_t smem, cudaStream_t s);  \
     cudaError_t launch_parts_##NAME(const FwdParams& p, bool weighted, bool mapid, int grid,      \
                                     cudaStream_t s);
 EBAG_DECLARE_LAUNCHERS(f32)
@@ -1078,6 +1131,14 @@ EBAG_DECLARE_LAUNCHERS(int8)
         }                                                                                        \
         if (weighted) return cudaLaunchKernelEx(&cfg, ebag_fwd_kernel<DT, true, false>, p);       \
         return cudaLaunchKernelEx(&cfg, ebag_fwd_kernel<DT, false, false>, p);                   \
+    }                                                                                            \
+    cudaError_t launch_fwdmax_##NAME(const FwdParams& p, int grid, size_t smem, cudaStream_t s) { \
+        cudaError_t e = cudaFuncSetAttribute((const void*)ebag_fwd_kernel<DT, false, false, 1>,   \
+                                             cudaFuncAttributeMaxDynamicSharedMemorySize,        \
+                                             (int)kMaxItemTableBytes);                           \
+        if (e != cudaSuccess) return e;                                                          \
+        ebag_fwd_kernel<DT, false, false, 1><<<grid, kThreads, smem, s>>>(p);                     \
+        return cudaGetLastError();                                                               \
     }                                                                                            \
     cudaError_t launch_parts_##NAME(const FwdParams& p, bool weighted, bool mapid, int grid,      \
                                     cudaStream_t s) {                                            \

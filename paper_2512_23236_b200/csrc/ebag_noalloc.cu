@@ -136,6 +136,7 @@ extern "C" ebag_status ebag_forward_noalloc(int32_t T, const int64_t* rows, cons
     if (T <= 0 || !rows || !D || !tables || !offsets || B < 0 || n_indices < 0)
         return EBAG_ERR_INVALID_ARG;
     if (dtype < EBAG_F32 || dtype > EBAG_UINT8_ROWWISE) return EBAG_ERR_INVALID_ARG;
+    if (mode == EBAG_MAX) return EBAG_ERR_UNSUPPORTED;
     if (mode != EBAG_SUM && mode != EBAG_MEAN) return EBAG_ERR_INVALID_ARG;
     if (T > kMaxTables) return EBAG_ERR_UNSUPPORTED;       // beyond the static scratch
     if ((int64_t)T * B >= (1ll << 31)) return EBAG_ERR_UNSUPPORTED;

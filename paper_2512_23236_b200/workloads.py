@@ -38,7 +38,7 @@ import numpy as np
 import torch
 
 F32, F16, BF16, INT8_ROWWISE, UINT8_ROWWISE = 0, 1, 2, 3, 4
-SUM, MEAN = 0, 1
+SUM, MEAN, MAX = 0, 1, 2
 
 DTYPE_NAMES = {F32: "f32", F16: "f16", BF16: "bf16", INT8_ROWWISE: "int8_rowwise",
                UINT8_ROWWISE: "uint8_rowwise"}

@@ -154,6 +154,55 @@ def test_int32_ids(dtype, Ds, mode, weighted):
     assert np.array_equal(gpu32.view(np.uint32), gpu64.view(np.uint32))
 
 
+# ------------------------------------------------------------------ max pooling
+@pytest.mark.parametrize("dtype,Ds", [
+    (wl.F32, [4, 12, 64, 260, 1028]),
+    (wl.F16, [8, 128, 520]),
+    (wl.BF16, [16, 72, 256, 2056]),
+    (wl.INT8_ROWWISE, [16, 128, 528, 2064]),
+    (wl.UINT8_ROWWISE, [16, 128]),
+])
+def test_max_pooling_is_bit_exact(dtype, Ds):
+    """A maximum involves no rounding, so the GPU must equal the oracle bit for bit, whatever the
+    order (rowwise 8-bit: scale*q and +bias are rounded separately on both sides).  Skipped ids
+    take no part, bags with no valid lookup are +0, a very long bag is pooled by one warp."""
+    rng = np.random.default_rng(61 + dtype)
+    T, B = len(Ds), 90
+    rows = [int(rng.integers(5, 400)) for _ in Ds]
+    lens = [rng.integers(0, 40, size=B) for _ in Ds]
+    for l in lens:
+        l[rng.random(B) < 0.15] = 0
+    lens[0][7] = 3000
+    idx, off, lengths = _jagged_from_lengths(rng, lens, rows)
+    bad = rng.choice(idx.shape[0], size=40, replace=False)
+    idx[bad] = -3
+    lens_last = lengths[(T - 1) * B + 4]
+    g = (T - 1) * B + 4                                     # one bag made of skipped ids only
+    idx[off[g]:off[g + 1]] = 10 ** 9
+    tabs = _rand_tables(rng, dtype, rows, Ds)
+    for ids in (idx, idx.astype(np.int32)):
+        gpu, status, ref = _both(dtype, rows, Ds, tabs, ids, off, B, wl.MAX)
+        assert status == (eb.EBAG_ERR_INDEX_OOB, ref["n_oob"], 0) and ref["n_oob"] >= 40
+        assert np.array_equal(gpu.view(np.uint32), ref["out32"].view(np.uint32))
+    col = sum(Ds[:T - 1])
+    assert np.all(gpu[4, col:col + Ds[T - 1]] == 0.0) and lens_last >= 0
+
+
+def test_max_pooling_argument_rules():
+    tbe = eb.TBE([10], [16], eb.EBAG_F32, device=torch.cuda.current_device())
+    try:
+        tab = torch.zeros(10, 16, device="cuda")
+        idx = torch.zeros(4, dtype=torch.int64, device="cuda")
+        off = torch.tensor([0, 4], dtype=torch.int64, device="cuda")
+        with pytest.raises(eb.EbagError) as e:
+            tbe.forward([tab], idx, off, 1, eb.EBAG_MAX, torch.ones(4, device="cuda"))
+        assert e.value.status == eb.EBAG_ERR_UNSUPPORTED
+        out = tbe.forward([tab - 2.0], idx, off, 1, eb.EBAG_MAX)
+        assert tbe.launch_count() == 1 and float(out.max()) == -2.0
+    finally:
+        tbe.close()
+
+
 # ------------------------------------------------------------------ 16-bit output
 def _round_bf16(x32):
     """fp32 array rounded to nearest-even bf16, returned as fp32."""
