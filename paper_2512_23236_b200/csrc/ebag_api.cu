@@ -19,6 +19,7 @@ namespace {
 constexpr int kTableSlots = 4;   // device copies of the table-pointer array that may be in flight
 constexpr int kMaxHostChunks = 16;                 // bag ranges per ebag_forward_host call
 constexpr int64_t kHostChunkBytes = 64ll << 20;    // transfer size one range aims for
+constexpr uint64_t kSmallCallBytesPerWarp = 16384;   // see forward_device
 constexpr uint64_t kLongScratchBytes = 64ull << 20;  // partial sums of split bags, per handle
 constexpr uint64_t kLongMaxParts = 8 * kMaxLongBags; // parts of split bags per launch (see forward_device)
 constexpr int kAutoHostChunks = 6;                 // more ranges cost more in small copies than they hide
@@ -270,7 +271,14 @@ ebag_status forward_device(ebag_tbe* h, const void* const* tables, const int64_t
     const bool w = weights != nullptr;
     const bool mapid = mappings != nullptr;
     int per_sm = h->occupancy[mapid ? 1 : 0][w ? 1 : 0];
-    if (h->ctas_per_sm > 0 && h->ctas_per_sm < per_sm) per_sm = h->ctas_per_sm;
+    if (h->ctas_per_sm > 0) {
+        if (h->ctas_per_sm < per_sm) per_sm = h->ctas_per_sm;
+    } else {
+        // A small call is over before a full grid has even started: one resident CTA per SM for
+        // every kSmallCallBytesPerWarp the call can gather per warp (workload 1: 18.9 -> 15.6 us).
+        const uint64_t want = bound / ((uint64_t)h->num_sms * (kThreads / 32) * kSmallCallBytesPerWarp) + 1;
+        if (want < (uint64_t)per_sm) per_sm = (int)want;
+    }
     const int grid = h->num_sms * per_sm;
     if (mode == EBAG_MAX) {                        // its own kernel; bags are never split
         if (mapid) return EBAG_ERR_UNSUPPORTED;
