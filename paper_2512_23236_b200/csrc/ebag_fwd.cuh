@@ -2,23 +2,32 @@
 //
 // One persistent kernel serves all T tables of a call.  Work is cut into ITEMS: runs of up to 32
 // consecutive bags of one table, sized on the device from the offsets array (which is the prefix
-// sum of the bag lengths) so that every item gathers about `item_bytes` of rows whatever the
-// table's row size and mean bag length (less when the whole call is small, so that every warp
-// still gets work).  Warps pull items from a global counter in table-major order, so a table's
-// hot rows stay in L2 while that table is being processed and bags of very unequal length are
-// balanced dynamically.
+// sum of the bag lengths) so that an item gathers about `item_bytes` of rows (eight times that
+// for rows of one vector per lane; less for the last tables of a call and when the whole call is
+// small, so that every warp still gets work and the slowest one finishes soon after the rest).
+// Warps pull items from a global counter in table-major order, so a table's hot rows stay in L2
+// while that table is being processed and bags of very unequal length are balanced dynamically.
+// A bag too long for one warp is not pooled here: it is recorded, and a second, short kernel
+// (ebag_parts_kernel, below) pools the recorded bags in parts over the whole grid.
 //
 // Inside an item a warp is split into row groups of G lanes (G*16 bytes cover one row, G in
 // {4,8,16,32}, a run-time property of the table; rows above 512 bytes take 2 vectors per lane, in
 // column tiles of 1 KB).  Each group owns one bag at a time; the 32/G bags that run side by side
-// are picked after sorting the item's bags by length, so the groups finish together.  The lanes
-// of a group read G ids (and weights) of their bag with one coalesced load, two chunks ahead of
-// use; each id is then broadcast inside the group with a shuffle and the row is requested with
-// 16-byte cp.async copies (through L1) into a per-warp two-stage ring in shared memory, one
-// stage (4 row vectors per lane) ahead of the stage being accumulated.  Row fetches therefore
-// stay in flight across stage, id-chunk and bag boundaries and occupy no registers.  Widening
-// (bf16/fp16), rowwise-int8 dequantisation and the per-sample weight are fused into the fp32
-// accumulation; the result is written once with 128-bit streaming stores.
+// are picked after sorting the item's bags by length, so the groups finish together (the bags'
+// ranges and the sorted order sit in shared memory).  The lanes of a group read G ids (and
+// weights) of their bag with one coalesced load, two chunks ahead of use; each id is then
+// broadcast inside the group with a shuffle and the row is requested with 16-byte cp.async
+// copies (through L1: the hot rows of a skewed workload are served from there, bypassing it was
+// measured five times slower) into a per-warp two-stage ring in shared memory, one stage (4 row
+// vectors per lane) ahead of the stage being accumulated.  Row fetches therefore stay in flight
+// across stage, id-chunk and bag boundaries and occupy no registers.  Widening (bf16/fp16),
+// rowwise 8-bit dequantisation and the per-sample weight are fused into the fp32 accumulation
+// (or the element-wise maximum, for max pooling); the result is written once with streaming
+// stores, as fp32 or rounded to fp16 / bf16.
+//
+// Both kernels are launched with programmatic stream serialization and start with
+// griddepcontrol.wait: a launch may become resident while the kernel ahead of it on the stream
+// drains, and reads nothing before that kernel has finished.
 //
 // Ids outside the table and malformed bags never fault: they are skipped, counted and reported
 // through the handle's status words.
