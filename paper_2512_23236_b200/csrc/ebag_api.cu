@@ -22,7 +22,7 @@ constexpr int64_t kHostChunkBytes = 64ll << 20;    // transfer size one range ai
 constexpr uint64_t kSmallCallBytesPerWarp = 16384;   // see forward_device
 constexpr uint64_t kLongScratchBytes = 64ull << 20;  // partial sums of split bags, per handle
 constexpr uint64_t kLongMaxParts = 8 * kMaxLongBags; // parts of split bags per launch (see forward_device)
-constexpr int kAutoHostChunks = 6;                 // more ranges cost more in small copies than they hide
+constexpr int kAutoHostChunks = 8;                 // more ranges cost more in small copies than they hide
 
 struct DeviceGuard {             // make the handle's device current for the duration of a call
     int prev = -1;
@@ -283,11 +283,11 @@ ebag_status forward_device(ebag_tbe* h, const void* const* tables, const int64_t
     if (mode == EBAG_MAX) {                        // its own kernel; bags are never split
         if (mapid) return EBAG_ERR_UNSUPPORTED;
         p.lg.ctl = nullptr;
-        EBAG_CUDA(h, launch_fwdmax(h->dtype, p, grid, fwd_smem_bytes(h->T), stream));
+        EBAG_CUDA(h, launch_fwdmax(h->dtype, p, grid, fwd_smem_bytes(p.T), stream));
         ++h->launches;
         return EBAG_OK;
     }
-    EBAG_CUDA(h, launch_fwd(h->dtype, p, w, mapid, grid, fwd_smem_bytes(h->T), stream));
+    EBAG_CUDA(h, launch_fwd(h->dtype, p, w, mapid, grid, fwd_smem_bytes(p.T), stream));
     ++h->launches;
     if (p.lg.ctl) {
         EBAG_CUDA(h, launch_parts(h->dtype, p, w, mapid, grid, stream));
@@ -713,11 +713,14 @@ ebag_status ebag_forward_host(ebag_tbe* h, const void* const* tables, const int3
         EBAG_CUDA(h, cudaMemcpyAsync(out, h->s_out, sizeof(float) * n_out, cudaMemcpyDeviceToHost, s));
         return EBAG_OK;
     }
-    // Pipeline: inputs of range k+1 travel while the kernel works on range k and the result of
-    // range k-1 travels back.  Kernels stay on the caller's stream.
+    // Pipeline: inputs of piece k+1 travel while the kernel works on piece k and the result of
+    // piece k-1 travels back.  Kernels stay on the caller's stream.
     EBAG_CUDA(h, cudaEventRecord(h->ev_fork, s));
     EBAG_CUDA(h, cudaStreamWaitEvent(h->s_h2d, h->ev_fork, 0));
     EBAG_CUDA(h, cudaStreamWaitEvent(h->s_d2h, h->ev_fork, 0));
+    // all offsets first, in one copy (every piece's item sizing reads the table boundaries)
+    EBAG_CUDA(h, cudaMemcpyAsync(h->s_offsets, offsets, sizeof(int64_t) * n_off, cudaMemcpyHostToDevice, h->s_h2d));
+    // pieces are ranges of bags: per table one block of ids (and weights) in, one block of rows out
     for (int64_t c = 0; c < chunks; ++c) {
         const int64_t b0 = c * B / chunks, b1 = (c + 1) * B / chunks;
         for (int t = 0; t < h->T; ++t) {
@@ -730,10 +733,6 @@ ebag_status ebag_forward_host(ebag_tbe* h, const void* const* tables, const int3
                     EBAG_CUDA(h, cudaMemcpyAsync(h->s_weights + lo, per_sample_weights + lo,
                                                  sizeof(float) * (hi - lo), cudaMemcpyHostToDevice, h->s_h2d));
             }
-            // (the entry at b0 came with the previous range; range 0 brings its own)
-            const int64_t first = c == 0 ? b0 : b0 + 1;
-            EBAG_CUDA(h, cudaMemcpyAsync(h->s_offsets + g + first, offsets + g + first,
-                                         sizeof(int64_t) * (b1 - first + 1), cudaMemcpyHostToDevice, h->s_h2d));
         }
         EBAG_CUDA(h, cudaEventRecord(h->ev_in[c], h->s_h2d));
         EBAG_CUDA(h, cudaStreamWaitEvent(s, h->ev_in[c], 0));
