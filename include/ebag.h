@@ -217,10 +217,14 @@ ebag_status ebag_mapid_tbe(ebag_tbe* h, const int64_t* values, int64_t n_values,
  * array [T]) and pools row 0 for unknown ids, row k for the k-th known id.  Table t therefore
  * has mapping_len[t] + 1 rows (create the handle with those row counts); a mapped id beyond the
  * table's rows is skipped and counted like any out-of-range id.  Everything else as
- * ebag_forward: no allocation, no synchronisation; the mapping arrays are read
- * before the call returns.  This is the producer of embedding ids the paper's preprocessing
- * section describes, placed directly in front of the gather so that the mapped ids never travel
- * through memory.
+ * ebag_forward; the mapping arrays are read before the call returns.  By default the transform
+ * runs for all tables in one launch into a buffer of n_values ids that the handle keeps (it is
+ * grown, with a device synchronisation, when a larger call arrives: the only allocation), and
+ * the plain forward follows on the same stream.  With ebag_set_param("mapid_fused", 1) the
+ * search runs inside the forward kernel instead, directly in front of the gather, so that the
+ * mapped ids never travel through memory and nothing is allocated: less traffic, but measured
+ * slower at the mapping sizes tried (the searches stall the row pipeline).  This is the
+ * producer of embedding ids the paper's preprocessing section describes.
  */
 ebag_status ebag_forward_mapid(ebag_tbe* h, const void* const* tables, const int32_t* D,
                                const int64_t* values, int64_t n_values, const int64_t* offsets,
@@ -309,6 +313,8 @@ ebag_status ebag_forward_noalloc(int32_t T, const int64_t* rows, const int32_t* 
  *   "item_bytes"   target bytes of gathered rows per work item (default 32768)
  *   "ctas_per_sm"  resident CTAs per SM of the persistent grid (default: occupancy limit)
  *   "host_chunks"  bag ranges per ebag_forward_host call, 1..16 (default 0: from the size)
+ *   "mapid_fused"  ebag_forward_mapid: 1 = search inside the forward kernel, 0 (default) = the
+ *                  transform in a launch of its own, then the plain forward
  *   "out_dtype"    element type of `out` in ebag_forward, ebag_forward_i32 and
  *                  ebag_forward_mapid: EBAG_F32 (default), EBAG_F16 or EBAG_BF16.  Sums are still
  *                  accumulated in fp32 and rounded to nearest-even once, when the bag is written;

@@ -49,7 +49,8 @@ def test_mapid_degenerate_sizes():
 
 @pytest.mark.parametrize("dtype", [wl.F32, wl.BF16, wl.INT8_ROWWISE])
 @pytest.mark.parametrize("mode,weighted", [(wl.SUM, False), (wl.MEAN, False), (wl.SUM, True)])
-def test_fused_mapid_forward(dtype, mode, weighted):
+@pytest.mark.parametrize("fused", [0, 1])
+def test_fused_mapid_forward(dtype, mode, weighted, fused):
     rng = np.random.default_rng(31 + dtype)
     T, B = 5, 300
     Ds = {wl.F32: [64, 8, 256, 132, 32], wl.BF16: [64, 128, 256, 8, 1032],
@@ -82,6 +83,7 @@ def test_fused_mapid_forward(dtype, mode, weighted):
     dev = pu.device_tables(dtype, tabs)
     dmaps = [torch.from_numpy(m).cuda() for m in mappings]
     tbe = eb.TBE(rows, Ds, dtype, device=torch.cuda.current_device())
+    tbe.set_param("mapid_fused", fused)       # 1: search inside the forward kernel; 0: two launches
     out = torch.full((B, sum(Ds)), float("nan"), dtype=torch.float32, device="cuda")
     tbe.forward_mapid(dev, torch.from_numpy(values).cuda(), torch.from_numpy(offsets).cuda(), dmaps, B,
                       mode, None if w is None else torch.from_numpy(w).cuda(), out=out)
