@@ -747,7 +747,11 @@ def main():
         default_out = d_out.clone()
         mapid_extra = {"mapid_then_forward_ms": elapsed_ms / args.steps, "fused_ms": timed(fused)}
         assert torch.equal(default_out, d_out), "fused MapId forward and the two-launch path disagree"
-        mapid_extra["mapid_alone_ms"] = timed(mapid_only)
+        mapid_extra["mapid_alone_ms"] = timed(mapid_only)              # hash tables of the mappings
+        assert torch.equal(ids, d_idx)
+        tbe.set_param("mapid_hash", 0)
+        mapid_extra["mapid_alone_binary_search_ms"] = timed(mapid_only)
+        tbe.set_param("mapid_hash", 1)
         mapid_extra["plain_forward_ms"] = timed(plain)
         assert torch.equal(default_out, d_out), "MapId forward and plain forward disagree"
         assert torch.equal(ids, d_idx)
@@ -782,7 +786,7 @@ def main():
                      "frac_of_nominal_8TBs": achieved / 8000.0,
                      "algorithmic_bytes_per_launch": ab["total"],
                      "ms_per_launch": ms_per_launch, "ms_per_launch_min": min(step_ms),
-                     "traffic": NCU_DRAM_BYTES_PER_LAUNCH.get(w.number)},
+                     "traffic": None if mapid else NCU_DRAM_BYTES_PER_LAUNCH.get(w.number)},
         "bags_per_sec": w.T * w.B * world * args.steps / (max_ms * 1e-3),
     }
     if mapid_extra:

@@ -205,6 +205,13 @@ ebag_status ebag_mapid(const int64_t* values, int64_t n, const int64_t* mapping,
  * receives the row ids, ready for ebag_forward.  The table slices are read from offsets on the
  * device, so there is no host synchronisation.  Followed by ebag_forward this was measured
  * faster than the fused call for mappings of 1 k - 100 k ids (the fused search stalls the gather).
+ * When the call has at least as many values as the hash tables of its mappings have slots (per
+ * table the power of two at or above twice its length, 16 bytes a slot, 2^24 slots in all at
+ * most), those tables are first built in a scratch buffer the handle keeps (grown, with a device
+ * synchronisation, when a larger call arrives) and every value is then found with one or two
+ * loads: three operations on the stream (clear, build, look up; two kernel launches) instead of
+ * one binary-search launch.  Both give the same ids for a sorted mapping, with equal keys mapped
+ * to the first of their run.  ebag_set_param("mapid_hash", 0) keeps to the binary search.
  */
 ebag_status ebag_mapid_tbe(ebag_tbe* h, const int64_t* values, int64_t n_values,
                            const int64_t* offsets, const int64_t* const* mappings,
@@ -315,6 +322,9 @@ ebag_status ebag_forward_noalloc(int32_t T, const int64_t* rows, const int32_t* 
  *   "host_chunks"  bag ranges per ebag_forward_host call, 1..16 (default 0: from the size)
  *   "mapid_fused"  ebag_forward_mapid: 1 = search inside the forward kernel, 0 (default) = the
  *                  transform in a launch of its own, then the plain forward
+ *   "mapid_hash"   ebag_mapid_tbe (and with it the default ebag_forward_mapid): 1 (default) =
+ *                  look values up through hash tables of the mappings when the call is large
+ *                  enough to pay for building them, 0 = always binary search
  *   "out_dtype"    element type of `out` in ebag_forward, ebag_forward_i32 and
  *                  ebag_forward_mapid: EBAG_F32 (default), EBAG_F16 or EBAG_BF16.  Sums are still
  *                  accumulated in fp32 and rounded to nearest-even once, when the bag is written;

@@ -42,6 +42,10 @@ int elem_bytes(int dtype) { return dtype == EBAG_F32 ? 4 : (is_rowwise8(dtype) ?
 
 }  // namespace
 
+namespace {
+struct MapSlot;
+}
+
 struct ebag_tbe {
     int T = 0, dtype = 0, device = 0, sumD = 0, num_sms = 0;
     std::vector<int64_t> rows;
@@ -74,6 +78,9 @@ struct ebag_tbe {
     std::string cuda_error;
     // staging for ebag_forward_host
     int64_t* s_indices = nullptr;
+    MapSlot* s_maphash = nullptr;     // hash tables of the mappings of the MapId call in flight
+    int64_t cap_maphash = 0;
+    int mapid_hash = 1;
     int64_t* s_offsets = nullptr;
     float* s_weights = nullptr;
     float* s_out = nullptr;
@@ -121,6 +128,7 @@ void free_handle(ebag_tbe* h) {
         if (h->ev_done[i]) cudaEventDestroy(h->ev_done[i]);
     }
     cudaFree(h->s_indices);
+    cudaFree(h->s_maphash);
     cudaFree(h->s_offsets);
     cudaFree(h->s_weights);
     cudaFree(h->s_out);
@@ -335,11 +343,96 @@ __global__ void pack_int8_rowwise_kernel(const int8_t* __restrict__ q, const flo
     }
 }
 
+// ---- MapId, stand-alone kernels.  A search is a chain of dependent loads; the first ten of its
+// steps are taken in shared memory: the CTA keeps up to kPivots pivots of its mapping there,
+// pivot j = the LAST entry of block j of `stride` consecutive entries.  The insertion index of v
+// lies in the first block whose pivot is >= v, so a search is a halving search over the pivots
+// (shared memory) followed by one over that block (global memory, log2(stride) steps instead of
+// log2(|M|)); mappings of up to kPivots entries never touch global memory again.
+constexpr int kPivots = 1024;
+
+__device__ __forceinline__ void load_pivots(const int64_t* __restrict__ M, uint32_t mlen, uint32_t stride,
+                                            uint32_t np, int64_t* pivots) {
+    for (uint32_t j = threadIdx.x; j < np; j += blockDim.x) {
+        const uint64_t last = (uint64_t)(j + 1) * stride - 1;
+        pivots[j] = __ldg(M + (last < mlen ? (uint32_t)last : mlen - 1));
+    }
+    __syncthreads();
+}
+
+// Four searches side by side (their chains of dependent loads overlap): out[k] = MapId(v[k]).
+__device__ __forceinline__ void map_id4_pivots(const int64_t* __restrict__ M, uint32_t mlen, uint32_t stride,
+                                               uint32_t np, int steps1, int steps2,
+                                               const int64_t* pivots, const int64_t (&v)[4], int64_t (&out)[4]) {
+    if (mlen == 0) {
+#pragma unroll
+        for (int k = 0; k < 4; ++k) out[k] = 0;
+        return;
+    }
+    uint32_t lo[4] = {0, 0, 0, 0}, hi[4] = {np, np, np, np};
+    for (int s = 0; s < steps1; ++s) {                      // first pivot >= v, in shared memory
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const uint32_t mid = (lo[k] + hi[k]) >> 1;
+            const int64_t pv = pivots[mid < np ? mid : np - 1];
+            const bool active = lo[k] < hi[k];
+            const bool right = pv < v[k];
+            lo[k] = (active && right) ? mid + 1 : lo[k];
+            hi[k] = (active && !right) ? mid : hi[k];
+        }
+    }
+    uint32_t blo[4], bhi[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {                           // that block (or past the end: v > max M)
+        const uint64_t b0 = (uint64_t)lo[k] * stride, b1 = b0 + stride;
+        blo[k] = b0 < mlen ? (uint32_t)b0 : mlen;
+        bhi[k] = b1 < mlen ? (uint32_t)b1 : mlen;
+    }
+    for (int s = 0; s < steps2; ++s) {                      // first entry >= v inside the block
+        int64_t mv[4];
+        uint32_t mid[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            mid[k] = (blo[k] + bhi[k]) >> 1;
+            mv[k] = __ldg(M + (mid[k] < mlen ? mid[k] : mlen - 1));
+        }
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const bool active = blo[k] < bhi[k];
+            const bool right = mv[k] < v[k];
+            blo[k] = (active && right) ? mid[k] + 1 : blo[k];
+            bhi[k] = (active && !right) ? mid[k] : bhi[k];
+        }
+    }
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const uint32_t idx = blo[k] < mlen ? blo[k] : mlen - 1;
+        out[k] = __ldg(M + idx) == v[k] ? (int64_t)idx + 1 : 0;
+    }
+}
+
+struct PivotPlan {
+    uint32_t stride, np;
+    int steps1, steps2;
+};
+__device__ __forceinline__ PivotPlan plan_pivots(uint32_t mlen) {
+    PivotPlan pl;
+    pl.stride = mlen ? (mlen + kPivots - 1) / kPivots : 1;
+    pl.np = mlen ? (mlen + pl.stride - 1) / pl.stride : 0;
+    pl.steps1 = 32 - __clz(pl.np);
+    pl.steps2 = 32 - __clz(pl.stride);           // bit length: enough halvings for a block of `stride`
+    if (pl.stride == 1) pl.steps2 = 1;           // one-entry blocks: a single step settles lo
+    return pl;
+}
+
 // MapId of values[lo, hi): every thread runs four searches at a time, on values a block-width
-// apart, so that loads and stores stay coalesced and the four dependent-load chains overlap.
+// apart, so that loads and stores stay coalesced.
 __device__ __forceinline__ void mapid_range(const int64_t* __restrict__ values, int64_t lo, int64_t hi,
-                                            const int64_t* __restrict__ M, uint32_t mlen, int steps,
-                                            int64_t* __restrict__ out, int64_t first, int64_t stride) {
+                                            const int64_t* __restrict__ M, uint32_t mlen,
+                                            int64_t* __restrict__ out, int64_t first, int64_t stride,
+                                            int64_t* pivots) {
+    const PivotPlan pl = plan_pivots(mlen);
+    if (mlen) load_pivots(M, mlen, pl.stride, pl.np, pivots);
     const int64_t step = stride * 4;
     for (int64_t i = lo + first; i < hi; i += step) {
         int64_t v[4], r[4];
@@ -348,7 +441,7 @@ __device__ __forceinline__ void mapid_range(const int64_t* __restrict__ values, 
             const int64_t j = i + k * stride;
             v[k] = j < hi ? __ldcs(reinterpret_cast<const long long*>(values + j)) : 0;
         }
-        map_id4(M, mlen, steps, v, r);
+        map_id4_pivots(M, mlen, pl.stride, pl.np, pl.steps1, pl.steps2, pivots, v, r);
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
             const int64_t j = i + k * stride;
@@ -357,29 +450,233 @@ __device__ __forceinline__ void mapid_range(const int64_t* __restrict__ values, 
     }
 }
 
-__global__ void mapid_kernel(const int64_t* __restrict__ values, int64_t n,
-                             const int64_t* __restrict__ mapping, uint32_t mlen, int steps,
-                             int64_t* __restrict__ out) {
-    mapid_range(values, 0, n, mapping, mlen, steps, out, blockIdx.x * (int64_t)blockDim.x + threadIdx.x,
-                (int64_t)gridDim.x * blockDim.x);
+__global__ void __launch_bounds__(256)
+mapid_kernel(const int64_t* __restrict__ values, int64_t n, const int64_t* __restrict__ mapping,
+             uint32_t mlen, int64_t* __restrict__ out) {
+    __shared__ int64_t pivots[kPivots];
+    mapid_range(values, 0, n, mapping, mlen, out, blockIdx.x * (int64_t)blockDim.x + threadIdx.x,
+                (int64_t)gridDim.x * blockDim.x, pivots);
 }
 
-// MapId for all tables of a TBE call in one launch: blockIdx.y is the table, whose slice of the
-// jagged value list is read from the offsets array on the device (no host synchronisation).
-__global__ void mapid_tbe_kernel(const int64_t* __restrict__ values, int64_t n_values,
-                                 const int64_t* __restrict__ offsets, int64_t B,
-                                 const int64_t* const* __restrict__ mappings,
-                                 const int64_t* __restrict__ mapping_len, int64_t* __restrict__ out) {
+// MapId for all tables of a TBE call in one launch.  The tables' slices of the jagged value list
+// are read from the offsets array on the device (no host synchronisation) and cut into chunks of
+// kMapChunk values; every CTA takes an equal run of consecutive chunks, so the work is balanced
+// whatever the tables' sizes, and reloads its pivots only when its run crosses into another table.
+constexpr int kMapChunk = 16384;
+constexpr int kMapMaxTables = 2048;
+
+__global__ void __launch_bounds__(256)
+mapid_tbe_kernel(const int64_t* __restrict__ values, int64_t n_values, const int64_t* __restrict__ offsets,
+                 int64_t B, int T, const int64_t* const* __restrict__ mappings,
+                 const int64_t* __restrict__ mapping_len, int64_t* __restrict__ out) {
+    __shared__ int64_t pivots[kPivots];
+    __shared__ int chunk_base[kMapMaxTables + 1];           // first chunk of every table
+    for (int t = threadIdx.x; t < T; t += blockDim.x) {
+        int64_t lo = offsets[(int64_t)t * B], hi = offsets[(int64_t)(t + 1) * B];
+        if (lo < 0) lo = 0;
+        if (hi > n_values) hi = n_values;
+        chunk_base[t + 1] = hi > lo ? (int)((hi - lo + kMapChunk - 1) / kMapChunk) : 0;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        chunk_base[0] = 0;
+        for (int t = 0; t < T; ++t) chunk_base[t + 1] += chunk_base[t];
+    }
+    __syncthreads();
+    const int total = chunk_base[T];
+    const int per_cta = (total + gridDim.x - 1) / gridDim.x;
+    const int c0 = blockIdx.x * per_cta;
+    const int c1 = c0 + per_cta < total ? c0 + per_cta : total;
+    int cur_t = -1;
+    const int64_t* M = nullptr;
+    uint32_t mlen = 0;
+    PivotPlan pl = plan_pivots(0);
+    for (int c = c0; c < c1; ++c) {
+        int lo_t = cur_t < 0 ? 0 : cur_t, hi_t = T;          // tables come in order: search from the current one
+        while (hi_t - lo_t > 1) {
+            const int mid = (lo_t + hi_t) >> 1;
+            if (chunk_base[mid] <= c) lo_t = mid; else hi_t = mid;
+        }
+        if (lo_t != cur_t) {
+            cur_t = lo_t;
+            M = mappings[cur_t];
+            const int64_t ml = mapping_len[cur_t];
+            mlen = (uint32_t)(ml < 0 ? 0 : ml);
+            pl = plan_pivots(mlen);
+            __syncthreads();                                 // everyone is done with the old pivots
+            if (mlen) load_pivots(M, mlen, pl.stride, pl.np, pivots);
+        }
+        int64_t lo = offsets[(int64_t)cur_t * B], hi = offsets[(int64_t)(cur_t + 1) * B];
+        if (lo < 0) lo = 0;
+        if (hi > n_values) hi = n_values;
+        const int64_t v0 = lo + (int64_t)(c - chunk_base[cur_t]) * kMapChunk;
+        const int64_t v1 = v0 + kMapChunk < hi ? v0 + kMapChunk : hi;
+        for (int64_t i = v0 + threadIdx.x; i < v1; i += 4 * blockDim.x) {
+            int64_t v[4], r[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const int64_t j = i + k * blockDim.x;
+                v[k] = j < v1 ? __ldcs(reinterpret_cast<const long long*>(values + j)) : 0;
+            }
+            map_id4_pivots(M, mlen, pl.stride, pl.np, pl.steps1, pl.steps2, pivots, v, r);
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const int64_t j = i + k * blockDim.x;
+                if (j < v1) out[j] = r[k];
+            }
+        }
+    }
+}
+
+// ---- MapId through a hash table.  When a call has many more values than mapping entries, the
+// handle first builds, per table, an open-addressing table of the mapping (16-byte slots: key,
+// index + 1; linear probing; at most half full) and the searches become one or two loads each
+// instead of log2(|M|) dependent ones.  The result is the same as the binary search's for a
+// sorted mapping: equal keys are adjacent there and only the first of a run is inserted.
+struct __align__(16) MapSlot {
+    int64_t key;
+    uint32_t idx1;      // index + 1; 0 = empty
+    uint32_t pad;
+};
+constexpr uint64_t kHashMul = 0x9E3779B97F4A7C15ull;     // multiplicative (Fibonacci) hashing
+constexpr int64_t kMapHashMaxSlots = 1ll << 24;          // 256 MB of slots per handle at most
+
+__host__ __device__ inline uint32_t map_hash_bits(int64_t mlen) {
+    uint32_t bits = 1;
+    while (bits < 31 && (1ll << bits) < 2 * mlen) ++bits;
+    return bits;
+}
+
+// base slot of every table's hash table, in shared memory (T + 1 entries), by thread 0
+__device__ __forceinline__ void map_hash_bases(int T, const int64_t* __restrict__ mapping_len, uint32_t* hbase) {
+    if (threadIdx.x == 0) {
+        uint32_t at = 0;
+        for (int t = 0; t < T; ++t) {
+            hbase[t] = at;
+            const int64_t ml = mapping_len[t];
+            at += 1u << map_hash_bits(ml < 0 ? 0 : ml);
+        }
+        hbase[T] = at;
+    }
+}
+
+__global__ void __launch_bounds__(256)
+map_hash_build_kernel(int T, const int64_t* const* __restrict__ mappings,
+                      const int64_t* __restrict__ mapping_len, MapSlot* __restrict__ slots) {
+    __shared__ uint32_t base_s;
     const int t = blockIdx.y;
-    int64_t lo = offsets[(int64_t)t * B], hi = offsets[(int64_t)(t + 1) * B];
-    if (lo < 0) lo = 0;
-    if (hi > n_values) hi = n_values;
-    const int64_t* M = mappings[t];
     const int64_t ml = mapping_len[t];
-    const uint32_t mlen = (uint32_t)(ml < 0 ? 0 : ml);
-    const int steps = 32 - __clz(mlen);
-    mapid_range(values, lo, hi, M, mlen, steps, out, blockIdx.x * (int64_t)blockDim.x + threadIdx.x,
-                (int64_t)gridDim.x * blockDim.x);
+    if (threadIdx.x == 0) {
+        uint32_t at = 0;
+        for (int u = 0; u < t; ++u) {
+            const int64_t l = mapping_len[u];
+            at += 1u << map_hash_bits(l < 0 ? 0 : l);
+        }
+        base_s = at;
+    }
+    __syncthreads();
+    if (ml <= 0) return;
+    const uint32_t bits = map_hash_bits(ml), mask = (1u << bits) - 1u;
+    MapSlot* tab = slots + base_s;
+    const int64_t* M = mappings[t];
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < ml; i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t key = M[i];
+        if (i > 0 && M[i - 1] == key) continue;              // only the first of a run of equal keys
+        uint32_t s = (uint32_t)(((uint64_t)key * kHashMul) >> (64 - bits));
+        for (uint32_t probe = 0; probe <= mask; ++probe) {   // at most half full: ends early
+            if (atomicCAS(&tab[s].idx1, 0u, (uint32_t)i + 1u) == 0u) {
+                tab[s].key = key;
+                break;
+            }
+            s = (s + 1) & mask;
+        }
+    }
+}
+
+// four look-ups side by side
+__device__ __forceinline__ void map_hash_lookup4(const MapSlot* __restrict__ tab, uint32_t bits,
+                                                 const int64_t (&v)[4], int64_t (&out)[4]) {
+    const uint32_t mask = (1u << bits) - 1u;
+    uint32_t s[4];
+    bool open[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        s[k] = (uint32_t)(((uint64_t)v[k] * kHashMul) >> (64 - bits));
+        open[k] = true;
+        out[k] = 0;
+    }
+    for (uint32_t probe = 0; probe <= mask; ++probe) {
+        int4 q[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+            q[k] = open[k] ? __ldg(reinterpret_cast<const int4*>(tab + s[k])) : make_int4(0, 0, 0, 0);
+        bool any = false;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const int64_t key = (int64_t)(((uint64_t)(uint32_t)q[k].y << 32) | (uint32_t)q[k].x);
+            const bool hit = q[k].z != 0 && key == v[k];
+            if (open[k] && hit) out[k] = (int64_t)(uint32_t)q[k].z;
+            open[k] = open[k] && q[k].z != 0 && !hit;        // an empty slot ends the search: not mapped
+            s[k] = (s[k] + 1) & mask;
+            any = any || open[k];
+        }
+        if (!any) break;
+    }
+}
+
+__global__ void __launch_bounds__(256)
+mapid_tbe_hash_kernel(const int64_t* __restrict__ values, int64_t n_values, const int64_t* __restrict__ offsets,
+                      int64_t B, int T, const int64_t* __restrict__ mapping_len,
+                      const MapSlot* __restrict__ slots, int64_t* __restrict__ out) {
+    __shared__ int chunk_base[kMapMaxTables + 1];           // first chunk of every table
+    __shared__ uint32_t hbase[kMapMaxTables + 1];
+    for (int t = threadIdx.x; t < T; t += blockDim.x) {
+        int64_t lo = offsets[(int64_t)t * B], hi = offsets[(int64_t)(t + 1) * B];
+        if (lo < 0) lo = 0;
+        if (hi > n_values) hi = n_values;
+        chunk_base[t + 1] = hi > lo ? (int)((hi - lo + kMapChunk - 1) / kMapChunk) : 0;
+    }
+    map_hash_bases(T, mapping_len, hbase);
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        chunk_base[0] = 0;
+        for (int t = 0; t < T; ++t) chunk_base[t + 1] += chunk_base[t];
+    }
+    __syncthreads();
+    const int total = chunk_base[T];
+    const int per_cta = (total + gridDim.x - 1) / gridDim.x;
+    const int c0 = blockIdx.x * per_cta;
+    const int c1 = c0 + per_cta < total ? c0 + per_cta : total;
+    int cur_t = 0;
+    for (int c = c0; c < c1; ++c) {
+        int hi_t = T;                                        // tables come in order: search from the current one
+        while (hi_t - cur_t > 1) {
+            const int mid = (cur_t + hi_t) >> 1;
+            if (chunk_base[mid] <= c) cur_t = mid; else hi_t = mid;
+        }
+        const int64_t ml = mapping_len[cur_t];
+        const uint32_t bits = map_hash_bits(ml < 0 ? 0 : ml);
+        const MapSlot* tab = slots + hbase[cur_t];
+        int64_t lo = offsets[(int64_t)cur_t * B], hi = offsets[(int64_t)(cur_t + 1) * B];
+        if (lo < 0) lo = 0;
+        if (hi > n_values) hi = n_values;
+        const int64_t v0 = lo + (int64_t)(c - chunk_base[cur_t]) * kMapChunk;
+        const int64_t v1 = v0 + kMapChunk < hi ? v0 + kMapChunk : hi;
+        for (int64_t i = v0 + threadIdx.x; i < v1; i += 4 * blockDim.x) {
+            int64_t v[4], r[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const int64_t j = i + k * blockDim.x;
+                v[k] = j < v1 ? __ldcs(reinterpret_cast<const long long*>(values + j)) : 0;
+            }
+            map_hash_lookup4(tab, bits, v, r);
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const int64_t j = i + k * blockDim.x;
+                if (j < v1) __stcs(reinterpret_cast<long long*>(out + j), r[k]);
+            }
+        }
+    }
 }
 
 }  // namespace
@@ -391,7 +688,8 @@ ebag_status ebag_mapid_tbe(ebag_tbe* h, const int64_t* values, int64_t n_values,
                            const int64_t* mapping_len, int64_t B, int64_t* out, ebag_stream stream) {
     if (!h || !offsets || !mappings || !mapping_len || B < 0 || n_values < 0) return EBAG_ERR_INVALID_ARG;
     if (n_values > 0 && (!values || !out)) return EBAG_ERR_INVALID_ARG;
-    if ((int64_t)h->T * B >= (1ll << 31) || h->T > 65535) return EBAG_ERR_UNSUPPORTED;
+    if ((int64_t)h->T * B >= (1ll << 31) || h->T > kMapMaxTables) return EBAG_ERR_UNSUPPORTED;
+    if (n_values / kMapChunk + h->T >= (1ll << 31)) return EBAG_ERR_UNSUPPORTED;
     for (int t = 0; t < h->T; ++t) {
         if (mapping_len[t] < 0 || mapping_len[t] >= (1ll << 31)) return EBAG_ERR_INVALID_ARG;
         if (mapping_len[t] > 0 && (!mappings[t] || ((uintptr_t)mappings[t] & 7u))) return EBAG_ERR_INVALID_ARG;
@@ -404,13 +702,35 @@ ebag_status ebag_mapid_tbe(ebag_tbe* h, const int64_t* values, int64_t n_values,
     const void* const* d_block = nullptr;
     ebag_status st = stage_tables(h, no_tables.data(), mappings, mapping_len, (cudaStream_t)stream, &d_block);
     if (st != EBAG_OK) return st;
-    const int64_t per_table = (n_values + h->T - 1) / h->T;
-    int64_t bx = (per_table + 255) / 256;
-    const int64_t cap = (int64_t)h->num_sms * 16 / h->T + 1;
+    // enough CTAs to fill the device a few times over, never more than there are chunks
+    int64_t bx = n_values / kMapChunk + h->T;
+    const int64_t cap = (int64_t)h->num_sms * 8;
     if (bx > cap) bx = cap;
     if (bx < 1) bx = 1;
-    mapid_tbe_kernel<<<dim3((unsigned)bx, (unsigned)h->T), 256, 0, (cudaStream_t)stream>>>(
-        values, n_values, offsets, B, reinterpret_cast<const int64_t* const*>(d_block + h->T),
+    // With many more values than mapping entries a hash table of the mappings pays for itself.
+    int64_t hash_slots = 0, max_len = 0;
+    for (int t = 0; t < h->T; ++t) {
+        hash_slots += 1ll << map_hash_bits(mapping_len[t]);
+        if (mapping_len[t] > max_len) max_len = mapping_len[t];
+    }
+    if (h->mapid_hash && hash_slots <= kMapHashMaxSlots && n_values >= hash_slots && max_len > 0) {
+        if ((st = grow(h, &h->s_maphash, &h->cap_maphash, hash_slots)) != EBAG_OK) return st;
+        EBAG_CUDA(h, cudaMemsetAsync(h->s_maphash, 0, (size_t)hash_slots * sizeof(MapSlot), (cudaStream_t)stream));
+        int64_t gx = (max_len + 255) / 256;
+        if (gx > 64) gx = 64;
+        map_hash_build_kernel<<<dim3((unsigned)gx, (unsigned)h->T), 256, 0, (cudaStream_t)stream>>>(
+            h->T, reinterpret_cast<const int64_t* const*>(d_block + h->T),
+            reinterpret_cast<const int64_t*>(d_block + 2 * h->T), h->s_maphash);
+        EBAG_CUDA(h, cudaGetLastError());
+        mapid_tbe_hash_kernel<<<(unsigned)bx, 256, 0, (cudaStream_t)stream>>>(
+            values, n_values, offsets, B, h->T, reinterpret_cast<const int64_t*>(d_block + 2 * h->T),
+            h->s_maphash, out);
+        EBAG_CUDA(h, cudaGetLastError());
+        h->launches += 2;
+        return EBAG_OK;
+    }
+    mapid_tbe_kernel<<<(unsigned)bx, 256, 0, (cudaStream_t)stream>>>(
+        values, n_values, offsets, B, h->T, reinterpret_cast<const int64_t* const*>(d_block + h->T),
         reinterpret_cast<const int64_t*>(d_block + 2 * h->T), out);
     EBAG_CUDA(h, cudaGetLastError());
     ++h->launches;
@@ -422,11 +742,10 @@ ebag_status ebag_mapid(const int64_t* values, int64_t n, const int64_t* mapping,
     if (n < 0 || m < 0 || m >= (1ll << 31)) return EBAG_ERR_INVALID_ARG;
     if (n == 0) return EBAG_OK;
     if (!values || !out || (m > 0 && !mapping)) return EBAG_ERR_INVALID_ARG;
-    int steps = 0;
-    while ((1ll << steps) <= m) ++steps;             // bit length of m
-    int64_t blocks = (n + 255) / 256;
-    if (blocks > 148 * 16) blocks = 148 * 16;
-    mapid_kernel<<<(int)blocks, 256, 0, (cudaStream_t)stream>>>(values, n, mapping, (uint32_t)m, steps, out);
+    int64_t blocks = (n + 1023) / 1024;              // four values per thread and step
+    if (blocks > 148 * 8) blocks = 148 * 8;
+    if (blocks < 1) blocks = 1;
+    mapid_kernel<<<(int)blocks, 256, 0, (cudaStream_t)stream>>>(values, n, mapping, (uint32_t)m, out);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(nullptr, e);
     return EBAG_OK;
@@ -453,7 +772,7 @@ ebag_status ebag_forward_mapid(ebag_tbe* h, const void* const* tables, const int
     // Default: the transform for all tables in one launch into a scratch buffer of ids that the
     // handle keeps (grown when a larger call arrives), then the plain forward.  The searches are
     // chains of dependent loads; run between the stages of the forward's row pipeline they stall
-    // it, and the two kernels together are faster (3.25 against 3.82 ms on bench workload 6).
+    // it, and the separate launches together are faster (2.34 against 3.82 ms on bench workload 6).
     if (B == 0) return EBAG_OK;
     if ((st = grow(h, &h->s_indices, &h->cap_indices, n_values > 0 ? n_values : 1)) != EBAG_OK) return st;
     if (n_values > 0) {
@@ -822,6 +1141,11 @@ ebag_status ebag_set_param(ebag_tbe* h, const char* name, int64_t value) {
     if (std::strcmp(name, "mapid_fused") == 0) {
         if (value != 0 && value != 1) return EBAG_ERR_INVALID_ARG;
         h->mapid_fused = (int)value;
+        return EBAG_OK;
+    }
+    if (std::strcmp(name, "mapid_hash") == 0) {
+        if (value != 0 && value != 1) return EBAG_ERR_INVALID_ARG;
+        h->mapid_hash = (int)value;
         return EBAG_OK;
     }
     if (std::strcmp(name, "out_dtype") == 0) {

@@ -49,8 +49,8 @@ def test_mapid_degenerate_sizes():
 
 @pytest.mark.parametrize("dtype", [wl.F32, wl.BF16, wl.INT8_ROWWISE])
 @pytest.mark.parametrize("mode,weighted", [(wl.SUM, False), (wl.MEAN, False), (wl.SUM, True)])
-@pytest.mark.parametrize("fused", [0, 1])
-def test_fused_mapid_forward(dtype, mode, weighted, fused):
+@pytest.mark.parametrize("path", ["fused", "hash", "search"])
+def test_fused_mapid_forward(dtype, mode, weighted, path):
     rng = np.random.default_rng(31 + dtype)
     T, B = 5, 300
     Ds = {wl.F32: [64, 8, 256, 132, 32], wl.BF16: [64, 128, 256, 8, 1032],
@@ -83,11 +83,16 @@ def test_fused_mapid_forward(dtype, mode, weighted, fused):
     dev = pu.device_tables(dtype, tabs)
     dmaps = [torch.from_numpy(m).cuda() for m in mappings]
     tbe = eb.TBE(rows, Ds, dtype, device=torch.cuda.current_device())
-    tbe.set_param("mapid_fused", fused)       # 1: search inside the forward kernel; 0: two launches
+    # fused: search inside the forward kernel; else the transform runs first, through hash tables
+    # of the mappings (this call has more values than those tables have slots) or by binary search
+    tbe.set_param("mapid_fused", int(path == "fused"))
+    tbe.set_param("mapid_hash", int(path == "hash"))
+    before = tbe.launch_count()
     out = torch.full((B, sum(Ds)), float("nan"), dtype=torch.float32, device="cuda")
     tbe.forward_mapid(dev, torch.from_numpy(values).cuda(), torch.from_numpy(offsets).cuda(), dmaps, B,
                       mode, None if w is None else torch.from_numpy(w).cuda(), out=out)
     assert tbe.last_status() == (0, 0, 0)
+    assert tbe.launch_count() - before == {"fused": 2, "hash": 4, "search": 3}[path]   # the forward itself is two launches
     # the fused call equals MapId followed by the plain forward, bit for bit
     ids = torch.cat([eb.ebag_mapid(torch.from_numpy(vals[t]).cuda(), dmaps[t]) for t in range(T)])
     out2 = tbe.forward(dev, ids, torch.from_numpy(offsets).cuda(), B, mode,
@@ -116,3 +121,48 @@ def test_fused_mapid_rejects_bad_arguments_and_counts_rows_beyond_the_table():
         eb.ebag_forward_mapid(tbe._h, [tab.data_ptr()], [8], vals.data_ptr(), 4, off.data_ptr(), None,
                               [mapping.data_ptr()], [-1], 1, 0, out.data_ptr(), 0)
     tbe.close()
+
+
+@pytest.mark.parametrize("use_hash", [0, 1])
+def test_mapid_for_all_tables_with_duplicates_empty_mappings_and_extreme_values(use_hash):
+    """Equal keys in a mapping map to the first of their run on both paths; a table without a
+    mapping maps everything to 0; the extreme int64 values and 0 are ordinary keys."""
+    rng = np.random.default_rng(5 + use_hash)
+    B = 64
+    lo64, hi64 = np.iinfo(np.int64).min, np.iinfo(np.int64).max
+    mappings = [np.array([lo64, -7, -7, -7, 0, 0, 5, 9, 9, hi64], np.int64),
+                np.zeros(0, np.int64),
+                np.sort(rng.integers(-50_000, 50_000, size=30_000).astype(np.int64)),     # many duplicates
+                np.arange(0, 3 * 70_001, 3, dtype=np.int64),
+                np.array([42], np.int64)]
+    T = len(mappings)
+    lengths = rng.integers(0, 3000, size=T * B)     # more values than hash slots: the hash path is taken
+    offsets = np.zeros(T * B + 1, np.int64)
+    np.cumsum(lengths, out=offsets[1:])
+    vals = []
+    for t, m in enumerate(mappings):
+        n = int(offsets[(t + 1) * B] - offsets[t * B])
+        v = rng.integers(-60_000, 220_000, size=n).astype(np.int64)
+        if m.size:
+            hit = rng.random(n) < 0.5
+            v[hit] = m[rng.integers(0, m.size, size=int(hit.sum()))]
+        v[:3] = [lo64, hi64, 0]
+        vals.append(v)
+    values = np.concatenate(vals)
+    tbe = eb.TBE([8] * T, [8] * T, eb.EBAG_F32, device=torch.cuda.current_device())
+    tbe.set_param("mapid_hash", use_hash)
+    before = tbe.launch_count()
+    got = tbe.mapid(torch.from_numpy(values).cuda(), torch.from_numpy(offsets).cuda(),
+                    [torch.from_numpy(m).cuda() for m in mappings], B).cpu().numpy()
+    assert tbe.launch_count() - before == (2 if use_hash else 1)
+    tbe.close()
+    want = []
+    for t, m in enumerate(mappings):
+        if m.size and np.all(m[1:] > m[:-1]):
+            want.append(mo.mapid(vals[t], m))                 # the oracle's domain: strictly increasing
+        else:                                                 # outside it: position of the first equal entry
+            first = {}
+            for i, key in enumerate(m.tolist()):
+                first.setdefault(key, i + 1)
+            want.append(np.array([first.get(v, 0) for v in vals[t].tolist()], np.int64))
+    assert np.array_equal(got, np.concatenate(want))
