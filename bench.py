@@ -723,6 +723,11 @@ def main():
             tbe.forward_mapid(tables, d_raw, d_off, d_maps, w.B, w.mode, d_w, out=d_out, stream=stream)
             tbe.set_param("mapid_fused", 0)
 
+        def fused_binary_search():
+            tbe.set_param("mapid_hash", 0)
+            fused()
+            tbe.set_param("mapid_hash", 1)
+
         def mapid_only():
             tbe.mapid(d_raw, d_off, d_maps, w.B, out=ids, stream=stream)
 
@@ -746,6 +751,8 @@ def main():
 
         default_out = d_out.clone()
         mapid_extra = {"mapid_then_forward_ms": elapsed_ms / args.steps, "fused_ms": timed(fused)}
+        assert torch.equal(default_out, d_out), "fused MapId forward and the two-launch path disagree"
+        mapid_extra["fused_binary_search_ms"] = timed(fused_binary_search)
         assert torch.equal(default_out, d_out), "fused MapId forward and the two-launch path disagree"
         mapid_extra["mapid_alone_ms"] = timed(mapid_only)              # hash tables of the mappings
         assert torch.equal(ids, d_idx)

@@ -228,9 +228,10 @@ ebag_status ebag_mapid_tbe(ebag_tbe* h, const int64_t* values, int64_t n_values,
  * runs for all tables in one launch into a buffer of n_values ids that the handle keeps (it is
  * grown, with a device synchronisation, when a larger call arrives: the only allocation), and
  * the plain forward follows on the same stream.  With ebag_set_param("mapid_fused", 1) the
- * search runs inside the forward kernel instead, directly in front of the gather, so that the
- * mapped ids never travel through memory and nothing is allocated: less traffic, but measured
- * slower at the mapping sizes tried (the searches stall the row pipeline).  This is the
+ * look-up runs inside the forward kernel instead, directly in front of the gather, so that the
+ * mapped ids never travel through memory: less traffic, but measured slower at the mapping sizes
+ * tried (the look-ups stall the row pipeline).  Either way the ids are found through hash tables
+ * of the mappings when the call is large enough (see ebag_mapid_tbe), else by binary search.  This is the
  * producer of embedding ids the paper's preprocessing section describes.
  */
 ebag_status ebag_forward_mapid(ebag_tbe* h, const void* const* tables, const int32_t* D,

@@ -42,10 +42,6 @@ int elem_bytes(int dtype) { return dtype == EBAG_F32 ? 4 : (is_rowwise8(dtype) ?
 
 }  // namespace
 
-namespace {
-struct MapSlot;
-}
-
 struct ebag_tbe {
     int T = 0, dtype = 0, device = 0, sumD = 0, num_sms = 0;
     std::vector<int64_t> rows;
@@ -78,8 +74,10 @@ struct ebag_tbe {
     std::string cuda_error;
     // staging for ebag_forward_host
     int64_t* s_indices = nullptr;
-    MapSlot* s_maphash = nullptr;     // hash tables of the mappings of the MapId call in flight
+    ebag::MapSlot* s_maphash = nullptr;     // hash tables of the mappings of the MapId call in flight
     int64_t cap_maphash = 0;
+    uint32_t* d_map_base = nullptr;   // [T] first slot of every table's hash table (written by the build kernel)
+    int64_t cap_map_base = 0;
     int mapid_hash = 1;
     int64_t* s_offsets = nullptr;
     float* s_weights = nullptr;
@@ -129,6 +127,7 @@ void free_handle(ebag_tbe* h) {
     }
     cudaFree(h->s_indices);
     cudaFree(h->s_maphash);
+    cudaFree(h->d_map_base);
     cudaFree(h->s_offsets);
     cudaFree(h->s_weights);
     cudaFree(h->s_out);
@@ -222,6 +221,11 @@ ebag_status stage_tables(ebag_tbe* h, const void* const* tables, const int64_t* 
     return EBAG_OK;
 }
 
+// Builds the hash tables of a call's mappings in the handle's scratch when that pays (defined
+// with the MapId kernels below); *used says whether it did.
+ebag_status prepare_map_hash(ebag_tbe* h, const void* const* d_block, const int64_t* mapping_len,
+                             int64_t n_values, cudaStream_t stream, bool* used);
+
 // Launch on device pointers for bags [b0, b1) of every table; arguments already checked.
 // offsets and out are the buffers of the WHOLE call (B bags per table).
 ebag_status forward_device(ebag_tbe* h, const void* const* tables, const int64_t* indices,
@@ -251,6 +255,16 @@ ebag_status forward_device(ebag_tbe* h, const void* const* tables, const int64_t
     p.status = h->d_status;
     p.mappings = reinterpret_cast<const int64_t* const*>(d_tables + h->T);
     p.mapping_len = reinterpret_cast<const int64_t*>(d_tables + 2 * h->T);
+    p.map_slots = nullptr;
+    p.map_base = nullptr;
+    if (mappings) {   // fused MapId: look ids up through hash tables when the call pays for building them
+        bool hashed = false;
+        if ((st = prepare_map_hash(h, d_tables, mapping_len, n_indices, stream, &hashed)) != EBAG_OK) return st;
+        if (hashed) {
+            p.map_slots = h->s_maphash;
+            p.map_base = h->d_map_base;
+        }
+    }
     p.n_indices = n_indices;
     p.B = b1 - b0;
     p.off_stride = B;
@@ -533,20 +547,6 @@ mapid_tbe_kernel(const int64_t* __restrict__ values, int64_t n_values, const int
 // index + 1; linear probing; at most half full) and the searches become one or two loads each
 // instead of log2(|M|) dependent ones.  The result is the same as the binary search's for a
 // sorted mapping: equal keys are adjacent there and only the first of a run is inserted.
-struct __align__(16) MapSlot {
-    int64_t key;
-    uint32_t idx1;      // index + 1; 0 = empty
-    uint32_t pad;
-};
-constexpr uint64_t kHashMul = 0x9E3779B97F4A7C15ull;     // multiplicative (Fibonacci) hashing
-constexpr int64_t kMapHashMaxSlots = 1ll << 24;          // 256 MB of slots per handle at most
-
-__host__ __device__ inline uint32_t map_hash_bits(int64_t mlen) {
-    uint32_t bits = 1;
-    while (bits < 31 && (1ll << bits) < 2 * mlen) ++bits;
-    return bits;
-}
-
 // base slot of every table's hash table, in shared memory (T + 1 entries), by thread 0
 __device__ __forceinline__ void map_hash_bases(int T, const int64_t* __restrict__ mapping_len, uint32_t* hbase) {
     if (threadIdx.x == 0) {
@@ -562,7 +562,8 @@ __device__ __forceinline__ void map_hash_bases(int T, const int64_t* __restrict_
 
 __global__ void __launch_bounds__(256)
 map_hash_build_kernel(int T, const int64_t* const* __restrict__ mappings,
-                      const int64_t* __restrict__ mapping_len, MapSlot* __restrict__ slots) {
+                      const int64_t* __restrict__ mapping_len, MapSlot* __restrict__ slots,
+                      uint32_t* __restrict__ table_base) {
     __shared__ uint32_t base_s;
     const int t = blockIdx.y;
     const int64_t ml = mapping_len[t];
@@ -573,6 +574,7 @@ map_hash_build_kernel(int T, const int64_t* const* __restrict__ mappings,
             at += 1u << map_hash_bits(l < 0 ? 0 : l);
         }
         base_s = at;
+        if (blockIdx.x == 0) table_base[t] = at;             // for the forward kernel's fused look-up
     }
     __syncthreads();
     if (ml <= 0) return;
@@ -679,6 +681,31 @@ mapid_tbe_hash_kernel(const int64_t* __restrict__ values, int64_t n_values, cons
     }
 }
 
+// With many more values than mapping entries a hash table of the mappings pays for itself.
+ebag_status prepare_map_hash(ebag_tbe* h, const void* const* d_block, const int64_t* mapping_len,
+                             int64_t n_values, cudaStream_t stream, bool* used) {
+    *used = false;
+    int64_t hash_slots = 0, max_len = 0;
+    for (int t = 0; t < h->T; ++t) {
+        hash_slots += 1ll << map_hash_bits(mapping_len[t]);
+        if (mapping_len[t] > max_len) max_len = mapping_len[t];
+    }
+    if (!h->mapid_hash || hash_slots > kMapHashMaxSlots || n_values < hash_slots || max_len <= 0) return EBAG_OK;
+    ebag_status st;
+    if ((st = grow(h, &h->s_maphash, &h->cap_maphash, hash_slots)) != EBAG_OK) return st;
+    if ((st = grow(h, &h->d_map_base, &h->cap_map_base, (int64_t)h->T)) != EBAG_OK) return st;
+    EBAG_CUDA(h, cudaMemsetAsync(h->s_maphash, 0, (size_t)hash_slots * sizeof(MapSlot), stream));
+    int64_t gx = (max_len + 255) / 256;
+    if (gx > 64) gx = 64;
+    map_hash_build_kernel<<<dim3((unsigned)gx, (unsigned)h->T), 256, 0, stream>>>(
+        h->T, reinterpret_cast<const int64_t* const*>(d_block + h->T),
+        reinterpret_cast<const int64_t*>(d_block + 2 * h->T), h->s_maphash, h->d_map_base);
+    EBAG_CUDA(h, cudaGetLastError());
+    ++h->launches;
+    *used = true;
+    return EBAG_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -707,26 +734,14 @@ ebag_status ebag_mapid_tbe(ebag_tbe* h, const int64_t* values, int64_t n_values,
     const int64_t cap = (int64_t)h->num_sms * 8;
     if (bx > cap) bx = cap;
     if (bx < 1) bx = 1;
-    // With many more values than mapping entries a hash table of the mappings pays for itself.
-    int64_t hash_slots = 0, max_len = 0;
-    for (int t = 0; t < h->T; ++t) {
-        hash_slots += 1ll << map_hash_bits(mapping_len[t]);
-        if (mapping_len[t] > max_len) max_len = mapping_len[t];
-    }
-    if (h->mapid_hash && hash_slots <= kMapHashMaxSlots && n_values >= hash_slots && max_len > 0) {
-        if ((st = grow(h, &h->s_maphash, &h->cap_maphash, hash_slots)) != EBAG_OK) return st;
-        EBAG_CUDA(h, cudaMemsetAsync(h->s_maphash, 0, (size_t)hash_slots * sizeof(MapSlot), (cudaStream_t)stream));
-        int64_t gx = (max_len + 255) / 256;
-        if (gx > 64) gx = 64;
-        map_hash_build_kernel<<<dim3((unsigned)gx, (unsigned)h->T), 256, 0, (cudaStream_t)stream>>>(
-            h->T, reinterpret_cast<const int64_t* const*>(d_block + h->T),
-            reinterpret_cast<const int64_t*>(d_block + 2 * h->T), h->s_maphash);
-        EBAG_CUDA(h, cudaGetLastError());
+    bool hashed = false;
+    if ((st = prepare_map_hash(h, d_block, mapping_len, n_values, (cudaStream_t)stream, &hashed)) != EBAG_OK) return st;
+    if (hashed) {
         mapid_tbe_hash_kernel<<<(unsigned)bx, 256, 0, (cudaStream_t)stream>>>(
             values, n_values, offsets, B, h->T, reinterpret_cast<const int64_t*>(d_block + 2 * h->T),
             h->s_maphash, out);
         EBAG_CUDA(h, cudaGetLastError());
-        h->launches += 2;
+        ++h->launches;
         return EBAG_OK;
     }
     mapid_tbe_kernel<<<(unsigned)bx, 256, 0, (cudaStream_t)stream>>>(

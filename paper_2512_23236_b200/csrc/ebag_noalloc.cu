@@ -194,6 +194,8 @@ extern "C" ebag_status ebag_forward_noalloc(int32_t T, const int64_t* rows, cons
     p.queue = &st->scratch->queue;
     p.mappings = nullptr;
     p.mapping_len = nullptr;
+    p.map_slots = nullptr;
+    p.map_base = nullptr;
     p.status = status_counts ? reinterpret_cast<Status*>(status_counts) : &st->scratch->status;
     p.n_indices = n_indices;
     p.B = B;

@@ -49,7 +49,7 @@ def test_mapid_degenerate_sizes():
 
 @pytest.mark.parametrize("dtype", [wl.F32, wl.BF16, wl.INT8_ROWWISE])
 @pytest.mark.parametrize("mode,weighted", [(wl.SUM, False), (wl.MEAN, False), (wl.SUM, True)])
-@pytest.mark.parametrize("path", ["fused", "hash", "search"])
+@pytest.mark.parametrize("path", ["fused", "fused_hash", "hash", "search"])
 def test_fused_mapid_forward(dtype, mode, weighted, path):
     rng = np.random.default_rng(31 + dtype)
     T, B = 5, 300
@@ -85,14 +85,14 @@ def test_fused_mapid_forward(dtype, mode, weighted, path):
     tbe = eb.TBE(rows, Ds, dtype, device=torch.cuda.current_device())
     # fused: search inside the forward kernel; else the transform runs first, through hash tables
     # of the mappings (this call has more values than those tables have slots) or by binary search
-    tbe.set_param("mapid_fused", int(path == "fused"))
-    tbe.set_param("mapid_hash", int(path == "hash"))
+    tbe.set_param("mapid_fused", int(path.startswith("fused")))
+    tbe.set_param("mapid_hash", int(path.endswith("hash")))
     before = tbe.launch_count()
     out = torch.full((B, sum(Ds)), float("nan"), dtype=torch.float32, device="cuda")
     tbe.forward_mapid(dev, torch.from_numpy(values).cuda(), torch.from_numpy(offsets).cuda(), dmaps, B,
                       mode, None if w is None else torch.from_numpy(w).cuda(), out=out)
     assert tbe.last_status() == (0, 0, 0)
-    assert tbe.launch_count() - before == {"fused": 2, "hash": 4, "search": 3}[path]   # the forward itself is two launches
+    assert tbe.launch_count() - before == {"fused": 2, "fused_hash": 3, "hash": 4, "search": 3}[path]   # the forward itself is two launches
     # the fused call equals MapId followed by the plain forward, bit for bit
     ids = torch.cat([eb.ebag_mapid(torch.from_numpy(vals[t]).cuda(), dmaps[t]) for t in range(T)])
     out2 = tbe.forward(dev, ids, torch.from_numpy(offsets).cuda(), B, mode,
