@@ -18,8 +18,9 @@
 // queues on them (measured: 13 times slower than uniform ids).  So a first, small kernel samples
 // the ids of every table and puts its most frequent rows into a small hashed table of K slots
 // (K = 2048 / D, at most 32); every warp of the main kernel sums the contributions to those
-// rows in its own 8 KB of shared memory and sends each sum to L2 once per table it passes
-// through.
+// rows in its own 8 KB of shared memory (plain loads and stores: a lane owns its columns, and
+// groups of lanes that hit one row at the same step take turns) and sends each sum to L2 once
+// per table it passes through.
 //
 // The order in which the contributions to a row arrive is not fixed, so results are
 // reproducible only up to fp32 rounding.  Ids outside the table and malformed bags are skipped
@@ -189,6 +190,7 @@ __global__ void __launch_bounds__(kBwdThreads) ebag_bwd_kernel(const BwdParams p
         }
         const int G = 1 << m.g_log2, ng = 32 >> m.g_log2;
         const int lig = lane & (G - 1), grp = lane >> m.g_log2;
+        const unsigned leaders = ng > 1 ? 0xffffffffu / ((1u << G) - 1u) : 1u;   // first lane of every group
         const int64_t b = (item - item_base[t]) * ng + grp;
         int64_t lo = 0, hi = 0;
         if (b < p.B) {
@@ -235,36 +237,49 @@ __global__ void __launch_bounds__(kBwdThreads) ebag_bwd_kernel(const BwdParams p
                         if (WEIGHTED) w[k] = __ldg(p.weights + i);
                     }
                 }
+                auto add_hot = [&](int slot, int k) {
+                    float* crow = cache + (size_t)slot * m.D;
+#pragma unroll
+                    for (int v = 0; v < kTileVecs; ++v)
+                        if (on[v]) {
+                            float4* a = reinterpret_cast<float4*>(crow + (size_t)(c0 + v * G + lig) * 4);
+                            const float ww = WEIGHTED ? w[k] : 1.0f;
+                            float4 c = *a;
+                            c.x += ww * gv[v].x; c.y += ww * gv[v].y; c.z += ww * gv[v].z; c.w += ww * gv[v].w;
+                            *a = c;
+                        }
+                };
 #pragma unroll
                 for (int k = 0; k < kIdBatch; ++k) {
-                    if (j0 + k >= L) continue;
-                    if ((uint64_t)r[k] >= (uint64_t)m.rows) {
-                        if (lig == 0 && c0 == 0) ++n_oob;
-                        continue;
-                    }
+                    // (no lane leaves this iteration early: the groups of a warp vote below)
+                    const bool live = j0 + k < L;
+                    const bool valid = live && (uint64_t)r[k] < (uint64_t)m.rows;
+                    if (live && !valid && lig == 0 && c0 == 0) ++n_oob;
                     int slot = -1;
-                    if (cur_K > 0) {
+                    if (valid && cur_K > 0) {
                         const int h1 = hot_slot((uint32_t)r[k], cur_K), h2 = hot_slot2((uint32_t)r[k], cur_K);
                         if (hot_s[h1] == (int)r[k]) slot = h1;
                         else if (hot_s[h2] == (int)r[k]) slot = h2;
                     }
-                    if (slot >= 0) {
-                        // a hot row: summed here, in this warp's shared memory (several groups of
-                        // the warp may hit the same row at once, hence the atomics)
-                        if (lig == 0) hot_s[kHotSlots + slot] = 1;
-                        float* crow = cache + (size_t)slot * m.D;
-#pragma unroll
-                        for (int v = 0; v < kTileVecs; ++v)
-                            if (on[v]) {
-                                float* a = crow + (size_t)(c0 + v * G + lig) * 4;
-                                const float ww = WEIGHTED ? w[k] : 1.0f;
-                                atomicAdd(a + 0, ww * gv[v].x);
-                                atomicAdd(a + 1, ww * gv[v].y);
-                                atomicAdd(a + 2, ww * gv[v].z);
-                                atomicAdd(a + 3, ww * gv[v].w);
+                    // A hot row is summed here, in this warp's shared memory.  A lane owns its
+                    // columns, so within one group of lanes the sums need no atomics; groups that
+                    // run side by side and hit the same row at the same step take turns.
+                    if (slot >= 0 && lig == 0) hot_s[kHotSlots + slot] = 1;
+                    if (ng > 1) {
+                        if (__any_sync(0xffffffffu, slot >= 0)) {
+                            const unsigned same = __match_any_sync(0xffffffffu, slot);
+                            // groups before mine that want the same slot
+                            const int rank = slot >= 0 ? __popc(same & leaders & ((1u << (grp << m.g_log2)) - 1u)) : 0;
+                            const int turns = __reduce_max_sync(0xffffffffu, (unsigned)rank);
+                            for (int turn = 0; turn <= turns; ++turn) {
+                                if (slot >= 0 && rank == turn) add_hot(slot, k);
+                                __syncwarp();
                             }
-                        continue;
+                        }
+                    } else if (slot >= 0) {
+                        add_hot(slot, k);
                     }
+                    if (slot >= 0 || !valid) continue;
                     float* row = gt + r[k] * (int64_t)m.D;
 #pragma unroll
                     for (int v = 0; v < kTileVecs; ++v)
