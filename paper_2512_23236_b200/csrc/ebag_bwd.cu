@@ -123,7 +123,7 @@ __global__ void __launch_bounds__(kBwdThreads) bwd_hot_rows_kernel(const BwdPara
 }
 
 template <bool WEIGHTED>
-__global__ void __launch_bounds__(kBwdThreads) ebag_bwd_kernel(const BwdParams p) {
+__global__ void __launch_bounds__(kBwdThreads, 3) ebag_bwd_kernel(const BwdParams p) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     // per warp: kCacheFloats floats of sums, then kHotSlots ids and kHotSlots flags; after all
     // warps: item_base[T+1]
@@ -224,19 +224,31 @@ __global__ void __launch_bounds__(kBwdThreads) ebag_bwd_kernel(const BwdParams p
                     }
                 }
             }
+            // the ids of the next batch are requested before the current batch is worked on
+            int64_t rn[kIdBatch];
+            float wn[kIdBatch];
+            auto fetch = [&](int64_t j0) {
+#pragma unroll
+                for (int k = 0; k < kIdBatch; ++k) {
+                    const int64_t i = lo + j0 + k;
+                    rn[k] = -1;
+                    wn[k] = 1.0f;
+                    if (j0 + k < L) {
+                        rn[k] = load_id(p.indices, p.idx32, i);
+                        if (WEIGHTED) wn[k] = __ldg(p.weights + i);
+                    }
+                }
+            };
+            fetch(0);
             for (int64_t j0 = 0; j0 < Lmax; j0 += kIdBatch) {
                 int64_t r[kIdBatch];
                 float w[kIdBatch];
 #pragma unroll
                 for (int k = 0; k < kIdBatch; ++k) {
-                    const int64_t i = lo + j0 + k;
-                    r[k] = -1;
-                    w[k] = 1.0f;
-                    if (j0 + k < L) {
-                        r[k] = load_id(p.indices, p.idx32, i);
-                        if (WEIGHTED) w[k] = __ldg(p.weights + i);
-                    }
+                    r[k] = rn[k];
+                    w[k] = wn[k];
                 }
+                fetch(j0 + kIdBatch);
                 auto add_hot = [&](int slot, int k) {
                     float* crow = cache + (size_t)slot * m.D;
 #pragma unroll
