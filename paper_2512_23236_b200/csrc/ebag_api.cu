@@ -472,6 +472,33 @@ mapid_kernel(const int64_t* __restrict__ values, int64_t n, const int64_t* __res
                 (int64_t)gridDim.x * blockDim.x, pivots);
 }
 
+// Prefix sums over a[0..n) in shared memory, in place, by a CTA of 256 threads: a[i] becomes
+// a[0] + ... + a[i].  Every thread takes a run of consecutive entries.  Ends with a barrier.
+__device__ __forceinline__ void block_scan_inclusive(uint32_t* a, int n) {
+    __shared__ uint32_t warp_total[8];
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    const int per = (n + 255) / 256;
+    const int i0 = threadIdx.x * per;
+    const int i1 = i0 + per < n ? i0 + per : n;
+    uint32_t sum = 0;
+    for (int i = i0; i < i1; ++i) sum += a[i];
+    uint32_t x = sum;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const uint32_t y = __shfl_up_sync(0xffffffffu, x, d);
+        if (lane >= d) x += y;
+    }
+    if (lane == 31) warp_total[wid] = x;
+    __syncthreads();
+    uint32_t run = x - sum;
+    for (int w = 0; w < wid; ++w) run += warp_total[w];
+    for (int i = i0; i < i1; ++i) {
+        run += a[i];
+        a[i] = run;
+    }
+    __syncthreads();
+}
+
 // MapId for all tables of a TBE call in one launch.  The tables' slices of the jagged value list
 // are read from the offsets array on the device (no host synchronisation) and cut into chunks of
 // kMapChunk values; every CTA takes an equal run of consecutive chunks, so the work is balanced
@@ -491,12 +518,9 @@ mapid_tbe_kernel(const int64_t* __restrict__ values, int64_t n_values, const int
         if (hi > n_values) hi = n_values;
         chunk_base[t + 1] = hi > lo ? (int)((hi - lo + kMapChunk - 1) / kMapChunk) : 0;
     }
+    if (threadIdx.x == 0) chunk_base[0] = 0;
     __syncthreads();
-    if (threadIdx.x == 0) {
-        chunk_base[0] = 0;
-        for (int t = 0; t < T; ++t) chunk_base[t + 1] += chunk_base[t];
-    }
-    __syncthreads();
+    block_scan_inclusive(reinterpret_cast<uint32_t*>(chunk_base), T + 1);
     const int total = chunk_base[T];
     const int per_cta = (total + gridDim.x - 1) / gridDim.x;
     const int c0 = blockIdx.x * per_cta;
@@ -547,17 +571,14 @@ mapid_tbe_kernel(const int64_t* __restrict__ values, int64_t n_values, const int
 // index + 1; linear probing; at most half full) and the searches become one or two loads each
 // instead of log2(|M|) dependent ones.  The result is the same as the binary search's for a
 // sorted mapping: equal keys are adjacent there and only the first of a run is inserted.
-// base slot of every table's hash table, in shared memory (T + 1 entries), by thread 0
-__device__ __forceinline__ void map_hash_bases(int T, const int64_t* __restrict__ mapping_len, uint32_t* hbase) {
-    if (threadIdx.x == 0) {
-        uint32_t at = 0;
-        for (int t = 0; t < T; ++t) {
-            hbase[t] = at;
-            const int64_t ml = mapping_len[t];
-            at += 1u << map_hash_bits(ml < 0 ? 0 : ml);
-        }
-        hbase[T] = at;
+// slots of every table's hash table into hbase[t + 1], hbase[0] = 0: after a prefix sum over
+// the T + 1 entries hbase[t] is the first slot of table t
+__device__ __forceinline__ void map_hash_sizes(int T, const int64_t* __restrict__ mapping_len, uint32_t* hbase) {
+    for (int t = threadIdx.x; t < T; t += blockDim.x) {
+        const int64_t ml = mapping_len[t];
+        hbase[t + 1] = 1u << map_hash_bits(ml < 0 ? 0 : ml);
     }
+    if (threadIdx.x == 0) hbase[0] = 0;
 }
 
 __global__ void __launch_bounds__(256)
@@ -567,16 +588,17 @@ map_hash_build_kernel(int T, const int64_t* const* __restrict__ mappings,
     __shared__ uint32_t base_s;
     const int t = blockIdx.y;
     const int64_t ml = mapping_len[t];
-    if (threadIdx.x == 0) {
-        uint32_t at = 0;
-        for (int u = 0; u < t; ++u) {
-            const int64_t l = mapping_len[u];
-            at += 1u << map_hash_bits(l < 0 ? 0 : l);
-        }
-        base_s = at;
-        if (blockIdx.x == 0) table_base[t] = at;             // for the forward kernel's fused look-up
-    }
+    if (threadIdx.x == 0) base_s = 0;
     __syncthreads();
+    uint32_t part = 0;                                       // slots of the tables before this one
+    for (int u = threadIdx.x; u < t; u += blockDim.x) {
+        const int64_t l = mapping_len[u];
+        part += 1u << map_hash_bits(l < 0 ? 0 : l);
+    }
+    part = __reduce_add_sync(0xffffffffu, part);
+    if ((threadIdx.x & 31) == 0 && part) atomicAdd(&base_s, part);
+    __syncthreads();
+    if (threadIdx.x == 0 && blockIdx.x == 0) table_base[t] = base_s;   // for the forward kernel's fused look-up
     if (ml <= 0) return;
     const uint32_t bits = map_hash_bits(ml), mask = (1u << bits) - 1u;
     MapSlot* tab = slots + base_s;
@@ -638,13 +660,11 @@ mapid_tbe_hash_kernel(const int64_t* __restrict__ values, int64_t n_values, cons
         if (hi > n_values) hi = n_values;
         chunk_base[t + 1] = hi > lo ? (int)((hi - lo + kMapChunk - 1) / kMapChunk) : 0;
     }
-    map_hash_bases(T, mapping_len, hbase);
+    map_hash_sizes(T, mapping_len, hbase);
+    if (threadIdx.x == 0) chunk_base[0] = 0;
     __syncthreads();
-    if (threadIdx.x == 0) {
-        chunk_base[0] = 0;
-        for (int t = 0; t < T; ++t) chunk_base[t + 1] += chunk_base[t];
-    }
-    __syncthreads();
+    block_scan_inclusive(reinterpret_cast<uint32_t*>(chunk_base), T + 1);
+    block_scan_inclusive(hbase, T + 1);
     const int total = chunk_base[T];
     const int per_cta = (total + gridDim.x - 1) / gridDim.x;
     const int c0 = blockIdx.x * per_cta;

@@ -166,3 +166,31 @@ def test_mapid_for_all_tables_with_duplicates_empty_mappings_and_extreme_values(
                 first.setdefault(key, i + 1)
             want.append(np.array([first.get(v, 0) for v in vals[t].tolist()], np.int64))
     assert np.array_equal(got, np.concatenate(want))
+
+
+@pytest.mark.parametrize("use_hash", [0, 1])
+def test_mapid_for_many_small_tables(use_hash):
+    """More tables than threads in a CTA (the per-table chunk and hash-table offsets are prefix
+    sums taken by the whole CTA), mapping sizes from 0 to a few hundred, some tables without values."""
+    rng = np.random.default_rng(77)
+    T, B = 700, 24
+    mappings = []
+    for t in range(T):
+        m = int(rng.integers(0, 300)) if t % 7 else 0
+        mappings.append(np.sort(rng.choice(np.arange(-1000, 5000, dtype=np.int64), size=m, replace=False)))
+    lengths = rng.integers(0, 40, size=T * B)
+    lengths[5 * B:9 * B] = 0                                # four tables in a row without values
+    offsets = np.zeros(T * B + 1, np.int64)
+    np.cumsum(lengths, out=offsets[1:])
+    values = rng.integers(-1200, 5200, size=int(offsets[-1])).astype(np.int64)
+    tbe = eb.TBE([8] * T, [8] * T, eb.EBAG_F32, device=torch.cuda.current_device())
+    tbe.set_param("mapid_hash", use_hash)
+    before = tbe.launch_count()
+    got = tbe.mapid(torch.from_numpy(values).cuda(), torch.from_numpy(offsets).cuda(),
+                    [torch.from_numpy(m).cuda() for m in mappings], B).cpu().numpy()
+    assert tbe.launch_count() - before == (2 if use_hash else 1)
+    tbe.close()
+    for t in range(T):
+        lo, hi = int(offsets[t * B]), int(offsets[(t + 1) * B])
+        want = mo.mapid(values[lo:hi], mappings[t]) if mappings[t].size else np.zeros(hi - lo, np.int64)
+        assert np.array_equal(got[lo:hi], want), t
