@@ -8,13 +8,13 @@ namespace {
 
 constexpr int kThreads = 256;
 constexpr int kSmemBorders = 64;     // border lists up to this long are counted linearly from smem
-constexpr int kIlp = 8;              // values per thread in flight (8 x 4 B x 2048 threads = 64 KB per SM)
+constexpr int kIlp = 16;             // values per thread in flight (8 and 32 measured slower: 0.169 and 0.253 ms against 0.154)
 
 // MergeBucketizedDense (Sec. 5.4.2): out[f, i] = #borders of feature f below values[f, i] + off[f].
 // blockIdx.y is the feature.  "Below" is written !(x <= b) so that NaN lands in the last bin,
 // like the library routine the paper's pseudocode calls.  Short lists are counted linearly
 // (the vectorised counting the paper's kernel uses), long ones by a branch-free halving search.
-template <bool VEC>       // VEC: B is a multiple of 4 and both arrays are 16-byte aligned
+template <bool VEC>       // VEC: B is even, values 8-byte and out 16-byte aligned
 __global__ void __launch_bounds__(kThreads)
 mbdt_kernel(const float* __restrict__ values, int64_t B, const float* __restrict__ borders,
             const int64_t* __restrict__ border_offsets, const int64_t* __restrict__ out_offsets,
@@ -53,35 +53,39 @@ mbdt_kernel(const float* __restrict__ values, int64_t B, const float* __restrict
         return lo;
     };
     if (VEC) {
-        // four consecutive values per thread and step: one 16-byte load, two 16-byte stores
-        const int64_t B4 = B >> 2;
-        const float4* __restrict__ v4 = reinterpret_cast<const float4*>(vf);
+        // two consecutive values per thread and access: 8-byte loads, 16-byte stores, so that a
+        // warp's store covers 512 contiguous bytes (with four values per thread every 32-byte
+        // sector of the output was written in two halves by two store instructions)
+        const int64_t B2 = B >> 1;
+        const float2* __restrict__ v2 = reinterpret_cast<const float2*>(vf);
         longlong2* __restrict__ o2 = reinterpret_cast<longlong2*>(of);
-        for (int64_t i = blockIdx.x * (int64_t)kThreads + threadIdx.x; i < B4; i += 2 * stride) {
-            const bool second = i + stride < B4;
-            const float4 a = __ldcs(v4 + i);
-            float4 c = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (second) c = __ldcs(v4 + i + stride);
-            const float x[8] = {a.x, a.y, a.z, a.w, c.x, c.y, c.z, c.w};
-            int n[8];
+        constexpr int kPairs = kIlp / 2;
+        for (int64_t i = blockIdx.x * (int64_t)kThreads + threadIdx.x; i < B2; i += kPairs * stride) {
+            float x[kIlp];
+#pragma unroll
+            for (int q = 0; q < kPairs; ++q) {
+                float2 a = make_float2(0.f, 0.f);
+                if (i + q * stride < B2) a = __ldcs(v2 + i + q * stride);
+                x[2 * q] = a.x;
+                x[2 * q + 1] = a.y;
+            }
+            int n[kIlp];
             if (K <= kSmemBorders) {
 #pragma unroll
-                for (int k = 0; k < 8; ++k) n[k] = 0;
+                for (int k = 0; k < kIlp; ++k) n[k] = 0;
                 for (int j = 0; j < K; ++j) {
                     const float b = sb[j];
 #pragma unroll
-                    for (int k = 0; k < 8; ++k) n[k] += !(x[k] <= b);
+                    for (int k = 0; k < kIlp; ++k) n[k] += !(x[k] <= b);
                 }
             } else {
 #pragma unroll
-                for (int k = 0; k < 8; ++k) n[k] = bin(x[k]);
+                for (int k = 0; k < kIlp; ++k) n[k] = bin(x[k]);
             }
-            __stcs(o2 + 2 * i, make_longlong2(n[0] + add, n[1] + add));
-            __stcs(o2 + 2 * i + 1, make_longlong2(n[2] + add, n[3] + add));
-            if (second) {
-                __stcs(o2 + 2 * (i + stride), make_longlong2(n[4] + add, n[5] + add));
-                __stcs(o2 + 2 * (i + stride) + 1, make_longlong2(n[6] + add, n[7] + add));
-            }
+#pragma unroll
+            for (int q = 0; q < kPairs; ++q)
+                if (i + q * stride < B2)
+                    __stcs(o2 + i + q * stride, make_longlong2(n[2 * q] + add, n[2 * q + 1] + add));
         }
         return;
     }
@@ -128,7 +132,7 @@ extern "C" ebag_status ebag_mbdt(const float* values, int32_t F, int64_t B, cons
     int64_t cap = (int64_t)sms * per_sm / F;
     if (cap < 1) cap = 1;
     if (bx > cap) bx = cap;
-    const bool vec = (B & 3) == 0 && !((uintptr_t)values & 15u) && !((uintptr_t)out & 15u);
+    const bool vec = (B & 1) == 0 && !((uintptr_t)values & 7u) && !((uintptr_t)out & 15u);
     if (vec)
         mbdt_kernel<true><<<dim3((unsigned)bx, (unsigned)F), kThreads, 0, (cudaStream_t)stream>>>(
             values, B, borders, border_offsets, out_offsets, out);
