@@ -174,6 +174,12 @@ __device__ __forceinline__ uint32_t pack16(float lo, float hi, int kind) {
     else asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
     return r;
 }
+// 32 bytes in one instruction (a whole sector; the address must be 32-byte aligned)
+__device__ __forceinline__ void st_stream32(float* p, float2 a, float2 b, float2 c, float2 d) {
+    asm volatile("st.global.cs.v8.f32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(p), "f"(a.x), "f"(a.y),
+                 "f"(b.x), "f"(b.y), "f"(c.x), "f"(c.y), "f"(d.x), "f"(d.y)
+                 : "memory");
+}
 __device__ __forceinline__ void st_stream16(float* p, float a, float b, float c, float d) {
     __stcs(reinterpret_cast<float4*>(p), make_float4(a, b, c, d));
 }
@@ -744,9 +750,22 @@ __device__ __forceinline__ void process_item(const FwdParams& p, const TableMeta
                     acc[v][a] = x;
                 }
                 if (PART || p.out16 == 0) {
+                    // 16- and 8-bit tables: a lane holds one or two whole 32-byte sectors of the
+                    // row; written 16 bytes at a time every store instruction of the warp would
+                    // write half of each sector it touches
+                    bool wide = false;
+                    if constexpr (NACC >= 8) wide = (reinterpret_cast<uintptr_t>(o) & 31u) == 0;
+                    if (wide) {
+                        if constexpr (NACC >= 8) {
 #pragma unroll
-                    for (int a = 0; a < NACC / 2; a += 2)
-                        st_stream16(o + 2 * a, acc[v][a].x, acc[v][a].y, acc[v][a + 1].x, acc[v][a + 1].y);
+                            for (int a = 0; a < NACC / 2; a += 4)
+                                st_stream32(o + 2 * a, acc[v][a], acc[v][a + 1], acc[v][a + 2], acc[v][a + 3]);
+                        }
+                    } else {
+#pragma unroll
+                        for (int a = 0; a < NACC / 2; a += 2)
+                            st_stream16(o + 2 * a, acc[v][a].x, acc[v][a].y, acc[v][a + 1].x, acc[v][a + 1].y);
+                    }
                 } else {
                     // 16-bit output: the same elements, half the bytes
                     uint32_t* o16 = reinterpret_cast<uint32_t*>(p.out) +
