@@ -776,6 +776,13 @@ __device__ __forceinline__ void process_item(const FwdParams& p, const TableMeta
                     for (int a = 0; a < NACC / 2; ++a) wd[a] = pack16(acc[v][a].x, acc[v][a].y, p.out16);
                     if constexpr (NACC == 4) {
                         __stcs(reinterpret_cast<uint2*>(o16), make_uint2(wd[0], wd[1]));
+                    } else if (NACC == 16 && (reinterpret_cast<uintptr_t>(o16) & 31u) == 0) {
+                        // 8-bit tables: the lane's 16 elements are one whole sector
+                        if constexpr (NACC == 16)
+                            asm volatile("st.global.cs.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(o16),
+                                         "r"(wd[0]), "r"(wd[1]), "r"(wd[2]), "r"(wd[3]), "r"(wd[4]), "r"(wd[5]),
+                                         "r"(wd[6]), "r"(wd[7])
+                                         : "memory");
                     } else {
 #pragma unroll
                         for (int a = 0; a < NACC / 2; a += 4)

@@ -14,7 +14,7 @@ constexpr int kIlp = 16;             // values per thread in flight (8 and 32 me
 // blockIdx.y is the feature.  "Below" is written !(x <= b) so that NaN lands in the last bin,
 // like the library routine the paper's pseudocode calls.  Short lists are counted linearly
 // (the vectorised counting the paper's kernel uses), long ones by a branch-free halving search.
-template <bool VEC>       // VEC: B is even, values 8-byte and out 16-byte aligned
+template <bool VEC>       // VEC: B is a multiple of 4, values 16-byte and out 32-byte aligned
 __global__ void __launch_bounds__(kThreads)
 mbdt_kernel(const float* __restrict__ values, int64_t B, const float* __restrict__ borders,
             const int64_t* __restrict__ border_offsets, const int64_t* __restrict__ out_offsets,
@@ -53,21 +53,22 @@ mbdt_kernel(const float* __restrict__ values, int64_t B, const float* __restrict
         return lo;
     };
     if (VEC) {
-        // two consecutive values per thread and access: 8-byte loads, 16-byte stores, so that a
-        // warp's store covers 512 contiguous bytes (with four values per thread every 32-byte
-        // sector of the output was written in two halves by two store instructions)
-        const int64_t B2 = B >> 1;
-        const float2* __restrict__ v2 = reinterpret_cast<const float2*>(vf);
-        longlong2* __restrict__ o2 = reinterpret_cast<longlong2*>(of);
-        constexpr int kPairs = kIlp / 2;
-        for (int64_t i = blockIdx.x * (int64_t)kThreads + threadIdx.x; i < B2; i += kPairs * stride) {
+        // four consecutive values per thread and access: one 16-byte load, one 32-byte store (a
+        // whole sector per lane; two 16-byte stores per lane would each write half of every sector
+        // the warp touches: 0.186 ms against 0.154 ms with dense stores)
+        const int64_t B4 = B >> 2;
+        const float4* __restrict__ v4 = reinterpret_cast<const float4*>(vf);
+        constexpr int kQuads = kIlp / 4;
+        for (int64_t i = blockIdx.x * (int64_t)kThreads + threadIdx.x; i < B4; i += kQuads * stride) {
             float x[kIlp];
 #pragma unroll
-            for (int q = 0; q < kPairs; ++q) {
-                float2 a = make_float2(0.f, 0.f);
-                if (i + q * stride < B2) a = __ldcs(v2 + i + q * stride);
-                x[2 * q] = a.x;
-                x[2 * q + 1] = a.y;
+            for (int q = 0; q < kQuads; ++q) {
+                float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (i + q * stride < B4) a = __ldcs(v4 + i + q * stride);
+                x[4 * q] = a.x;
+                x[4 * q + 1] = a.y;
+                x[4 * q + 2] = a.z;
+                x[4 * q + 3] = a.w;
             }
             int n[kIlp];
             if (K <= kSmemBorders) {
@@ -83,9 +84,12 @@ mbdt_kernel(const float* __restrict__ values, int64_t B, const float* __restrict
                 for (int k = 0; k < kIlp; ++k) n[k] = bin(x[k]);
             }
 #pragma unroll
-            for (int q = 0; q < kPairs; ++q)
-                if (i + q * stride < B2)
-                    __stcs(o2 + i + q * stride, make_longlong2(n[2 * q] + add, n[2 * q + 1] + add));
+            for (int q = 0; q < kQuads; ++q)
+                if (i + q * stride < B4)
+                    asm volatile("st.global.cs.v4.b64 [%0], {%1, %2, %3, %4};" ::"l"(of + 4 * (i + q * stride)),
+                                 "l"(n[4 * q] + add), "l"(n[4 * q + 1] + add), "l"(n[4 * q + 2] + add),
+                                 "l"(n[4 * q + 3] + add)
+                                 : "memory");
         }
         return;
     }
@@ -132,7 +136,7 @@ extern "C" ebag_status ebag_mbdt(const float* values, int32_t F, int64_t B, cons
     int64_t cap = (int64_t)sms * per_sm / F;
     if (cap < 1) cap = 1;
     if (bx > cap) bx = cap;
-    const bool vec = (B & 1) == 0 && !((uintptr_t)values & 7u) && !((uintptr_t)out & 15u);
+    const bool vec = (B & 3) == 0 && !((uintptr_t)values & 15u) && !((uintptr_t)out & 31u);
     if (vec)
         mbdt_kernel<true><<<dim3((unsigned)bx, (unsigned)F), kThreads, 0, (cudaStream_t)stream>>>(
             values, B, borders, border_offsets, out_offsets, out);
