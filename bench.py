@@ -42,7 +42,7 @@ L2_FLUSH_BYTES = 256 << 20
 # DRAM bytes per forward launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu
 # captures summarised under profiles/ (a smaller case of the same kernel, scaled to a full launch
 # by lookups); None where no capture of that workload exists.
-NCU_DRAM_BYTES_PER_LAUNCH = {3: 4.46e9, 4: 13.71e9, 5: 9.77e9}
+NCU_DRAM_BYTES_PER_LAUNCH = {3: 4.59e9, 4: 13.71e9, 5: 10.43e9}
 
 
 def parse_args():
