@@ -281,9 +281,17 @@ __device__ void tile_exscan2(const int64_t* __restrict__ a, const int64_t* __res
     }
 }
 
+// The four launches of a truncation are made with programmatic stream serialization: the CTAs of
+// a launch may become resident while the launch before it drains, and wait here for its results.
+__device__ __forceinline__ void wait_for_previous_launch() {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;");
+}
+
 __global__ void __launch_bounds__(kScanThreads)
 bet_scan_outer(const int64_t* __restrict__ outer, int64_t U, int64_t N, int64_t* __restrict__ outer_out,
                BetWorkspace w, int64_t* __restrict__ counts_out) {
+    wait_for_previous_launch();
     tile_exscan2<true>(outer, nullptr, N, U, blockIdx.x, outer_out, w.ev_in, w.ev_out);
     if ((int64_t)(blockIdx.x + 1) * kScanTile >= U) {
         __syncthreads();
@@ -301,6 +309,7 @@ constexpr int kSumBatch = 6;        // bet_user_sums: loads per lane requested o
 // one wave of resident CTAs and the (feature, users) tasks are dealt round-robin to its warps.
 __global__ void __launch_bounds__(256)
 bet_user_sums(const int64_t* __restrict__ inner, int64_t E, int64_t U, int F, BetWorkspace w) {
+    wait_for_previous_launch();
     const int lane = threadIdx.x & 31;
     const int64_t warps = (int64_t)gridDim.x * (blockDim.x >> 5);
     const int64_t chunks = (U + kTaskUsers - 1) / kTaskUsers;       // per feature
@@ -359,10 +368,17 @@ bet_user_sums(const int64_t* __restrict__ inner, int64_t E, int64_t U, int F, Be
                     if (j0 + 32 * q < kkeep) kept += n;
                 }
             }
+            // the lanes' sums added up: one warp reduction each while every lane's sum is below
+            // 2^26 (then the total fits 32 bits), else five 64-bit shuffle steps
+            if (!__any_sync(0xffffffffu, all >= (1ll << 26))) {
+                all = (int64_t)__reduce_add_sync(0xffffffffu, (unsigned)all);
+                kept = (int64_t)__reduce_add_sync(0xffffffffu, (unsigned)kept);
+            } else {
 #pragma unroll
-            for (int d = 16; d > 0; d >>= 1) {
-                all += __shfl_xor_sync(0xffffffffu, all, d);
-                kept += __shfl_xor_sync(0xffffffffu, kept, d);
+                for (int d = 16; d > 0; d >>= 1) {
+                    all += __shfl_xor_sync(0xffffffffu, all, d);
+                    kept += __shfl_xor_sync(0xffffffffu, kept, d);
+                }
             }
             if (lane == k) { my_all = all; my_kept = kept; }
 #pragma unroll
@@ -377,6 +393,7 @@ bet_user_sums(const int64_t* __restrict__ inner, int64_t E, int64_t U, int F, Be
 
 __global__ void __launch_bounds__(kScanThreads)
 bet_scan_values(int64_t U, BetWorkspace w, int64_t* __restrict__ counts_out) {
+    wait_for_previous_launch();
     const int f = blockIdx.y;
     tile_exscan2<false>(w.v_all + (int64_t)f * U, w.v_keep + (int64_t)f * U, 0, U, blockIdx.x, nullptr,
                         w.v_in + (int64_t)f * (U + 1), w.v_out + (int64_t)f * (U + 1));
@@ -412,6 +429,7 @@ __global__ void __launch_bounds__(256)
 bet_copy(const int64_t* __restrict__ inner, int64_t E, const int64_t* __restrict__ values,
          const int64_t* __restrict__ value_offsets, int64_t U, int F, BetWorkspace w,
          int64_t* __restrict__ inner_out, int64_t* __restrict__ values_out) {
+    wait_for_previous_launch();
     const int lane = threadIdx.x & 31;
     const int64_t warps = (int64_t)gridDim.x * (blockDim.x >> 5);
     const int64_t chunks = (U + kTaskUsers - 1) / kTaskUsers;       // per feature
@@ -485,14 +503,39 @@ extern "C" ebag_status ebag_batch_event_truncate(const int64_t* outer_lengths, i
     cudaStream_t s = (cudaStream_t)stream;
     const BetWorkspace w = carve(workspace, F, U);
     const unsigned tiles = (unsigned)(U > 0 ? (U + kScanTile - 1) / kScanTile : 1);
-    bet_scan_outer<<<tiles, kScanThreads, 0, s>>>(outer_lengths, U, N, outer_out, w, counts_out);
-    if (F > 0 && U > 0) {
-        bet_user_sums<<<bet_grid(bet_user_sums, F, U), 256, 0, s>>>(inner_lengths, E, U, F, w);
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    auto config = [&](dim3 grid, unsigned threads) {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = grid;
+        cfg.blockDim = dim3(threads);
+        cfg.stream = s;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        return cfg;
+    };
+    cudaError_t err;
+    {
+        cudaLaunchConfig_t cfg = config(dim3(tiles), kScanThreads);
+        err = cudaLaunchKernelEx(&cfg, bet_scan_outer, outer_lengths, U, N, outer_out, w, counts_out);
     }
-    if (F > 0) bet_scan_values<<<dim3(tiles, (unsigned)F), kScanThreads, 0, s>>>(U, w, counts_out);
-    if (F > 0 && U > 0) {
-        bet_copy<<<bet_grid(bet_copy, F, U), 256, 0, s>>>(inner_lengths, E, values, value_offsets, U, F, w,
-                                                          inner_out, values_out);
+    if (err == cudaSuccess && F > 0 && U > 0) {
+        cudaLaunchConfig_t cfg = config(dim3(bet_grid(bet_user_sums, F, U)), 256);
+        err = cudaLaunchKernelEx(&cfg, bet_user_sums, inner_lengths, E, U, (int)F, w);
+    }
+    if (err == cudaSuccess && F > 0) {
+        cudaLaunchConfig_t cfg = config(dim3(tiles, (unsigned)F), kScanThreads);
+        err = cudaLaunchKernelEx(&cfg, bet_scan_values, U, w, counts_out);
+    }
+    if (err == cudaSuccess && F > 0 && U > 0) {
+        cudaLaunchConfig_t cfg = config(dim3(bet_grid(bet_copy, F, U)), 256);
+        err = cudaLaunchKernelEx(&cfg, bet_copy, inner_lengths, E, values, value_offsets, U, (int)F, w, inner_out,
+                                 values_out);
+    }
+    if (err != cudaSuccess) {
+        cudaGetLastError();
+        return EBAG_ERR_CUDA;
     }
     if (cudaGetLastError() != cudaSuccess) return EBAG_ERR_CUDA;
     return EBAG_OK;
