@@ -203,18 +203,27 @@ __device__ void tile_exscan2(const int64_t* __restrict__ a, const int64_t* __res
         if (CLAMP) return av < clamp ? av : clamp;
         return nonneg(b[i]);
     };
+    // ---- the tile's own entries, kScanItems consecutive ones per thread: requested first, so
+    // that they travel while everything before the tile is added up
+    const int64_t i0 = t0 + (int64_t)tid * kScanItems;
+    int64_t xa[kScanItems], xb[kScanItems];
+#pragma unroll
+    for (int k = 0; k < kScanItems; ++k) {
+        xa[k] = i0 + k < n ? nonneg(a[i0 + k]) : 0;
+        xb[k] = i0 + k < n ? bval(xa[k], i0 + k) : 0;
+    }
     // ---- everything before the tile
     int64_t pa = 0, pb = 0;
-    for (int64_t i0 = tid; i0 < t0; i0 += (int64_t)kScanThreads * 8) {
-        int64_t xa[8], xb[8];
+    for (int64_t j0 = tid; j0 < t0; j0 += (int64_t)kScanThreads * 8) {
+        int64_t ya[8], yb[8];
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
-            const int64_t i = i0 + (int64_t)k * kScanThreads;
-            xa[k] = i < t0 ? nonneg(a[i]) : 0;
-            xb[k] = i < t0 ? bval(xa[k], i) : 0;
+            const int64_t i = j0 + (int64_t)k * kScanThreads;
+            ya[k] = i < t0 ? nonneg(a[i]) : 0;
+            yb[k] = i < t0 ? bval(ya[k], i) : 0;
         }
 #pragma unroll
-        for (int k = 0; k < 8; ++k) { pa += xa[k]; pb += xb[k]; }
+        for (int k = 0; k < 8; ++k) { pa += ya[k]; pb += yb[k]; }
     }
 #pragma unroll
     for (int d = 16; d > 0; d >>= 1) {
@@ -233,14 +242,10 @@ __device__ void tile_exscan2(const int64_t* __restrict__ a, const int64_t* __res
         if (lane == 0) { base[0] = wa; base[1] = wb; }
     }
     __syncthreads();
-    // ---- the tile itself: every thread owns kScanItems consecutive entries
-    const int64_t i0 = t0 + (int64_t)tid * kScanItems;
-    int64_t xa[kScanItems], xb[kScanItems];
+    // ---- the tile itself (its entries were requested before the reduction above)
     int64_t ta = 0, tb = 0;                          // this thread's totals
 #pragma unroll
     for (int k = 0; k < kScanItems; ++k) {
-        xa[k] = i0 + k < n ? nonneg(a[i0 + k]) : 0;
-        xb[k] = i0 + k < n ? bval(xa[k], i0 + k) : 0;
         ta += xa[k];
         tb += xb[k];
     }
