@@ -206,8 +206,8 @@ ebag_status ebag_mapid(const int64_t* values, int64_t n, const int64_t* mapping,
  * device, so there is no host synchronisation.  Followed by ebag_forward this was measured
  * faster than the fused call for mappings of 1 k - 100 k ids (the fused search stalls the gather).
  * When the call has at least as many values as the hash tables of its mappings have slots (per
- * table the power of two at or above twice its length, 16 bytes a slot, 2^24 slots in all at
- * most), those tables are first built in a scratch buffer the handle keeps (grown, with a device
+ * table the power of two at or above four times its length, 16 bytes a slot, 2^24 slots in all
+ * at most), those tables are first built in a scratch buffer the handle keeps (grown, with a device
  * synchronisation, when a larger call arrives) and every value is then found with one or two
  * loads: three operations on the stream (clear, build, look up; two kernel launches) instead of
  * one binary-search launch.  Both give the same ids for a sorted mapping, with equal keys mapped

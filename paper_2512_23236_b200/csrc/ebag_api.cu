@@ -568,7 +568,7 @@ mapid_tbe_kernel(const int64_t* __restrict__ values, int64_t n_values, const int
 
 // ---- MapId through a hash table.  When a call has many more values than mapping entries, the
 // handle first builds, per table, an open-addressing table of the mapping (16-byte slots: key,
-// index + 1; linear probing; at most half full) and the searches become one or two loads each
+// index + 1; linear probing; at most a quarter full) and the searches become one or two loads each
 // instead of log2(|M|) dependent ones.  The result is the same as the binary search's for a
 // sorted mapping: equal keys are adjacent there and only the first of a run is inserted.
 // slots of every table's hash table into hbase[t + 1], hbase[0] = 0: after a prefix sum over
@@ -607,7 +607,7 @@ map_hash_build_kernel(int T, const int64_t* const* __restrict__ mappings,
         const int64_t key = M[i];
         if (i > 0 && M[i - 1] == key) continue;              // only the first of a run of equal keys
         uint32_t s = (uint32_t)(((uint64_t)key * kHashMul) >> (64 - bits));
-        for (uint32_t probe = 0; probe <= mask; ++probe) {   // at most half full: ends early
+        for (uint32_t probe = 0; probe <= mask; ++probe) {   // at most a quarter full: ends early
             if (atomicCAS(&tab[s].idx1, 0u, (uint32_t)i + 1u) == 0u) {
                 tab[s].key = key;
                 break;

@@ -118,7 +118,7 @@ struct PartArgs {                        // one part of a long bag (parts kernel
     float* slot;                         // where its rows of partial sums go
 };
 
-// Hash table of a MapId mapping: open addressing, linear probing, at most half full, 2^bits
+// Hash table of a MapId mapping: open addressing, linear probing, at most a quarter full, 2^bits
 // slots with bits = map_hash_bits(|M|); slot of key k on the first probe = (k * kHashMul) >> (64 - bits).
 struct __align__(16) MapSlot {
     int64_t key;
@@ -130,7 +130,7 @@ constexpr int64_t kMapHashMaxSlots = 1ll << 24;          // 256 MB of slots per 
 
 __host__ __device__ inline uint32_t map_hash_bits(int64_t mlen) {
     uint32_t bits = 1;
-    while (bits < 31 && (1ll << bits) < 2 * mlen) ++bits;
+    while (bits < 31 && (1ll << bits) < 4 * mlen) ++bits;
     return bits;
 }
 
@@ -380,7 +380,7 @@ __device__ __forceinline__ int64_t map_id(const int64_t* __restrict__ M, uint32_
 __device__ __forceinline__ int64_t map_hash_lookup(const MapSlot* __restrict__ tab, uint32_t bits, int64_t v) {
     const uint32_t mask = (1u << bits) - 1u;
     uint32_t s = (uint32_t)(((uint64_t)v * kHashMul) >> (64 - bits));
-    for (uint32_t probe = 0; probe <= mask; ++probe) {       // at most half full: ends early
+    for (uint32_t probe = 0; probe <= mask; ++probe) {       // at most a quarter full: ends early
         const int4 q = __ldg(reinterpret_cast<const int4*>(tab + s));
         if (q.z == 0) return 0;                               // an empty slot: not mapped
         const int64_t key = (int64_t)(((uint64_t)(uint32_t)q.y << 32) | (uint32_t)q.x);

@@ -59,7 +59,7 @@ def test_fused_mapid_forward(dtype, mode, weighted, path):
     mappings = [np.sort(rng.choice(np.arange(0, 20 * m + 50, dtype=np.int64), size=m, replace=False))
                 for m in mlens]
     rows = [m + 1 for m in mlens]
-    lengths = np.concatenate([rng.integers(0, 40, size=B) for _ in range(T)])
+    lengths = np.concatenate([rng.integers(0, 80, size=B) for _ in range(T)])
     offsets = np.zeros(T * B + 1, np.int64)
     np.cumsum(lengths, out=offsets[1:])
     vals = []
@@ -136,7 +136,7 @@ def test_mapid_for_all_tables_with_duplicates_empty_mappings_and_extreme_values(
                 np.arange(0, 3 * 70_001, 3, dtype=np.int64),
                 np.array([42], np.int64)]
     T = len(mappings)
-    lengths = rng.integers(0, 3000, size=T * B)     # more values than hash slots: the hash path is taken
+    lengths = rng.integers(0, 6000, size=T * B)     # more values than hash slots: the hash path is taken
     offsets = np.zeros(T * B + 1, np.int64)
     np.cumsum(lengths, out=offsets[1:])
     vals = []
@@ -178,7 +178,7 @@ def test_mapid_for_many_small_tables(use_hash):
     for t in range(T):
         m = int(rng.integers(0, 300)) if t % 7 else 0
         mappings.append(np.sort(rng.choice(np.arange(-1000, 5000, dtype=np.int64), size=m, replace=False)))
-    lengths = rng.integers(0, 40, size=T * B)
+    lengths = rng.integers(0, 120, size=T * B)
     lengths[5 * B:9 * B] = 0                                # four tables in a row without values
     offsets = np.zeros(T * B + 1, np.int64)
     np.cumsum(lengths, out=offsets[1:])
