@@ -789,6 +789,8 @@ def main():
     # event pair and counted in gpu_launches)
     ms_per_launch = elapsed_ms / max(1, args.steps)
     achieved = ab["total"] / (ms_per_launch * 1e-3) / 1e9
+    full_size = not (args.max_tables or args.scale_rows != 1.0 or args.scale_b != 1.0)
+    traffic = NCU_DRAM_BYTES_PER_LAUNCH.get(w.number) if (full_size and not mapid) else None
     line = {
         "metric": METRIC, "value": total_lookups / (max_ms * 1e-3), "unit": UNIT, "n_gpus": world,
         "steps": args.steps, "warmup": warmup, "ms_per_step": max_ms / args.steps,
@@ -807,7 +809,11 @@ def main():
                      "ms_per_launch": ms_per_launch, "ms_per_launch_min": min(step_ms),
                      "ms_per_launch_median": sorted(step_ms)[len(step_ms) // 2],
                      "ms_per_launch_warm_l2": warm_ms,
-                     "traffic": None if mapid else NCU_DRAM_BYTES_PER_LAUNCH.get(w.number)},
+                     "traffic": traffic,
+                     # the same launch seen from DRAM: stored ncu traffic over the live launch time
+                     "dram_gbs": None if traffic is None else traffic / (ms_per_launch * 1e-3) / 1e9,
+                     "dram_frac": None if traffic is None
+                     else traffic / (ms_per_launch * 1e-3) / 1e9 / peaks["hbm_gbs"]},
         "bags_per_sec": w.T * w.B * world * args.steps / (max_ms * 1e-3),
     }
     if mapid_extra:
