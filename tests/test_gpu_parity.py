@@ -452,3 +452,36 @@ def test_repeated_calls_and_changing_table_pointers():
     for (o, _), r in zip(outs, refs):
         pu.compare(o.cpu().numpy(), r, wl.F32, lengths, 2, B, D)
     tbe.close()
+
+
+# ------------------------------------------------------------------ output alignment
+@pytest.mark.parametrize("dtype,Ds", [(wl.BF16, [8, 64, 136]), (wl.INT8_ROWWISE, [16, 128, 48]),
+                                      (wl.F32, [4, 64])])
+def test_output_that_is_only_16_byte_aligned(dtype, Ds):
+    """16- and 8-bit tables write whole 32-byte sectors with one store where the output allows it;
+    an output buffer that starts 16 bytes into a sector must give the same bits through the
+    16-byte stores."""
+    rng = np.random.default_rng(9 + dtype)
+    T, B = len(Ds), 50
+    rows = [int(rng.integers(5, 200)) for _ in Ds]
+    lens = [rng.integers(0, 30, size=B) for _ in Ds]
+    idx, off, lengths = _jagged_from_lengths(rng, lens, rows)
+    tabs = _rand_tables(rng, dtype, rows, Ds)
+    dev = pu.device_tables(dtype, tabs)
+    sumD = sum(Ds)
+    d_idx, d_off = torch.from_numpy(idx).cuda(), torch.from_numpy(off).cuda()
+    tbe = eb.TBE(rows, Ds, dtype, device=torch.cuda.current_device())
+    aligned = torch.full((B, sumD), float("nan"), dtype=torch.float32, device="cuda")
+    assert aligned.data_ptr() % 32 == 0
+    tbe.forward(dev, d_idx, d_off, B, wl.SUM, None, out=aligned)
+    store = torch.full((B * sumD + 8,), float("nan"), dtype=torch.float32, device="cuda")
+    shifted = store[4:4 + B * sumD].view(B, sumD)
+    assert shifted.data_ptr() % 32 == 16
+    tbe.forward(dev, d_idx, d_off, B, wl.SUM, None, out=shifted)
+    assert tbe.last_status() == (0, 0, 0)
+    tbe.close()
+    assert torch.equal(aligned, shifted)
+    assert torch.isnan(store[:4]).all() and torch.isnan(store[4 + B * sumD:]).all()   # nothing written outside
+    ot, sc, bi = pu.oracle_tables(dtype, tabs)
+    ref = orc.forward(ot, dtype, idx, off, B, wl.SUM, scales=sc, biases=bi)
+    pu.compare(aligned.cpu().numpy(), ref, dtype, lengths, T, B, Ds)
