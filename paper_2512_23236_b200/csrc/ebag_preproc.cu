@@ -356,11 +356,10 @@ bet_user_sums(const int64_t* __restrict__ inner, int64_t E, int64_t U, int F, Be
         auto first_batch = [&](int k, int64_t (&x)[kSumBatch]) {
             const int64_t ke0 = __shfl_sync(0xffffffffu, e0, k & 31);
             const int64_t cnt = k < users ? __shfl_sync(0xffffffffu, e1, k & 31) - ke0 : 0;
+            const int cnt32 = cnt > 0x7fffffffll ? 0x7fffffff : (int)cnt;      // the batch looks at 192 entries
+            const long long* __restrict__ src = reinterpret_cast<const long long*>(row + ke0) + lane;
 #pragma unroll
-            for (int q = 0; q < kSumBatch; ++q) {
-                const int64_t j = lane + 32 * q;
-                x[q] = j < cnt ? __ldcs(reinterpret_cast<const long long*>(row + ke0 + j)) : 0;
-            }
+            for (int q = 0; q < kSumBatch; ++q) x[q] = lane + 32 * q < cnt32 ? __ldcs(src + 32 * q) : 0;
         };
         first_batch(0, cur);
         for (int k = 0; k < users; ++k) {
@@ -369,11 +368,12 @@ bet_user_sums(const int64_t* __restrict__ inner, int64_t E, int64_t U, int F, Be
             const int64_t cnt = __shfl_sync(0xffffffffu, e1, k) - ke0;
             const int64_t kkeep = __shfl_sync(0xffffffffu, keep, k);
             int64_t all = 0, kept = 0;
+            const int keep32 = kkeep > 0x7fffffffll ? 0x7fffffff : (int)kkeep;
 #pragma unroll
             for (int q = 0; q < kSumBatch; ++q) {
                 const int64_t n = nonneg(cur[q]);
                 all += n;
-                if (lane + 32 * q < kkeep) kept += n;
+                if (lane + 32 * q < keep32) kept += n;
             }
             for (int64_t j0 = lane + 32 * kSumBatch; j0 < cnt; j0 += 32 * kCopyBatch) {   // the rest, if any
                 int64_t x[kCopyBatch];
