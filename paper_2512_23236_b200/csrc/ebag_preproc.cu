@@ -8,7 +8,7 @@ namespace {
 
 constexpr int kThreads = 256;
 constexpr int kSmemBorders = 64;     // border lists up to this long are counted linearly from smem
-constexpr int kIlp = 16;             // values per thread in flight (8 and 32 measured slower: 0.169 and 0.253 ms against 0.154)
+constexpr int kIlp = 16;             // values per thread in flight at 3 CTAs per SM (8, 12, 32 and 2 or 4 CTAs measured slower)
 
 // Launches here are made with programmatic stream serialization: the CTAs of a launch may become
 // resident while the launch before it on the stream drains, and wait here for its results.
@@ -34,7 +34,7 @@ inline cudaLaunchConfig_t serialized_launch(dim3 grid, unsigned threads, cudaStr
 // like the library routine the paper's pseudocode calls.  Short lists are counted linearly
 // (the vectorised counting the paper's kernel uses), long ones by a branch-free halving search.
 template <bool VEC>       // VEC: B is a multiple of 4, values 16-byte and out 32-byte aligned
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, 3)
 mbdt_kernel(const float* __restrict__ values, int64_t B, const float* __restrict__ borders,
             const int64_t* __restrict__ border_offsets, const int64_t* __restrict__ out_offsets,
             int64_t* __restrict__ out) {
