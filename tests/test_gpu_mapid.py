@@ -194,3 +194,25 @@ def test_mapid_for_many_small_tables(use_hash):
         lo, hi = int(offsets[t * B]), int(offsets[(t + 1) * B])
         want = mo.mapid(values[lo:hi], mappings[t]) if mappings[t].size else np.zeros(hi - lo, np.int64)
         assert np.array_equal(got[lo:hi], want), t
+
+
+def test_mapid_with_a_mapping_too_large_for_the_hash_scratch_uses_the_binary_search():
+    """Hash tables are capped at 2^24 slots per handle; a mapping of 5 M ids would need 2^25, so
+    the call keeps to the binary search (one launch) and still maps every value."""
+    rng = np.random.default_rng(123)
+    m = 5_000_000
+    mapping = np.cumsum(rng.integers(1, 4, size=m)).astype(np.int64)        # strictly increasing
+    B = 256
+    lengths = rng.integers(0, 400, size=B)
+    offsets = np.zeros(B + 1, np.int64)
+    np.cumsum(lengths, out=offsets[1:])
+    n = int(offsets[-1])
+    values = rng.integers(0, int(mapping[-1]) + 10, size=n).astype(np.int64)
+    values[::2] = mapping[rng.integers(0, m, size=values[::2].shape[0])]
+    tbe = eb.TBE([8], [8], eb.EBAG_F32, device=torch.cuda.current_device())
+    before = tbe.launch_count()
+    got = tbe.mapid(torch.from_numpy(values).cuda(), torch.from_numpy(offsets).cuda(),
+                    [torch.from_numpy(mapping).cuda()], B).cpu().numpy()
+    assert tbe.launch_count() - before == 1
+    tbe.close()
+    assert np.array_equal(got, mo.mapid(values, mapping))
