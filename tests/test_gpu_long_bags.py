@@ -9,7 +9,7 @@ import paper_2512_23236_b200 as eb
 from oracle import ebag_oracle as orc
 from paper_2512_23236_b200 import workloads as wl
 
-from parity_util import compare, device_tables, oracle_tables, run_gpu
+from parity_util import compare, device_tables, oracle_forward, oracle_tables, run_gpu
 
 pytestmark = pytest.mark.gpu
 
@@ -45,7 +45,7 @@ def _check(dtype, rows, D, B, lengths, mode=wl.SUM, weighted=False, seed=0, para
         spoil(idx, off)
     dev = device_tables(dtype, tables)
     tabs, sc, bi = oracle_tables(dtype, tables)
-    ref = orc.forward(tabs, dtype, idx, off, B, mode, weights=w, scales=sc, biases=bi)
+    ref = oracle_forward(tabs, dtype, idx, off, B, mode, weights=w, scales=sc, biases=bi)
     gpu1, st1 = run_gpu(dtype, rows, D, dev, idx, off, B, mode, w, params)
     gpu2, st2 = run_gpu(dtype, rows, D, dev, idx, off, B, mode, w, params)
     whole, st3 = run_gpu(dtype, rows, D, dev, idx, off, B, mode, w, {"split_bytes": 0})

@@ -104,6 +104,8 @@ def test_fused_mapid_forward(dtype, mode, weighted, path):
     tbe.close()
     ot, sc, bi = pu.oracle_tables(dtype, tabs)
     ref = mo.forward_mapid(ot, dtype, values, offsets, B, mappings, mode, weights=w, scales=sc, biases=bi)
+    if dtype in pu.ROWWISE8:            # the floor of the bar for rowwise 8-bit tables, on the mapped ids
+        ref["F"] = pu.rowwise8_floor(ot, sc, bi, ids.cpu().numpy(), offsets, B, mode, w)
     pu.compare(out.cpu().numpy(), ref, dtype, lengths, T, B, Ds)
 
 

@@ -50,7 +50,7 @@ def _both(dtype, rows, D, tabs, idx, off, B, mode, w=None, params=None, host_pat
     dev = pu.device_tables(dtype, tabs)
     gpu, status = pu.run_gpu(dtype, rows, D, dev, idx, off, B, mode, w, params, host_path)
     ot, sc, bi = pu.oracle_tables(dtype, tabs)
-    ref = orc.forward(ot, dtype, idx, off, B, mode, weights=w, scales=sc, biases=bi)
+    ref = pu.oracle_forward(ot, dtype, idx, off, B, mode, weights=w, scales=sc, biases=bi)
     return gpu, status, ref
 
 
@@ -230,7 +230,7 @@ def test_sixteen_bit_output(dtype, Ds, out_dtype, mode, weighted):
     tabs = _rand_tables(rng, dtype, rows, Ds)
     dev = pu.device_tables(dtype, tabs)
     ot, sc, bi = pu.oracle_tables(dtype, tabs)
-    ref = orc.forward(ot, dtype, idx, off, B, mode, weights=w, scales=sc, biases=bi)
+    ref = pu.oracle_forward(ot, dtype, idx, off, B, mode, weights=w, scales=sc, biases=bi)
     tbe = eb.TBE(rows, Ds, dtype, device=torch.cuda.current_device())
     try:
         tbe.set_param("out_dtype", out_dtype)
@@ -483,5 +483,5 @@ def test_output_that_is_only_16_byte_aligned(dtype, Ds):
     assert torch.equal(aligned, shifted)
     assert torch.isnan(store[:4]).all() and torch.isnan(store[4 + B * sumD:]).all()   # nothing written outside
     ot, sc, bi = pu.oracle_tables(dtype, tabs)
-    ref = orc.forward(ot, dtype, idx, off, B, wl.SUM, scales=sc, biases=bi)
+    ref = pu.oracle_forward(ot, dtype, idx, off, B, wl.SUM, scales=sc, biases=bi)
     pu.compare(aligned.cpu().numpy(), ref, dtype, lengths, T, B, Ds)
