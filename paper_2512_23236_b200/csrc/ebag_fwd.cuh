@@ -450,17 +450,33 @@ struct IdChunk {          // ids of up to G consecutive entries of the bags one 
 
 // Offsets of bag `lane` of an item relative to the item's first lookup (both 0 for a malformed
 // bag, which is reported through `bad`).
-__device__ __forceinline__ void load_bag_range(const FwdParams& p, int64_t g0, int lane,
-                                               int64_t base_raw, int64_t base, uint32_t& off_lo,
-                                               uint32_t& off_hi, bool& bad) {
-    const int64_t room = p.n_indices - base;
-    const int64_t lo = ld_stream_i64(p.offsets + g0 + lane) - base;
-    const int64_t hi = ld_stream_i64(p.offsets + g0 + lane + 1) - base;
+// The offsets of an item's bags as 32-bit distances from `base`, the smallest start among the
+// item's well-formed bags (with offsets that do not decrease that is the first bag's start; with
+// malformed ones a later bag may start before it, and is still pooled if it is well-formed itself).
+// All 32 lanes call this; lanes at or beyond `cnt` hold no bag.
+__device__ __forceinline__ void load_bag_range(const FwdParams& p, int64_t g0, int lane, int cnt,
+                                               int64_t& base, uint32_t& off_lo, uint32_t& off_hi,
+                                               bool& bad) {
+    int64_t s = 0, e = 0;
+    if (lane < cnt) {
+        s = ld_stream_i64(p.offsets + g0 + lane);
+        e = ld_stream_i64(p.offsets + g0 + lane + 1);
+    }
+    bad = lane < cnt && (s < 0 || e < s || e > p.n_indices);
+    // smallest start of a well-formed bag: high words first, then the low words of those
+    const bool in = lane < cnt && !bad;
+    const unsigned hi_w = in ? (unsigned)((uint64_t)s >> 32) : 0xffffffffu;
+    const unsigned hi_min = __reduce_min_sync(0xffffffffu, hi_w);
+    const unsigned lo_w = (in && hi_w == hi_min) ? (unsigned)s : 0xffffffffu;
+    const unsigned lo_min = __reduce_min_sync(0xffffffffu, lo_w);
+    base = hi_min == 0xffffffffu ? 0 : (int64_t)(((uint64_t)hi_min << 32) | lo_min);
     off_lo = off_hi = 0;
-    bad = base_raw != base || lo < 0 || hi < lo || hi > room || hi > 0x7fffffffll;
-    if (!bad) {
-        off_lo = (uint32_t)lo;
-        off_hi = (uint32_t)hi;
+    if (in) {
+        if (e - base > 0x7fffffffll) bad = true;       // an item that spans 2^31 lookups or more
+        else {
+            off_lo = (uint32_t)(s - base);
+            off_hi = (uint32_t)(e - base);
+        }
     }
 }
 
@@ -496,13 +512,9 @@ __device__ __forceinline__ void process_item(const FwdParams& p, const TableMeta
         }
     } else {
         const int64_t g0 = (int64_t)t * p.off_stride + bag0;
-        const int64_t base_raw = ld_stream_i64(p.offsets + g0);
-        base = base_raw < 0 ? 0 : (base_raw > p.n_indices ? p.n_indices : base_raw);
-        if (lane < cnt) {
-            bool bad;
-            load_bag_range(p, g0, lane, base_raw, base, off_lo, off_hi, bad);
-            if (bad && vec0 == 0) ++n_bad;
-        }
+        bool bad;
+        load_bag_range(p, g0, lane, cnt, base, off_lo, off_hi, bad);
+        if (bad && vec0 == 0) ++n_bad;
         if (p.lg.ctl) {
             // ---- bags long enough to be split are recorded for the parts kernel (by the call
             // for the first column tile) and count as empty here

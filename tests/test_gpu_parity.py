@@ -384,6 +384,28 @@ def test_bad_offsets_treated_as_empty_and_counted():
     pu.compare(gpu, ref, wl.F32)
 
 
+@pytest.mark.parametrize("dtype,D", [(wl.F32, [16, 260]), (wl.BF16, [64, 8]), (wl.INT8_ROWWISE, [128, 16])])
+def test_offsets_that_jump_forward_and_come_back(dtype, D):
+    """An offset far ahead of its neighbours makes the bag before it reach over later bags (still
+    a well-formed bag: it is pooled, overlap and all) and the bag after it run backwards (empty,
+    counted).  The bags that follow start BEFORE that offset and are well-formed themselves: they
+    must be pooled too, wherever the work items happen to be cut."""
+    rng = np.random.default_rng(12 + dtype)
+    T, B = len(D), 70
+    rows = [150] * T
+    lens = [rng.integers(0, 12, size=B) for _ in D]
+    idx, off, lengths = _jagged_from_lengths(rng, lens, rows)
+    tabs = _rand_tables(rng, dtype, rows, D)
+    for g in (1, 7, 32, 33, 64, B + 3, B + 31, 2 * B - 2):          # first bags of items, middles, table ends
+        bad = off.copy()
+        bad[g] = min(bad[g + 1] + 5, idx.shape[0])
+        for params in (None, dict(item_bytes=256)):                   # small items: other cut points
+            gpu, status, ref = _both(dtype, rows, D, tabs, idx, bad, B, wl.SUM, params=params)
+            assert ref["n_bad_offsets"] == (1 if bad[g] > bad[g + 1] else 0)
+            assert status[1:] == (ref["n_oob"], ref["n_bad_offsets"]), (g, params)
+            pu.compare(gpu, ref, dtype)
+
+
 def test_maximum_number_of_tables():
     """EBAG_MAX_TABLES tables in one launch (the item table of the kernel lives in shared memory
     and grows with T); one more table is refused at create time."""
