@@ -974,7 +974,9 @@ ebag_status ebag_backward(ebag_tbe* h, const float* grad_out, const void* indice
         if (!grad_tables[t] && h->rows[t] > 0) return EBAG_ERR_INVALID_ARG;
         if ((uintptr_t)grad_tables[t] & 15u) return EBAG_ERR_INVALID_ARG;
     }
-    if (B == 0 || n_indices == 0) return EBAG_OK;
+    // (no ids is not the same as nothing to do: offsets that reach past an empty id list are
+    // malformed bags, and the kernel counts them as the forward does)
+    if (B == 0) return EBAG_OK;
     DeviceGuard guard(h->device);
     if (!guard.ok) return EBAG_ERR_CUDA;
     cudaStream_t s = (cudaStream_t)stream;

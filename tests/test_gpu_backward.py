@@ -116,6 +116,20 @@ def test_rejected_ids_and_malformed_bags():
     _compare(got, ref)
 
 
+def test_offsets_that_reach_past_an_empty_id_list_are_counted():
+    """No ids at all, but a bag that claims five: a malformed bag, counted as the oracle counts it
+    (the call must not take "no ids" for "nothing to do")."""
+    rows, D, B = [7], [8], 1
+    off = np.array([0, 5], np.int64)
+    idx = np.zeros(0, np.int64)
+    G = np.ones((B, 8), np.float32)
+    ref = bo.backward(rows, D, G, idx, off, B, wl.SUM)
+    assert (ref["n_oob"], ref["n_bad_offsets"]) == (0, 1)
+    got, status = _run(wl.F32, rows, D, B, off, idx, None, G, wl.SUM)
+    assert status == (eb.EBAG_ERR_BAD_OFFSETS, 0, 1)
+    assert not got[0].any()
+
+
 def test_adjoint_of_the_gpu_forward():
     """<forward(T), G> = <T, backward(G)> with both sides computed on the GPU."""
     rng = np.random.default_rng(8)
