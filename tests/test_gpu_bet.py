@@ -50,7 +50,10 @@ def test_paper_worked_example_on_gpu():
 
 @pytest.mark.parametrize("U,F,max_events,max_attr,N", [
     (3, 1, 5, 3, 2), (64, 1, 200, 12, 100), (64, 5, 200, 12, 100), (40, 9, 200, 6, 200),
-    (33, 32, 50, 5, 20), (1500, 3, 9, 4, 3), (2049, 2, 3, 2, 1), (10, 2, 4, 3, 0), (7, 3, 6, 0, 2)])
+    (33, 32, 50, 5, 20), (1500, 3, 9, 4, 3), (2049, 2, 3, 2, 1), (10, 2, 4, 3, 0), (7, 3, 6, 0, 2),
+    # more users than one scan tile of 4096 holds: the tiles' prefixes come from separate CTAs
+    (4097, 2, 4, 3, 2), (9000, 3, 6, 3, 2), (20001, 1, 3, 2, 1), (40000, 2, 60, 2, 25),
+    (32768, 2, 200, 4, 100)])                      # the benchmark's users, events and N (two of its nine features)
 def test_matches_oracle_bit_for_bit(U, F, max_events, max_attr, N):
     rng = np.random.default_rng(U * 31 + F)
     outer = rng.integers(0, max_events + 1, size=U)
