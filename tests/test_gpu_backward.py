@@ -116,6 +116,31 @@ def test_rejected_ids_and_malformed_bags():
     _compare(got, ref)
 
 
+def test_many_warps_and_tables_against_an_index_add_in_fp64():
+    """A size at which every warp of the grid has work in every table and the hot-row sums are
+    flushed many times: 0.6 M skewed lookups over four tables.  The oracle's Python loops are too
+    slow here; the check is the operator's definition through a library routine (torch index_add_
+    in fp64 on the CPU), with the same bar as the oracle-sized cases."""
+    rng = np.random.default_rng(17)
+    rows, D, B = [50_000, 3_000, 200_000, 64], [32, 64, 8, 128], 6000
+    lengths, off, idx, w, G = _problem(rng, rows, D, B, 50, True, zipf=True)
+    got, status = _run(wl.F32, rows, D, B, off, idx, w, G, wl.SUM)
+    assert status == (0, 0, 0)
+    col = 0
+    for t, (r, d) in enumerate(zip(rows, D)):
+        lo, hi = int(off[t * B]), int(off[(t + 1) * B])
+        bag = np.repeat(np.arange(B), lengths[t * B:(t + 1) * B])
+        terms = torch.from_numpy(G[bag, col:col + d].astype(np.float64) * w[lo:hi, None].astype(np.float64))
+        ids = torch.from_numpy(idx[lo:hi])
+        ref = torch.zeros(r, d, dtype=torch.float64).index_add_(0, ids, terms).numpy()
+        S = torch.zeros(r, d, dtype=torch.float64).index_add_(0, ids, terms.abs()).numpy()
+        n = np.bincount(idx[lo:hi], minlength=r)[:, None].astype(np.float64)
+        err = np.abs(got[t].astype(np.float64) - ref)
+        assert np.all(err <= (8.0 * np.sqrt(n) + 4.0) * U * S), t
+        assert not got[t][n[:, 0] == 0].any()
+        col += d
+
+
 def test_offsets_that_reach_past_an_empty_id_list_are_counted():
     """No ids at all, but a bag that claims five: a malformed bag, counted as the oracle counts it
     (the call must not take "no ids" for "nothing to do")."""

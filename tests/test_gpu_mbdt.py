@@ -30,7 +30,8 @@ def test_paper_worked_example_on_gpu():
 
 
 @pytest.mark.parametrize("B,F,K", [(64, 2, 2), (256, 2, 3), (2048, 2, 4), (1000, 7, 10), (5000, 3, 64),
-                                   (5000, 3, 65), (33333, 5, 1000), (10, 4, 0)])
+                                   (5000, 3, 65), (33333, 5, 1000), (10, 4, 0),
+                                   (1 << 20, 3, 10), ((1 << 20) + 2, 2, 10)])   # the benchmark's batch; the same, not a multiple of 4
 def test_matches_oracle_bit_for_bit(B, F, K):
     rng = np.random.default_rng(B + F + K)
     borders = [np.sort(rng.standard_normal(K + (f % 2 if K else 0))).astype(np.float32) for f in range(F)]
