@@ -2,12 +2,13 @@
  * ebag.h -- C ABI of libebag.so: jagged, pooled embedding-bag forward over one or many tables
  * ("TBE", table-batched embedding) on one NVIDIA B200 (sm_100a).
  *
- * The operator.  Recommendation models keep categorical features as embedding tables whose
- * lookups are memory-bound and irregular ("embedding lookup and aggregation kernels optimized
- * for irregular memory access patterns", paper Sec. 1.1, paragraph "Model Diversity Across
- * Ranking Stages"; "sparse feature embeddings", Sec. 2.1, paragraph "DLRM Architecture").
- * The ids arrive as jagged lists of int64 and, for weighted features, as (int64 id, float32
- * score) pairs (Sec. 2.2, paragraph "Feature Types and Memory Layout").  For T tables and B
+ * The operator.  Recommendation models keep categorical features as embedding tables, in
+ * production often larger than 100 GB; looking rows up and pooling them touches memory
+ * irregularly and is bound by memory capacity and bandwidth, which is why the paper asks for
+ * kernels specialised to it (Sec. 1.1, paragraph "Model Diversity Across Ranking Stages";
+ * Sec. 2.1, paragraph "DLRM Architecture", has the sparse features go through embeddings).  The ids arrive as jagged lists of int64 and, for weighted
+ * features, as (int64 id, float32 score) pairs (Sec. 2.2, paragraph "Feature Types and Memory
+ * Layout").  For T tables and B
  * bags per table this library computes, with bag id g = t*B + b,
  *
  *     out[b, Doff[t] + d] = pool_{i = offsets[g] .. offsets[g+1]-1} w_i * value(t, indices[i], d)
@@ -103,8 +104,13 @@ ebag_status ebag_create_tbe(int32_t T, const int64_t* rows, const int32_t* D, eb
  *   B        bags per table, B >= 0, T*B < 2^31.
  *   out      device fp32 [B, sum(D)] row-major, 16-byte aligned; every element is overwritten
  *            exactly once; must not alias an input.
- * No allocation, no host-device synchronisation.  Host-detectable problems return an error and
- * launch nothing.  Problems only the device can see never fault: an id outside [0, rows[t]) is
+ * No allocation.  The host does not wait for the device, with one exception: the handle keeps
+ * four device copies of the `tables` pointer array (re-sent only when the array's contents
+ * change); a call that brings a fifth different array while the call that used the oldest copy
+ * is still running waits for that call (cudaEventSynchronize).  A call on another stream than
+ * the one that sent the copy it reuses is ordered behind that copy on the device
+ * (cudaStreamWaitEvent).  Callers that pass the same pointers every time never meet either.
+ * Host-detectable problems return an error and launch nothing.  Problems only the device can see never fault: an id outside [0, rows[t]) is
  * skipped (it adds nothing but still counts in the mean's divisor) and a bag with
  * offsets[g+1] < offsets[g], or reaching outside [0, n_indices], is treated as empty; both are
  * counted and reported by ebag_last_status.  B == 0 or n_indices == 0 is fine.
@@ -212,6 +218,10 @@ ebag_status ebag_mapid(const int64_t* values, int64_t n, const int64_t* mapping,
  * loads: three operations on the stream (clear, build, look up; two kernel launches) instead of
  * one binary-search launch.  Both give the same ids for a sorted mapping, with equal keys mapped
  * to the first of their run.  ebag_set_param("mapid_hash", 0) keeps to the binary search.
+ * Table t's values are the range [offsets[t*B], offsets[(t+1)*B]) of the list (clipped to
+ * [0, n_values]), which is the union of its bags whenever offsets do not decrease.  With
+ * malformed offsets a bag may lie outside its table's range: its values are then mapped by the
+ * list of whichever table's range covers them, or not written at all.
  */
 ebag_status ebag_mapid_tbe(ebag_tbe* h, const int64_t* values, int64_t n_values,
                            const int64_t* offsets, const int64_t* const* mappings,
@@ -233,6 +243,12 @@ ebag_status ebag_mapid_tbe(ebag_tbe* h, const int64_t* values, int64_t n_values,
  * tried (the look-ups stall the row pipeline).  Either way the ids are found through hash tables
  * of the mappings when the call is large enough (see ebag_mapid_tbe), else by binary search.  This is the
  * producer of embedding ids the paper's preprocessing section describes.
+ * The two ways agree bit for bit when offsets do not decrease.  Offsets that do decrease can
+ * leave a bag that is well-formed by itself outside its table's range of the value list; the
+ * fused way still maps such a bag with its own table's list (the per-bag definition), the
+ * default way pools whatever ebag_mapid_tbe left at those positions (see there), still without a
+ * fault since every id is range-checked.  Callers that cannot vouch for their offsets and need
+ * the per-bag definition use the fused way.
  */
 ebag_status ebag_forward_mapid(ebag_tbe* h, const void* const* tables, const int32_t* D,
                                const int64_t* values, int64_t n_values, const int64_t* offsets,

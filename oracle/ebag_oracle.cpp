@@ -4,10 +4,10 @@
 // checked against.  Only the tests, the smoke check and the benchmark's CPU-baseline leg may call
 // it; the product (libebag.so and its Python binding) never does, and the two share no code.
 //
-// What it computes.  The paper motivates the operator ("embedding lookup and aggregation kernels
-// optimized for irregular memory access patterns", Sec. 1.1, paragraph "Model Diversity Across
-// Ranking Stages"; "sparse feature embeddings", Sec. 2.1, paragraph "DLRM Architecture") and fixes
-// the input types (Sec. 2.2, paragraph "Feature Types and Memory Layout": sparse features are
+// What it computes.  The paper motivates the operator (Sec. 1.1, paragraph "Model Diversity Across
+// Ranking Stages": production embedding tables pass 100 GB and need kernels that look rows up and
+// pool them under irregular memory access; Sec. 2.1, paragraph "DLRM Architecture": sparse
+// features pass through embeddings) and fixes the input types (Sec. 2.2, paragraph "Feature Types and Memory Layout": sparse features are
 // jagged lists of int64 ids, weighted sparse features are lists of (int64 id, float32 score)
 // pairs) but prints no formula.  The formula is the operator's plain definition:
 //

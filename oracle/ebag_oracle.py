@@ -3,7 +3,8 @@
 TEST INFRASTRUCTURE ONLY: the tests, the smoke check and the benchmark's CPU-baseline leg use
 it; the CUDA library and its binding never import it.  Inputs and outputs are numpy arrays.
 The operator it defines is the pooled embedding-bag forward over jagged id lists
-(Sec. 1.1 "embedding lookup and aggregation"; Sec. 2.2 "Feature Types and Memory Layout").
+(motivated in Sec. 1.1, paragraph "Model Diversity Across Ranking Stages"; input types from
+Sec. 2.2, paragraph "Feature Types and Memory Layout").
 """
 from __future__ import annotations
 

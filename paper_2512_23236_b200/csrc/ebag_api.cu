@@ -58,6 +58,7 @@ struct ebag_tbe {
     const void** h_tables[kTableSlots] = {};       // pinned
     cudaEvent_t slot_event[kTableSlots] = {};
     bool slot_busy[kTableSlots] = {};
+    cudaStream_t slot_stream[kTableSlots] = {};    // the stream the slot's copy was enqueued on
     int slot = -1;
     int occupancy[2][2] = {};                      // CTAs per SM, [plain, MapId][unweighted, weighted]
     uint32_t item_bytes = 32768;
@@ -204,6 +205,10 @@ ebag_status stage_tables(ebag_tbe* h, const void* const* tables, const int64_t* 
         if (mapping_len) std::memcpy(&blob[2 * T + t], &mapping_len[t], sizeof(int64_t));
     }
     if (h->slot >= 0 && std::memcmp(h->h_tables[h->slot], blob.data(), bytes) == 0) {
+        // the copy of this block was enqueued on the stream of an earlier call: a launch on
+        // another stream has to be ordered behind it (a device-side wait, the host does not block)
+        if (h->slot_stream[h->slot] != stream)
+            EBAG_CUDA(h, cudaStreamWaitEvent(stream, h->slot_event[h->slot], 0));
         *d_out = h->d_tables[h->slot];
         return EBAG_OK;
     }
@@ -216,6 +221,7 @@ ebag_status stage_tables(ebag_tbe* h, const void* const* tables, const int64_t* 
     EBAG_CUDA(h, cudaMemcpyAsync(h->d_tables[s], h->h_tables[s], bytes, cudaMemcpyHostToDevice, stream));
     EBAG_CUDA(h, cudaEventRecord(h->slot_event[s], stream));
     h->slot_busy[s] = true;
+    h->slot_stream[s] = stream;
     h->slot = s;
     *d_out = h->d_tables[s];
     return EBAG_OK;

@@ -95,15 +95,17 @@ def run_gpu(dtype, rows, D, dev_tables, indices, offsets, B, mode, weights=None,
         tbe.close()
 
 
-def compare(gpu, ref, dtype, lengths=None, T=None, B=None, D=None):
-    """Assert the parity bar; returns max(|gpu - out32| / S) over elements with S > 0."""
+def compare(gpu, ref, dtype, lengths=None, T=None, B=None, D=None, floor=True):
+    """Assert the parity bar; returns max(|gpu - out32| / S) over elements with S > 0.
+    floor=False holds rowwise 8-bit tables to the plain 2e-3 * S as well (the five published
+    workloads are checked that way: none of them needs the floor)."""
     out32, S = ref["out32"], ref["S"]
     assert gpu.shape == out32.shape
     assert not np.isnan(gpu).any(), "an output element was never written"
     tol = TOL[dtype]
     err = np.abs(gpu.astype(np.float64) - out32.astype(np.float64))
     bar = tol * S
-    if dtype in ROWWISE8 and "F" in ref:
+    if floor and dtype in ROWWISE8 and "F" in ref:
         bar = bar + ROWWISE8_FLOOR * ref["F"]
     bad = err > bar
     if bad.any():
@@ -121,7 +123,7 @@ def compare(gpu, ref, dtype, lengths=None, T=None, B=None, D=None):
     return float((err[pos] / S[pos]).max()) if pos.any() else 0.0
 
 
-def check_workload(w, jag=None, tables=None, params=None, host_path=False):
+def check_workload(w, jag=None, tables=None, params=None, host_path=False, floor=True):
     """Element-by-element parity of a (small enough) workload.  Returns the max relative error."""
     jag = jag or wl.gen_jagged(w)
     tables = tables or wl.gen_tables(w, "cpu")
@@ -132,60 +134,4 @@ def check_workload(w, jag=None, tables=None, params=None, host_path=False):
     ref = oracle_forward(tabs, w.dtype, jag.indices, jag.offsets, w.B, w.mode, weights=jag.weights,
                          scales=sc, biases=bi)
     assert status == (eb.EBAG_OK, ref["n_oob"], ref["n_bad_offsets"]) == (0, 0, 0)
-    return compare(gpu, ref, w.dtype, jag.lengths, w.T, w.B, w.D)
-
-
-def sampled_check(w, jag, dev_tables_raw, gpu_out, bags_per_table, seed=0):
-    """Parity at full size on sampled bags: for every table pick ``bags_per_table`` bags (the
-    longest, an empty one if there is one, the first, the last, the rest at random), copy only the
-    rows they reference to the host, renumber, and run the oracle on that compact problem.
-
-    dev_tables_raw: per table the UNPACKED device tensors (for int8 the (q, scale, bias) tuple).
-    gpu_out: device tensor [B, sumD] produced by the library for the full workload."""
-    rng = np.random.default_rng(seed)
-    K = bags_per_table
-    sel_bags, c_tables, c_sc, c_bi = [], [], [], []
-    c_idx, c_w = [], []
-    c_len = []
-    for t in range(w.T):
-        lens = jag.lengths[t * w.B:(t + 1) * w.B]
-        picks = {0, w.B - 1, int(np.argmax(lens))}
-        if (lens == 0).any():
-            picks.add(int(np.argmax(lens == 0)))
-        while len(picks) < min(K, w.B):
-            picks.add(int(rng.integers(0, w.B)))
-        picks = np.array(sorted(picks))[:K]
-        sel_bags.append(picks)
-        segs = [jag.indices[jag.offsets[t * w.B + b]:jag.offsets[t * w.B + b + 1]] for b in picks]
-        flat = np.concatenate(segs) if segs else np.zeros(0, np.int64)
-        uniq, inv = np.unique(flat, return_inverse=True)
-        if uniq.size == 0:
-            uniq = np.zeros(1, np.int64)
-        sel = torch.from_numpy(uniq).cuda()
-        tab = dev_tables_raw[t]
-        if w.dtype in ROWWISE8:
-            c_tables.append(wl.raw_numpy(tab[0].index_select(0, sel)))
-            c_sc.append(wl.raw_numpy(tab[1].index_select(0, sel)))
-            c_bi.append(wl.raw_numpy(tab[2].index_select(0, sel)))
-        else:
-            c_tables.append(wl.raw_numpy(tab.index_select(0, sel)))
-        c_idx.append(inv.astype(np.int64))
-        c_len.append(np.array([s.size for s in segs], dtype=np.int64))
-        if jag.weights is not None:
-            c_w.append(np.concatenate(
-                [jag.weights[jag.offsets[t * w.B + b]:jag.offsets[t * w.B + b + 1]] for b in picks]))
-    Ks = len(sel_bags[0])
-    lengths = np.concatenate(c_len)
-    offsets = np.zeros(w.T * Ks + 1, dtype=np.int64)
-    np.cumsum(lengths, out=offsets[1:])
-    ref = oracle_forward(c_tables, w.dtype, np.concatenate(c_idx), offsets, Ks, w.mode,
-                         weights=np.concatenate(c_w) if c_w else None,
-                         scales=c_sc or None, biases=c_bi or None)
-    assert ref["n_oob"] == 0 and ref["n_bad_offsets"] == 0
-    gpu = np.empty((Ks, w.sumD), dtype=np.float32)
-    col = 0
-    for t in range(w.T):
-        rows_sel = torch.from_numpy(sel_bags[t]).cuda()
-        gpu[:, col:col + w.D[t]] = gpu_out.index_select(0, rows_sel)[:, col:col + w.D[t]].cpu().numpy()
-        col += w.D[t]
-    return compare(gpu, ref, w.dtype, lengths, w.T, Ks, w.D)
+    return compare(gpu, ref, w.dtype, jag.lengths, w.T, w.B, w.D, floor=floor)
