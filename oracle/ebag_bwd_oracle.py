@@ -20,6 +20,14 @@ Plain loops over bags; numpy only for the per-lookup vector arithmetic.
 Pins (tests/test_oracle_bwd.py): the adjoint identity <forward(T), G> = <T, backward(G)> against
 the separately pinned forward oracle, a hand-worked example, closed forms (all lookups on one
 row; one-hot grad_out), linearity in grad_out and the mean/sum relation.
+
+The forward is linear in the per-sample weights as well (the scores of Sec. 2.2's weighted
+sparse features), so their gradient is the other transpose, `backward_weights`:
+    grad_w[i] = (1/L_g in mean mode, else 1) * sum_d grad_out[b, Doff[t] + d] * value(t, indices[i], d)
+for lookup i of bag g = t*B + b; 0 for a skipped id or a malformed bag.  Pins: the adjoint
+identity in the weights, <forward(w), G> = <w, backward_weights(G)>, against the forward oracle; a
+hand-worked example; the all-ones table (every lookup of a bag collects the bag's grad_out row
+sum); agreement with `backward` through sum_i w_i grad_w[i] = <T, backward(G)>.
 """
 from __future__ import annotations
 
@@ -74,3 +82,49 @@ def backward(rows, D, grad_out, indices, offsets, B, mode=SUM, weights=None):
                 counts[t][r] += 1
         col += D[t]
     return dict(grads=grads, S=S, counts=counts, n_oob=n_oob, n_bad_offsets=n_bad)
+
+
+def backward_weights(tables, grad_out, indices, offsets, B, mode=SUM):
+    """tables: T float arrays [rows_t, D_t] holding the VALUES the forward pools (16-bit storage
+    widened, rowwise 8-bit codes dequantised as scale * code + bias in fp32, by the caller).
+    grad_out: [B, sum(D)].  Returns dict(grad_w f64 [n], S f64 [n] = the same sums over absolute
+    values, n_oob, n_bad_offsets)."""
+    T = len(tables)
+    D = [int(t.shape[1]) for t in tables]
+    grad_out = np.asarray(grad_out, dtype=np.float64)
+    indices = np.asarray(indices, dtype=np.int64)
+    offsets = np.asarray(offsets, dtype=np.int64)
+    if offsets.shape[0] != T * B + 1:
+        raise ValueError("offsets must hold T*B+1 entries")
+    if grad_out.shape != (B, int(sum(D))):
+        raise ValueError("grad_out must be [B, sum(D)]")
+    if mode not in (SUM, MEAN):
+        raise ValueError("mode")
+    n = indices.shape[0]
+    gw = np.zeros(n, dtype=np.float64)
+    S = np.zeros(n, dtype=np.float64)
+    n_oob = n_bad = 0
+    col = 0
+    for t in range(T):
+        tab = np.asarray(tables[t], dtype=np.float64)
+        for b in range(B):
+            g = t * B + b
+            lo, hi = int(offsets[g]), int(offsets[g + 1])
+            if lo < 0 or hi < lo or hi > n:
+                n_bad += 1
+                continue
+            L = hi - lo
+            if L == 0:
+                continue
+            go = grad_out[b, col:col + D[t]]
+            if mode == MEAN:
+                go = go / L
+            for i in range(lo, hi):
+                r = int(indices[i])
+                if r < 0 or r >= tab.shape[0]:
+                    n_oob += 1
+                    continue
+                gw[i] += float((go * tab[r]).sum())
+                S[i] += float(np.abs(go * tab[r]).sum())
+        col += D[t]
+    return dict(grad_w=gw, S=S, n_oob=n_oob, n_bad_offsets=n_bad)
