@@ -147,11 +147,35 @@ ebag_status ebag_forward_i32(ebag_tbe* h, const void* const* tables, const int32
  * few KB of metadata), no synchronisation.  Contributions are added with floating-point reductions in
  * memory whose order is not fixed: two runs agree up to fp32 rounding, not bit for bit.  Ids
  * outside the table and malformed bags are skipped and counted as in the forward
- * (ebag_last_status).  The gradient with respect to per_sample_weights is not computed.
+ * (ebag_last_status).  The gradient with respect to per_sample_weights: ebag_backward_weights.
  */
 ebag_status ebag_backward(ebag_tbe* h, const float* grad_out, const void* indices, int32_t index_bits,
                           int64_t n_indices, const int64_t* offsets, const float* per_sample_weights,
                           int64_t B, ebag_mode mode, float* const* grad_tables, ebag_stream stream);
+
+/*
+ * Backward of the pooled forward with respect to the per-sample weights (the scores of the
+ * paper's weighted sparse features, Sec. 2.2 "Feature Types and Memory Layout"; the forward is
+ * linear in them):
+ *     grad_weights[i] = sum_d grad_out[b, Doff[t] + d] * value(t, indices[i], d)     (EBAG_MEAN: / L)
+ * for lookup i of bag (t, b), value() as in the forward (16-bit storage widened, rowwise 8-bit
+ * codes dequantised).  It does not depend on the weights themselves.
+ *   tables, D     as given to the forward (host array [T] of DEVICE pointers; read before the call returns).
+ *   grad_out      device fp32 [B, sum(D)], 16-byte aligned.
+ *   indices       device int64 or int32 ids (index_bits = 64 or 32); offsets, B, mode as given to the forward.
+ *   grad_weights  device fp32 [n_indices]; entry i is written for every lookup of a well-formed
+ *                 bag (0 for an id outside its table, which is counted); entries that no
+ *                 well-formed bag covers are left as they are, and an entry that malformed
+ *                 offsets put into several bags receives the value of one of them.
+ * One kernel on `stream`, no allocation; the sums over a row are added in a fixed order, so two
+ * runs give the same bits.  D[t] must be a multiple of 4.  A bag is walked by one group of lanes,
+ * so a single very long bag is slow (it is not split as in the forward).  Counts of skipped ids
+ * and malformed bags go to ebag_last_status.
+ */
+ebag_status ebag_backward_weights(ebag_tbe* h, const void* const* tables, const int32_t* D,
+                                  const float* grad_out, const void* indices, int32_t index_bits,
+                                  int64_t n_indices, const int64_t* offsets, int64_t B, ebag_mode mode,
+                                  float* grad_weights, ebag_stream stream);
 
 /*
  * The same forward for callers whose per-step data lives in HOST memory: indices, offsets,

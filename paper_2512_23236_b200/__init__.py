@@ -30,6 +30,7 @@ SIGNATURES = {
     "ebag_forward": (_int, [_vp, _vp, _vp, _vp, _i64, _vp, _vp, _i64, _int, _vp, _vp]),
     "ebag_forward_i32": (_int, [_vp, _vp, _vp, _vp, _i64, _vp, _vp, _i64, _int, _vp, _vp]),
     "ebag_backward": (_int, [_vp, _vp, _vp, _i32, _i64, _vp, _vp, _i64, _int, _vp, _vp]),
+    "ebag_backward_weights": (_int, [_vp, _vp, _vp, _vp, _vp, _i32, _i64, _vp, _i64, _int, _vp, _vp]),
     "ebag_forward_host": (_int, [_vp, _vp, _vp, _vp, _i64, _vp, _vp, _i64, _int, _vp, _vp]),
     "ebag_forward_noalloc": (_int, [_i32, _vp, _vp, _int, _vp, _vp, _i64, _vp, _vp, _i64, _int, _vp,
                                     _vp, _vp]),
@@ -333,6 +334,25 @@ class TBE:
                                  _ptr(offsets), _ptr(per_sample_weights), B, mode,
                                  ctypes.cast(arr, _vp), _stream_ptr(stream))
         _check(st, "ebag_backward")
+
+    def backward_weights(self, tables: List, grad_out, indices, offsets, B: int, mode: int = EBAG_SUM,
+                         out=None, stream=None):
+        """Gradient of the forward with respect to the per-sample weights: float32 [n_indices],
+        one dot product of the bag's grad_out slice with the looked-up row per lookup.  Enqueues only."""
+        import torch
+        bits = 32 if indices.dtype == torch.int32 else 64
+        if indices.dtype not in (torch.int32, torch.int64):
+            raise TypeError("indices must be int64 or int32")
+        if out is None:
+            out = torch.zeros(int(indices.numel()), dtype=torch.float32, device=indices.device)
+        if not hasattr(self, "_d_arr"):
+            self._d_arr = (ctypes.c_int32 * self.T)(*self.D)
+            self._d_ptr = ctypes.cast(self._d_arr, _vp)
+        st = lib().ebag_backward_weights(self._h, self._table_array(tables), self._d_ptr, _ptr(grad_out),
+                                         _ptr(indices), bits, int(indices.numel()), _ptr(offsets), B, mode,
+                                         _ptr(out), _stream_ptr(stream))
+        _check(st, "ebag_backward_weights")
+        return out
 
     def forward_mapid(self, tables: List, values, offsets, mappings: List, B: int,
                       mode: int = EBAG_SUM, per_sample_weights=None, out=None, stream=None):

@@ -10,6 +10,7 @@
 
 #include "ebag.h"
 #include "ebag_bwd.cuh"
+#include "ebag_bwd_weights.cuh"
 #include "ebag_fwd.cuh"
 
 using namespace ebag;
@@ -1122,6 +1123,53 @@ ebag_status ebag_forward_host(ebag_tbe* h, const void* const* tables, const int3
     }
     EBAG_CUDA(h, cudaEventRecord(h->ev_join, h->s_d2h));
     EBAG_CUDA(h, cudaStreamWaitEvent(s, h->ev_join, 0));
+    return EBAG_OK;
+}
+
+ebag_status ebag_backward_weights(ebag_tbe* h, const void* const* tables, const int32_t* D,
+                                  const float* grad_out, const void* indices, int32_t index_bits,
+                                  int64_t n_indices, const int64_t* offsets, int64_t B, ebag_mode mode,
+                                  float* grad_weights, ebag_stream stream) {
+    if (!h || !tables || !D || !offsets || B < 0 || n_indices < 0) return EBAG_ERR_INVALID_ARG;
+    if (index_bits != 32 && index_bits != 64) return EBAG_ERR_INVALID_ARG;
+    if (mode != EBAG_SUM && mode != EBAG_MEAN) return EBAG_ERR_INVALID_ARG;
+    if (n_indices > 0 && (!indices || !grad_weights)) return EBAG_ERR_INVALID_ARG;
+    if (B > 0 && !grad_out) return EBAG_ERR_INVALID_ARG;
+    if ((int64_t)h->T * B >= (1ll << 31)) return EBAG_ERR_UNSUPPORTED;
+    if (((uintptr_t)grad_out & 15u) || ((uintptr_t)indices & (index_bits == 32 ? 3u : 7u)) ||
+        ((uintptr_t)offsets & 7u) || ((uintptr_t)grad_weights & 3u))
+        return EBAG_ERR_INVALID_ARG;
+    for (int t = 0; t < h->T; ++t) {
+        if (D[t] != h->D[t]) return EBAG_ERR_INVALID_ARG;
+        if (h->D[t] % 4 != 0) return EBAG_ERR_UNSUPPORTED;          // grad_out slices in 16-byte vectors
+        if (!tables[t] && h->rows[t] > 0) return EBAG_ERR_INVALID_ARG;
+        if ((uintptr_t)tables[t] & 15u) return EBAG_ERR_INVALID_ARG;
+    }
+    if (B == 0) return EBAG_OK;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) return EBAG_ERR_CUDA;
+    cudaStream_t s = (cudaStream_t)stream;
+    const void* const* d_tables = nullptr;
+    ebag_status st = stage_tables(h, tables, nullptr, nullptr, s, &d_tables);
+    if (st != EBAG_OK) return st;
+    BwdWeightsParams p;
+    p.tables = d_tables;
+    p.meta = h->d_meta;
+    p.indices = indices;
+    p.offsets = offsets;
+    p.grad_out = grad_out;
+    p.grad_w = grad_weights;
+    p.status = h->d_status;
+    p.n_indices = n_indices;
+    p.B = B;
+    p.T = h->T;
+    p.sumD = h->sumD;
+    p.mean = mode == EBAG_MEAN ? 1 : 0;
+    p.idx32 = index_bits == 32 ? 1 : 0;
+    p.code_zero = h->dtype == EBAG_UINT8_ROWWISE ? 0.0f : 128.0f;
+    EBAG_CUDA(h, launch_bwd_weights(h->dtype == EBAG_UINT8_ROWWISE ? (int)EBAG_INT8_ROWWISE : h->dtype, p,
+                                    h->num_sms * 6, s));
+    ++h->launches;
     return EBAG_OK;
 }
 

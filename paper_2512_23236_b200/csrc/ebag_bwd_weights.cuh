@@ -1,0 +1,31 @@
+// Parameters of the kernel that computes the gradient of the per-sample weights (ebag_bwd_weights.cu).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "ebag_fwd.cuh"     // TableMeta, Status, Elem
+
+namespace ebag {
+
+struct BwdWeightsParams {
+    const void* const* tables;   // device [T]
+    const TableMeta* meta;       // device [T]
+    const void* indices;         // int64 ids, or int32 when idx32
+    const int64_t* offsets;
+    const float* grad_out;       // [B, sumD]
+    float* grad_w;               // [n_indices]
+    Status* status;
+    int64_t n_indices;
+    int64_t B;
+    int32_t T;
+    int32_t sumD;
+    int32_t mean;
+    int32_t idx32;
+    float code_zero;             // rowwise 8-bit tables: the stored byte that means code 0
+};
+
+size_t bwd_weights_smem_bytes(int T);
+cudaError_t launch_bwd_weights(int dtype, const BwdWeightsParams& p, int grid, cudaStream_t s);
+
+}  // namespace ebag
