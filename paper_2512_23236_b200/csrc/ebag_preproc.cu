@@ -176,9 +176,10 @@ extern "C" ebag_status ebag_mbdt(const float* values, int32_t F, int64_t B, cons
 // user are a prefix of that user's events, so per feature a user's kept inner lengths and kept
 // values are each ONE contiguous range; only user-level prefix sums are needed:
 //   1. scan outer lengths            -> first event of every user, before and after (1 CTA per tile)
-//   2. per (feature, user) sums      -> values held / kept by the user   (a warp per 8 users)
+//   2. per (feature, user) sums      -> values held / kept by the user; the kept inner lengths are
+//                                       written out as they are read       (a warp per 8 users)
 //   3. scan those per feature        -> first value of every user, before and after (1 CTA per tile)
-//   4. copy the two ranges per (feature, user)                            (a warp per 8 users)
+//   4. copy the kept values per (feature, user)                            (a warp per 8 users)
 namespace {
 
 constexpr int kScanThreads = 1024;
@@ -329,7 +330,8 @@ constexpr int kSumBatch = 6;        // bet_user_sums: loads per lane requested o
 // of them, then the warp adds up the users' inner lengths one user after the other.  The grid is
 // one wave of resident CTAs and the (feature, users) tasks are dealt round-robin to its warps.
 __global__ void __launch_bounds__(256, 4)
-bet_user_sums(const int64_t* __restrict__ inner, int64_t E, int64_t U, int F, BetWorkspace w) {
+bet_user_sums(const int64_t* __restrict__ inner, int64_t E, int64_t U, int F, BetWorkspace w,
+              int64_t* __restrict__ inner_out) {
     wait_for_previous_launch();
     const int lane = threadIdx.x & 31;
     const int64_t warps = (int64_t)gridDim.x * (blockDim.x >> 5);
@@ -339,14 +341,17 @@ bet_user_sums(const int64_t* __restrict__ inner, int64_t E, int64_t U, int F, Be
         const int f = (int)(task / chunks);
         const int64_t u0 = (task - (int64_t)f * chunks) * kTaskUsers;
         const int64_t* __restrict__ row = inner + (int64_t)f * E;
+        int64_t* __restrict__ row_out = inner_out + (int64_t)f * E;
         const int64_t u = u0 + lane;
-        int64_t e0 = 0, e1 = 0, keep = 0;
+        int64_t e0 = 0, e1 = 0, keep = 0, eo = 0;
         if (lane < kTaskUsers && u < U) {
             e0 = w.ev_in[u];
             e1 = w.ev_in[u + 1];
-            keep = w.ev_out[u + 1] - w.ev_out[u];
+            eo = w.ev_out[u];
+            keep = w.ev_out[u + 1] - eo;
             if (e1 > E) e1 = E;                       // never read past the caller's array
             if (e0 > e1) e0 = e1;
+            if (keep > e1 - e0) keep = e1 - e0;       // nor write more than was read
         }
         const int users = U - u0 < kTaskUsers ? (int)(U - u0) : kTaskUsers;
         int64_t my_all = 0, my_kept = 0;              // results of user u0 + lane
@@ -367,13 +372,19 @@ bet_user_sums(const int64_t* __restrict__ inner, int64_t E, int64_t U, int F, Be
             const int64_t ke0 = __shfl_sync(0xffffffffu, e0, k);
             const int64_t cnt = __shfl_sync(0xffffffffu, e1, k) - ke0;
             const int64_t kkeep = __shfl_sync(0xffffffffu, keep, k);
+            // the kept inner lengths go to the output as they pass through (they are a prefix of
+            // the user's, so this is the whole copy of that array: the copy kernel moves values only)
+            long long* __restrict__ dst = reinterpret_cast<long long*>(row_out + __shfl_sync(0xffffffffu, eo, k));
             int64_t all = 0, kept = 0;
             const int keep32 = kkeep > 0x7fffffffll ? 0x7fffffff : (int)kkeep;
 #pragma unroll
             for (int q = 0; q < kSumBatch; ++q) {
                 const int64_t n = nonneg(cur[q]);
                 all += n;
-                if (lane + 32 * q < keep32) kept += n;
+                if (lane + 32 * q < keep32) {
+                    kept += n;
+                    __stcs(dst + lane + 32 * q, n);
+                }
             }
             for (int64_t j0 = lane + 32 * kSumBatch; j0 < cnt; j0 += 32 * kCopyBatch) {   // the rest, if any
                 int64_t x[kCopyBatch];
@@ -386,7 +397,10 @@ bet_user_sums(const int64_t* __restrict__ inner, int64_t E, int64_t U, int F, Be
                 for (int q = 0; q < kCopyBatch; ++q) {
                     const int64_t n = nonneg(x[q]);
                     all += n;
-                    if (j0 + 32 * q < kkeep) kept += n;
+                    if (j0 + 32 * q < kkeep) {
+                        kept += n;
+                        __stcs(dst + j0 + 32 * q, n);
+                    }
                 }
             }
             // the lanes' sums added up: one warp reduction each while every lane's sum is below
@@ -443,13 +457,12 @@ __device__ __forceinline__ void warp_copy64(const int64_t* __restrict__ src, int
     }
 }
 
-// A warp takes kTaskUsers consecutive users of a feature at a time: a lane each reads the ranges
-// of one of them, then the warp copies the users' kept inner lengths and kept values, both
-// contiguous per user, one user after the other.  Same task dealing as bet_user_sums.
+// A warp takes kTaskUsers consecutive users of a feature at a time: a lane each reads the range
+// of one of them, then the warp copies the users' kept values, contiguous per user, one user
+// after the other.  Same task dealing as bet_user_sums.
 __global__ void __launch_bounds__(256, 4)
-bet_copy(const int64_t* __restrict__ inner, int64_t E, const int64_t* __restrict__ values,
-         const int64_t* __restrict__ value_offsets, int64_t U, int F, BetWorkspace w,
-         int64_t* __restrict__ inner_out, int64_t* __restrict__ values_out) {
+bet_copy(const int64_t* __restrict__ values, const int64_t* __restrict__ value_offsets, int64_t U, int F,
+         BetWorkspace w, int64_t* __restrict__ values_out) {
     wait_for_previous_launch();
     const int lane = threadIdx.x & 31;
     const int64_t warps = (int64_t)gridDim.x * (blockDim.x >> 5);
@@ -459,15 +472,9 @@ bet_copy(const int64_t* __restrict__ inner, int64_t E, const int64_t* __restrict
         const int f = (int)(task / chunks);
         const int64_t u0 = (task - (int64_t)f * chunks) * kTaskUsers;
         const int64_t vbase = value_offsets[f], vend = value_offsets[f + 1];
-        const int64_t* __restrict__ src_row = inner + (int64_t)f * E;
-        int64_t* __restrict__ dst_row = inner_out + (int64_t)f * E;
         const int64_t u = u0 + lane;
-        int64_t e_in = 0, e_out = 0, keep = 0, v_in = 0, v_out = 0, nv = 0;
+        int64_t v_in = 0, v_out = 0, nv = 0;
         if (lane < kTaskUsers && u < U) {
-            e_in = w.ev_in[u];
-            e_out = w.ev_out[u];
-            keep = w.ev_out[u + 1] - e_out;
-            if (e_in + keep > E) keep = E > e_in ? E - e_in : 0;
             v_in = vbase + w.v_in[(int64_t)f * (U + 1) + u];
             v_out = vbase + w.v_out[(int64_t)f * (U + 1) + u];
             nv = w.v_keep[(int64_t)f * U + u];
@@ -475,12 +482,9 @@ bet_copy(const int64_t* __restrict__ inner, int64_t E, const int64_t* __restrict
         }
         const int users = U - u0 < kTaskUsers ? (int)(U - u0) : kTaskUsers;
         for (int k = 0; k < users; ++k) {
-            const int64_t ke_in = __shfl_sync(0xffffffffu, e_in, k), ke_out = __shfl_sync(0xffffffffu, e_out, k);
-            const int64_t kkeep = __shfl_sync(0xffffffffu, keep, k);
             const int64_t kv_in = __shfl_sync(0xffffffffu, v_in, k), kv_out = __shfl_sync(0xffffffffu, v_out, k);
             const int64_t knv = __shfl_sync(0xffffffffu, nv, k);
-            warp_copy64<true>(src_row + ke_in, dst_row + ke_out, kkeep, lane);
-            warp_copy64<false, 8>(values + kv_in, values_out + kv_out, knv, lane);   // 8 loads in flight: 0.411 -> 0.393 ms (16 spill)
+            warp_copy64<false, 8>(values + kv_in, values_out + kv_out, knv, lane);   // 8 loads in flight
         }
     }
 }
@@ -533,7 +537,7 @@ extern "C" ebag_status ebag_batch_event_truncate(const int64_t* outer_lengths, i
     }
     if (err == cudaSuccess && F > 0 && U > 0) {
         cudaLaunchConfig_t cfg = config(dim3(bet_grid(bet_user_sums, F, U)), 256);
-        err = cudaLaunchKernelEx(&cfg, bet_user_sums, inner_lengths, E, U, (int)F, w);
+        err = cudaLaunchKernelEx(&cfg, bet_user_sums, inner_lengths, E, U, (int)F, w, inner_out);
     }
     if (err == cudaSuccess && F > 0) {
         cudaLaunchConfig_t cfg = config(dim3(tiles, (unsigned)F), kScanThreads);
@@ -541,8 +545,7 @@ extern "C" ebag_status ebag_batch_event_truncate(const int64_t* outer_lengths, i
     }
     if (err == cudaSuccess && F > 0 && U > 0) {
         cudaLaunchConfig_t cfg = config(dim3(bet_grid(bet_copy, F, U)), 256);
-        err = cudaLaunchKernelEx(&cfg, bet_copy, inner_lengths, E, values, value_offsets, U, (int)F, w, inner_out,
-                                 values_out);
+        err = cudaLaunchKernelEx(&cfg, bet_copy, values, value_offsets, U, (int)F, w, values_out);
     }
     if (err != cudaSuccess) {
         cudaGetLastError();
