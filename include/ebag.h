@@ -301,7 +301,8 @@ ebag_status ebag_mbdt(const float* values, int32_t F, int64_t B, const float* bo
  * jagged batch of event features keeps only the first N events of every user, in all F features
  * at once, in four launches whatever F is.
  *   outer_lengths  device int64 [U]: events per user (shared by all features)
- *   inner_lengths  device int64 [F, E] row-major: attributes per event, E = sum(outer_lengths)
+ *   inner_lengths  device int64 [F, E] row-major: attributes per event, E = sum(outer_lengths) < 2^31
+ *                  (more returns EBAG_ERR_UNSUPPORTED)
  *   values         device int64: the attribute values of feature 0, then feature 1, ...;
  *   value_offsets  device int64 [F+1]: feature f owns values[value_offsets[f] .. [f+1])
  *   outer_out      device int64 [U]: min(outer_lengths[u], N)

@@ -336,68 +336,62 @@ bet_user_sums(const int64_t* __restrict__ inner, int64_t E, int64_t U, int F, Be
     const int lane = threadIdx.x & 31;
     const int64_t warps = (int64_t)gridDim.x * (blockDim.x >> 5);
     const int64_t chunks = (U + kTaskUsers - 1) / kTaskUsers;       // per feature
+    auto clamp_e = [&](int64_t x) { return x < 0 ? 0 : (x > E ? E : x); };   // never read or write past the arrays
     for (int64_t task = blockIdx.x * (int64_t)(blockDim.x >> 5) + (threadIdx.x >> 5); task < chunks * F;
          task += warps) {
         const int f = (int)(task / chunks);
         const int64_t u0 = (task - (int64_t)f * chunks) * kTaskUsers;
-        const int64_t* __restrict__ row = inner + (int64_t)f * E;
-        int64_t* __restrict__ row_out = inner_out + (int64_t)f * E;
-        const int64_t u = u0 + lane;
-        int64_t e0 = 0, e1 = 0, keep = 0, eo = 0;
-        if (lane < kTaskUsers && u < U) {
-            e0 = w.ev_in[u];
-            e1 = w.ev_in[u + 1];
-            eo = w.ev_out[u];
-            keep = w.ev_out[u + 1] - eo;
-            if (e1 > E) e1 = E;                       // never read past the caller's array
-            if (e0 > e1) e0 = e1;
-            if (keep > e1 - e0) keep = e1 - e0;       // nor write more than was read
-        }
         const int users = U - u0 < kTaskUsers ? (int)(U - u0) : kTaskUsers;
+        // Lane k holds user u0 + k: its event count, how many of them are kept, and where its kept
+        // inner lengths go, the latter relative to the task's first user (E < 2^31, so 32 bits
+        // hold everything below; the users of a task follow one another in the input, so the
+        // read position simply runs on).
+        const int64_t a0 = clamp_e(w.ev_in[u0]), o0 = clamp_e(w.ev_out[u0]);
+        int c = 0, kp = 0, orel = 0;
+        if (lane < users) {
+            const int64_t a = clamp_e(w.ev_in[u0 + lane]), b = clamp_e(w.ev_in[u0 + lane + 1]);
+            const int64_t oa = clamp_e(w.ev_out[u0 + lane]), ob = clamp_e(w.ev_out[u0 + lane + 1]);
+            c = (int)(b - a);
+            kp = (int)(ob - oa < b - a ? ob - oa : b - a);
+            orel = (int)(oa - o0);
+        }
+        const long long* __restrict__ src = reinterpret_cast<const long long*>(inner + (int64_t)f * E + a0) + lane;
+        long long* __restrict__ dst0 = reinterpret_cast<long long*>(inner_out + (int64_t)f * E + o0) + lane;
         int64_t my_all = 0, my_kept = 0;              // results of user u0 + lane
         // the first kSumBatch * 32 inner lengths of the NEXT user are requested before the
         // current user's are added up, so that a warp always has a user's worth of loads in flight
-        int64_t cur[kSumBatch], nxt[kSumBatch];
-        auto first_batch = [&](int k, int64_t (&x)[kSumBatch]) {
-            const int64_t ke0 = __shfl_sync(0xffffffffu, e0, k & 31);
-            const int64_t cnt = k < users ? __shfl_sync(0xffffffffu, e1, k & 31) - ke0 : 0;
-            const int cnt32 = cnt > 0x7fffffffll ? 0x7fffffff : (int)cnt;      // the batch looks at 192 entries
-            const long long* __restrict__ src = reinterpret_cast<const long long*>(row + ke0) + lane;
+        long long cur[kSumBatch], nxt[kSumBatch];
+        int cnt = __shfl_sync(0xffffffffu, c, 0);
 #pragma unroll
-            for (int q = 0; q < kSumBatch; ++q) x[q] = lane + 32 * q < cnt32 ? __ldcs(src + 32 * q) : 0;
-        };
-        first_batch(0, cur);
+        for (int q = 0; q < kSumBatch; ++q) cur[q] = lane + 32 * q < cnt ? __ldcs(src + 32 * q) : 0;
         for (int k = 0; k < users; ++k) {
-            first_batch(k + 1, nxt);
-            const int64_t ke0 = __shfl_sync(0xffffffffu, e0, k);
-            const int64_t cnt = __shfl_sync(0xffffffffu, e1, k) - ke0;
-            const int64_t kkeep = __shfl_sync(0xffffffffu, keep, k);
+            const int keep = __shfl_sync(0xffffffffu, kp, k);
+            long long* __restrict__ dst = dst0 + __shfl_sync(0xffffffffu, orel, k);
+            const int cnt_n = __shfl_sync(0xffffffffu, c, (k + 1) & 31);     // 0 behind the task's last user
+            const long long* __restrict__ src_n = src + cnt;
+#pragma unroll
+            for (int q = 0; q < kSumBatch; ++q) nxt[q] = lane + 32 * q < cnt_n ? __ldcs(src_n + 32 * q) : 0;
             // the kept inner lengths go to the output as they pass through (they are a prefix of
             // the user's, so this is the whole copy of that array: the copy kernel moves values only)
-            long long* __restrict__ dst = reinterpret_cast<long long*>(row_out + __shfl_sync(0xffffffffu, eo, k));
             int64_t all = 0, kept = 0;
-            const int keep32 = kkeep > 0x7fffffffll ? 0x7fffffff : (int)kkeep;
 #pragma unroll
             for (int q = 0; q < kSumBatch; ++q) {
                 const int64_t n = nonneg(cur[q]);
                 all += n;
-                if (lane + 32 * q < keep32) {
+                if (lane + 32 * q < keep) {
                     kept += n;
-                    __stcs(dst + lane + 32 * q, n);
+                    __stcs(dst + 32 * q, n);
                 }
             }
-            for (int64_t j0 = lane + 32 * kSumBatch; j0 < cnt; j0 += 32 * kCopyBatch) {   // the rest, if any
-                int64_t x[kCopyBatch];
+            for (int j0 = 32 * kSumBatch; j0 < cnt; j0 += 32 * kCopyBatch) {       // the rest, if any
+                long long x[kCopyBatch];
 #pragma unroll
-                for (int q = 0; q < kCopyBatch; ++q) {
-                    const int64_t j = j0 + 32 * q;
-                    x[q] = j < cnt ? __ldcs(reinterpret_cast<const long long*>(row + ke0 + j)) : 0;
-                }
+                for (int q = 0; q < kCopyBatch; ++q) x[q] = lane + j0 + 32 * q < cnt ? __ldcs(src + j0 + 32 * q) : 0;
 #pragma unroll
                 for (int q = 0; q < kCopyBatch; ++q) {
                     const int64_t n = nonneg(x[q]);
                     all += n;
-                    if (j0 + 32 * q < kkeep) {
+                    if (lane + j0 + 32 * q < keep) {
                         kept += n;
                         __stcs(dst + j0 + 32 * q, n);
                     }
@@ -416,12 +410,14 @@ bet_user_sums(const int64_t* __restrict__ inner, int64_t E, int64_t U, int F, Be
                 }
             }
             if (lane == k) { my_all = all; my_kept = kept; }
+            src = src_n;
+            cnt = cnt_n;
 #pragma unroll
             for (int q = 0; q < kSumBatch; ++q) cur[q] = nxt[q];
         }
         if (lane < users) {                            // coalesced
-            w.v_all[(int64_t)f * U + u] = my_all;
-            w.v_keep[(int64_t)f * U + u] = my_kept;
+            w.v_all[(int64_t)f * U + u0 + lane] = my_all;
+            w.v_keep[(int64_t)f * U + u0 + lane] = my_kept;
         }
     }
 }
@@ -520,6 +516,7 @@ extern "C" ebag_status ebag_batch_event_truncate(const int64_t* outer_lengths, i
                                                  int64_t* counts_out, void* workspace,
                                                  int64_t workspace_bytes, ebag_stream stream) {
     if (F < 0 || F > 65535 || U < 0 || E < 0 || N < 0) return EBAG_ERR_INVALID_ARG;
+    if (E >= (1ll << 31)) return EBAG_ERR_UNSUPPORTED;     // positions inside a feature travel in 32 bits
     if (!counts_out) return EBAG_ERR_INVALID_ARG;
     if (U > 0 && (!outer_lengths || !outer_out)) return EBAG_ERR_INVALID_ARG;
     if (F > 0 && (!value_offsets || (E > 0 && (!inner_lengths || !inner_out)))) return EBAG_ERR_INVALID_ARG;
