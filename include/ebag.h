@@ -190,12 +190,20 @@ ebag_status ebag_backward_weights(ebag_tbe* h, const void* const* tables, const 
  * non-decreasing within [0, n_indices] the call falls back to one piece and the device reports
  * the malformed bags as usual.  The staging buffers are (re)allocated inside this call whenever
  * n_indices or B exceed what they hold, so the first call, and any call with larger inputs,
- * allocates and synchronises.
+ * allocates and synchronises.  `out` holds elements of the handle's "out_dtype" (fp32 unless
+ * changed with ebag_set_param; 16-bit output halves the bytes that travel back, which is the
+ * longest leg of this call).
  */
 ebag_status ebag_forward_host(ebag_tbe* h, const void* const* tables, const int32_t* D,
                               const int64_t* indices, int64_t n_indices, const int64_t* offsets,
                               const float* per_sample_weights, int64_t B, ebag_mode mode,
                               float* out, ebag_stream stream);
+
+/* ebag_forward_host for 32-bit ids: `indices` is host int32 [n_indices]; the rest as above. */
+ebag_status ebag_forward_host_i32(ebag_tbe* h, const void* const* tables, const int32_t* D,
+                                  const int32_t* indices, int64_t n_indices, const int64_t* offsets,
+                                  const float* per_sample_weights, int64_t B, ebag_mode mode,
+                                  float* out, ebag_stream stream);
 
 /*
  * Wait for `stream`, then report and clear what the device counted since the last call:

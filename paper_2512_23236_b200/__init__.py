@@ -32,6 +32,7 @@ SIGNATURES = {
     "ebag_backward": (_int, [_vp, _vp, _vp, _i32, _i64, _vp, _vp, _i64, _int, _vp, _vp]),
     "ebag_backward_weights": (_int, [_vp, _vp, _vp, _vp, _vp, _i32, _i64, _vp, _i64, _int, _vp, _vp]),
     "ebag_forward_host": (_int, [_vp, _vp, _vp, _vp, _i64, _vp, _vp, _i64, _int, _vp, _vp]),
+    "ebag_forward_host_i32": (_int, [_vp, _vp, _vp, _vp, _i64, _vp, _vp, _i64, _int, _vp, _vp]),
     "ebag_forward_noalloc": (_int, [_i32, _vp, _vp, _int, _vp, _vp, _i64, _vp, _vp, _i64, _int, _vp,
                                     _vp, _vp]),
     "ebag_mapid": (_int, [_vp, _i64, _vp, _i64, _vp, _vp]),
@@ -113,14 +114,14 @@ def ebag_create_tbe(rows: Sequence[int], D: Sequence[int], dtype: int, device: i
 
 def ebag_forward(h: int, table_ptrs: Sequence[int], D: Sequence[int], indices_ptr, n_indices: int,
                  offsets_ptr, weights_ptr, B: int, mode: int, out_ptr, stream_ptr,
-                 host: bool = False) -> None:
+                 host: bool = False, idx32: bool = False) -> None:
     T = len(table_ptrs)
     tp = (ctypes.c_void_p * T)(*[int(p) if p else None for p in table_ptrs])
     d = (ctypes.c_int32 * T)(*[int(x) for x in D])
-    fn = lib().ebag_forward_host if host else lib().ebag_forward
-    st = fn(h, ctypes.cast(tp, _vp), ctypes.cast(d, _vp), indices_ptr, n_indices, offsets_ptr,
-            weights_ptr, B, mode, out_ptr, stream_ptr)
-    _check(st, "ebag_forward_host" if host else "ebag_forward")
+    name = ("ebag_forward_host" if host else "ebag_forward") + ("_i32" if idx32 else "")
+    st = getattr(lib(), name)(h, ctypes.cast(tp, _vp), ctypes.cast(d, _vp), indices_ptr, n_indices, offsets_ptr,
+                              weights_ptr, B, mode, out_ptr, stream_ptr)
+    _check(st, name)
 
 
 def ebag_forward_noalloc(rows: Sequence[int], D: Sequence[int], dtype: int,
@@ -386,10 +387,14 @@ class TBE:
         The caller synchronises the stream before reading ``out``."""
         import torch
         if out is None:
-            out = torch.empty((B, self.sumD), dtype=torch.float32).pin_memory()
+            out = torch.empty((B, self.sumD), dtype=self._out_torch_dtype()).pin_memory()
+        elif out.dtype != self._out_torch_dtype():
+            raise TypeError("out must have the handle's out_dtype")
+        if indices.dtype not in (torch.int32, torch.int64):
+            raise TypeError("indices must be int64 or int32")
         ebag_forward(self._h, [t.data_ptr() for t in tables], self.D, _ptr(indices),
                      int(indices.numel()), _ptr(offsets), _ptr(per_sample_weights), B, mode,
-                     _ptr(out), _stream_ptr(stream), host=True)
+                     _ptr(out), _stream_ptr(stream), host=True, idx32=indices.dtype == torch.int32)
         return out
 
     def last_status(self, stream=None) -> tuple:

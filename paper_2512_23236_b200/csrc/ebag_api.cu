@@ -1037,15 +1037,21 @@ ebag_status ebag_backward(ebag_tbe* h, const float* grad_out, const void* indice
     return EBAG_OK;
 }
 
-ebag_status ebag_forward_host(ebag_tbe* h, const void* const* tables, const int32_t* D,
-                              const int64_t* indices, int64_t n_indices, const int64_t* offsets,
-                              const float* per_sample_weights, int64_t B, ebag_mode mode,
-                              float* out, ebag_stream stream) {
+namespace {
+// ebag_forward_host and ebag_forward_host_i32: `indices` holds 8-byte ids, or 4-byte ids when
+// idx32; `out` holds elements of the handle's out_dtype.
+ebag_status forward_host(ebag_tbe* h, const void* const* tables, const int32_t* D,
+                         const int64_t* indices, int64_t n_indices, const int64_t* offsets,
+                         const float* per_sample_weights, int64_t B, ebag_mode mode,
+                         float* out, ebag_stream stream, bool idx32) {
     ebag_status st = check_forward_args(h, tables, D, indices, n_indices, offsets,
                                         per_sample_weights, B, mode, out);
     if (st != EBAG_OK) return st;
-    if (h->out_dtype != EBAG_F32) return EBAG_ERR_UNSUPPORTED;      // the host path stages and returns fp32
     if (B == 0) return EBAG_OK;
+    const size_t isz = idx32 ? sizeof(int32_t) : sizeof(int64_t);      // bytes per id
+    const size_t osz = h->out_dtype == EBAG_F32 ? 4 : 2;               // bytes per output element
+    const char* idx_b = reinterpret_cast<const char*>(indices);
+    char* out_b = reinterpret_cast<char*>(out);
     DeviceGuard guard(h->device);
     if (!guard.ok) return EBAG_ERR_CUDA;
     cudaStream_t s = (cudaStream_t)stream;
@@ -1060,7 +1066,7 @@ ebag_status ebag_forward_host(ebag_tbe* h, const void* const* tables, const int3
     // How many bag ranges: enough for copies and kernels to overlap, few enough that a range
     // still moves tens of MB.  The ranges need sane offsets at their borders (read here, on the
     // host); otherwise everything goes in one piece and the device sorts it out.
-    const int64_t bytes = sizeof(int64_t) * (n_indices + n_off) + sizeof(float) * n_out +
+    const int64_t bytes = (int64_t)isz * n_indices + sizeof(int64_t) * n_off + (int64_t)osz * n_out +
                           (per_sample_weights ? sizeof(float) * n_indices : 0);
     int64_t chunks = h->host_chunks;
     if (chunks <= 0) {
@@ -1080,14 +1086,15 @@ ebag_status ebag_forward_host(ebag_tbe* h, const void* const* tables, const int3
     }
     if (chunks == 1) {
         if (n_indices > 0)
-            EBAG_CUDA(h, cudaMemcpyAsync(h->s_indices, indices, sizeof(int64_t) * n_indices, cudaMemcpyHostToDevice, s));
+            EBAG_CUDA(h, cudaMemcpyAsync(h->s_indices, indices, isz * n_indices, cudaMemcpyHostToDevice, s));
         EBAG_CUDA(h, cudaMemcpyAsync(h->s_offsets, offsets, sizeof(int64_t) * n_off, cudaMemcpyHostToDevice, s));
         if (per_sample_weights && n_indices > 0)
             EBAG_CUDA(h, cudaMemcpyAsync(h->s_weights, per_sample_weights, sizeof(float) * n_indices, cudaMemcpyHostToDevice, s));
         st = forward_device(h, tables, h->s_indices, n_indices, h->s_offsets,
-                            per_sample_weights ? h->s_weights : nullptr, B, 0, B, mode, h->s_out, s);
+                            per_sample_weights ? h->s_weights : nullptr, B, 0, B, mode, h->s_out, s, nullptr,
+                            nullptr, idx32);
         if (st != EBAG_OK) return st;
-        EBAG_CUDA(h, cudaMemcpyAsync(out, h->s_out, sizeof(float) * n_out, cudaMemcpyDeviceToHost, s));
+        EBAG_CUDA(h, cudaMemcpyAsync(out, h->s_out, osz * n_out, cudaMemcpyDeviceToHost, s));
         return EBAG_OK;
     }
     // Pipeline: inputs of piece k+1 travel while the kernel works on piece k and the result of
@@ -1104,8 +1111,8 @@ ebag_status ebag_forward_host(ebag_tbe* h, const void* const* tables, const int3
             const int64_t g = (int64_t)t * B;
             const int64_t lo = offsets[g + b0], hi = offsets[g + b1];
             if (hi > lo) {
-                EBAG_CUDA(h, cudaMemcpyAsync(h->s_indices + lo, indices + lo, sizeof(int64_t) * (hi - lo),
-                                             cudaMemcpyHostToDevice, h->s_h2d));
+                EBAG_CUDA(h, cudaMemcpyAsync(reinterpret_cast<char*>(h->s_indices) + isz * lo, idx_b + isz * lo,
+                                             isz * (hi - lo), cudaMemcpyHostToDevice, h->s_h2d));
                 if (per_sample_weights)
                     EBAG_CUDA(h, cudaMemcpyAsync(h->s_weights + lo, per_sample_weights + lo,
                                                  sizeof(float) * (hi - lo), cudaMemcpyHostToDevice, h->s_h2d));
@@ -1114,16 +1121,34 @@ ebag_status ebag_forward_host(ebag_tbe* h, const void* const* tables, const int3
         EBAG_CUDA(h, cudaEventRecord(h->ev_in[c], h->s_h2d));
         EBAG_CUDA(h, cudaStreamWaitEvent(s, h->ev_in[c], 0));
         st = forward_device(h, tables, h->s_indices, n_indices, h->s_offsets,
-                            per_sample_weights ? h->s_weights : nullptr, B, b0, b1, mode, h->s_out, s);
+                            per_sample_weights ? h->s_weights : nullptr, B, b0, b1, mode, h->s_out, s, nullptr,
+                            nullptr, idx32);
         if (st != EBAG_OK) return st;
         EBAG_CUDA(h, cudaEventRecord(h->ev_done[c], s));
         EBAG_CUDA(h, cudaStreamWaitEvent(h->s_d2h, h->ev_done[c], 0));
-        EBAG_CUDA(h, cudaMemcpyAsync(out + b0 * (int64_t)h->sumD, h->s_out + b0 * (int64_t)h->sumD,
-                                     sizeof(float) * (b1 - b0) * h->sumD, cudaMemcpyDeviceToHost, h->s_d2h));
+        EBAG_CUDA(h, cudaMemcpyAsync(out_b + osz * b0 * h->sumD, reinterpret_cast<char*>(h->s_out) + osz * b0 * h->sumD,
+                                     osz * (b1 - b0) * h->sumD, cudaMemcpyDeviceToHost, h->s_d2h));
     }
     EBAG_CUDA(h, cudaEventRecord(h->ev_join, h->s_d2h));
     EBAG_CUDA(h, cudaStreamWaitEvent(s, h->ev_join, 0));
     return EBAG_OK;
+}
+}  // namespace
+
+ebag_status ebag_forward_host(ebag_tbe* h, const void* const* tables, const int32_t* D,
+                              const int64_t* indices, int64_t n_indices, const int64_t* offsets,
+                              const float* per_sample_weights, int64_t B, ebag_mode mode,
+                              float* out, ebag_stream stream) {
+    return forward_host(h, tables, D, indices, n_indices, offsets, per_sample_weights, B, mode, out, stream,
+                        false);
+}
+
+ebag_status ebag_forward_host_i32(ebag_tbe* h, const void* const* tables, const int32_t* D,
+                                  const int32_t* indices, int64_t n_indices, const int64_t* offsets,
+                                  const float* per_sample_weights, int64_t B, ebag_mode mode,
+                                  float* out, ebag_stream stream) {
+    return forward_host(h, tables, D, reinterpret_cast<const int64_t*>(indices), n_indices, offsets,
+                        per_sample_weights, B, mode, out, stream, true);
 }
 
 ebag_status ebag_backward_weights(ebag_tbe* h, const void* const* tables, const int32_t* D,

@@ -90,6 +90,31 @@ def test_host_buffer_entry_point(chunks):
                       host_path=True, params=params)
 
 
+@pytest.mark.parametrize("chunks", [1, 3])
+@pytest.mark.parametrize("idx32", [False, True])
+@pytest.mark.parametrize("out_dtype", [wl.F32, wl.F16, wl.BF16])
+def test_host_buffer_entry_point_with_narrow_ids_and_output(chunks, idx32, out_dtype):
+    """Host buffers with 32-bit ids and / or 16-bit output: bit for bit what the device entry point
+    gives for the same settings (which the tests above and below hold to the oracle)."""
+    w = wl.make_workload(3, scale_rows=0.004, scale_B=1 / 97, max_tables=5)
+    jag = wl.gen_jagged(w)
+    dev = pu.device_tables(w.dtype, wl.gen_tables(w, "cpu"))
+    idx = torch.from_numpy(jag.indices.astype(np.int32) if idx32 else jag.indices)
+    off = torch.from_numpy(jag.offsets)
+    tbe = eb.TBE(w.rows, w.D, w.dtype, device=torch.cuda.current_device())
+    try:
+        tbe.set_param("out_dtype", out_dtype)
+        tbe.set_param("host_chunks", chunks)
+        want = tbe.forward(dev, idx.cuda(), off.cuda(), w.B, w.mode)
+        got = tbe.forward_host(dev, idx.pin_memory(), off.pin_memory(), w.B, w.mode)
+        assert tbe.last_status() == (0, 0, 0)
+    finally:
+        tbe.close()
+    assert got.dtype == want.dtype and got.dtype == {wl.F32: torch.float32, wl.F16: torch.float16,
+                                                     wl.BF16: torch.bfloat16}[out_dtype]
+    assert torch.equal(got, want.cpu())
+
+
 def test_host_buffer_entry_point_with_malformed_offsets_falls_back():
     rng = np.random.default_rng(12)
     rows, D, B = [100, 50], [16, 8], 40
