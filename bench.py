@@ -84,6 +84,8 @@ def parse_args():
     ap.add_argument("--split-bytes", type=int, default=-1,
                     help="bags gathering this many bytes or more are pooled in parts (0: never)")
     ap.add_argument("--ctas-per-sm", type=int, default=0)
+    ap.add_argument("--bwd-sorted", type=int, default=-1,
+                    help="workload 9: 1/0 = the reproducible (sorted) / the reduction backward; -1: the library's default")
     # shrunk variants of a workload, for profiler captures and quick checks (not bench lines)
     ap.add_argument("--max-tables", type=int, default=0)
     ap.add_argument("--scale-rows", type=float, default=1.0)
@@ -553,6 +555,8 @@ def run_bwd(args, rank, local_rank, world):
     h_status = torch.zeros(2, dtype=torch.int64).pin_memory()
     flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
     tbe = eb.TBE(base.rows, base.D, wl.F32, device=local_rank)
+    if args.bwd_sorted >= 0:
+        tbe.set_param("bwd_sorted", args.bwd_sorted)
     stream = torch.cuda.Stream(device=dev)
     sampler = bl.ClockSampler(f"GPU-{torch.cuda.get_device_properties(dev).uuid}").start()
     with torch.cuda.stream(stream):

@@ -10,6 +10,7 @@
 
 #include "ebag.h"
 #include "ebag_bwd.cuh"
+#include "ebag_bwd_sorted.cuh"
 #include "ebag_bwd_weights.cuh"
 #include "ebag_fwd.cuh"
 
@@ -51,6 +52,9 @@ struct ebag_tbe {
     BwdTableMeta* d_bwd_meta = nullptr;            // built by the first ebag_backward
     int32_t* d_bwd_hot = nullptr;                  // [T, kHotSlots] sampled hot rows of the current call
     int bwd_occupancy[2] = {};
+    int bwd_sorted = 1;                            // 1: lookups sorted by row, summed run by run (reproducible); 0: reductions
+    void* s_bwd = nullptr;                         // scratch of the sorted backward, grown with the calls
+    int64_t cap_bwd = 0;
     Queue* d_queue = nullptr;
     Status* d_status = nullptr;
     // per-call pointer block [tables T][mappings T][mapping lengths T]: cached on the device,
@@ -128,6 +132,7 @@ void free_handle(ebag_tbe* h) {
         if (h->ev_done[i]) cudaEventDestroy(h->ev_done[i]);
     }
     cudaFree(h->s_indices);
+    cudaFree(h->s_bwd);
     cudaFree(h->s_maphash);
     cudaFree(h->d_map_base);
     cudaFree(h->s_offsets);
@@ -1030,7 +1035,46 @@ ebag_status ebag_backward(ebag_tbe* h, const float* grad_out, const void* indice
     p.idx32 = index_bits == 32 ? 1 : 0;
     p.hot = h->d_bwd_hot;
     p.use_cache = 1;
+    p.only_if = nullptr;
     const bool w = per_sample_weights != nullptr;
+    // The reproducible path: lookups sorted by row, every run of equal rows added up in the order
+    // of the lookups and written once.  It needs offsets that do not decrease (checked on the
+    // device: if they do, its kernels return at once and the reduction kernel below runs instead).
+    int64_t max_rows = 1;
+    int max_d = 4;
+    for (int t = 0; t < h->T; ++t) {
+        max_rows = std::max<int64_t>(max_rows, h->rows[t]);
+        max_d = std::max<int>(max_d, h->D[t]);
+    }
+    if (h->bwd_sorted && n_indices > 0 && n_indices < (1ll << 32) && max_d <= kSortedMaxD) {
+        const bool scaled = w || mode == EBAG_MEAN;
+        const size_t need = bwd_sorted_scratch_bytes(n_indices, h->T, max_d, scaled);
+        char* scratch = static_cast<char*>(h->s_bwd);
+        if ((st = grow(h, &scratch, &h->cap_bwd, (int64_t)need)) != EBAG_OK) return st;
+        h->s_bwd = scratch;
+        BwdSortedParams q;
+        q.grad_tables = p.grad_tables;
+        q.meta = p.meta;
+        q.indices = indices;
+        q.offsets = offsets;
+        q.weights = per_sample_weights;
+        q.grad_out = grad_out;
+        q.status = h->d_status;
+        q.n_indices = n_indices;
+        q.B = B;
+        q.T = h->T;
+        q.sumD = h->sumD;
+        q.mean = p.mean;
+        q.idx32 = p.idx32;
+        bwd_sorted_carve(q, h->s_bwd, n_indices, h->T, max_d, scaled);
+        int bits = 1;
+        while (bits < 32 && (1ll << bits) <= max_rows) ++bits;       // the key of a skipped id is rows[t] itself
+        q.passes = (bits + 7) / 8;
+        int launches = 0;
+        EBAG_CUDA(h, launch_bwd_sorted(q, h->num_sms, s, &launches));
+        h->launches += launches;
+        p.only_if = q.ctl;
+    }
     const int grid = h->num_sms * h->bwd_occupancy[w ? 1 : 0];
     EBAG_CUDA(h, launch_bwd(p, w, grid, s));
     h->launches += 2;                           // the hot-row sampler, then the backward kernel
@@ -1252,6 +1296,11 @@ ebag_status ebag_set_param(ebag_tbe* h, const char* name, int64_t value) {
     if (std::strcmp(name, "item_bytes") == 0) {
         if (value < 256 || value > (1ll << 30)) return EBAG_ERR_INVALID_ARG;
         h->item_bytes = (uint32_t)value;
+        return EBAG_OK;
+    }
+    if (std::strcmp(name, "bwd_sorted") == 0) {
+        if (value != 0 && value != 1) return EBAG_ERR_INVALID_ARG;
+        h->bwd_sorted = (int)value;
         return EBAG_OK;
     }
     if (std::strcmp(name, "split_bytes") == 0) {

@@ -60,6 +60,7 @@ __device__ __forceinline__ int64_t load_id(const void* indices, int idx32, int64
 // the kHotRows largest counts are picked one after the other.  A row must show up at least
 // three times in the sample to be named.
 __global__ void __launch_bounds__(kBwdThreads) bwd_hot_rows_kernel(const BwdParams p) {
+    if (p.only_if && *p.only_if == 0) return;
     __shared__ int keys[kSampleSlots];
     __shared__ int counts[kSampleSlots];
     __shared__ unsigned long long best;
@@ -124,6 +125,7 @@ __global__ void __launch_bounds__(kBwdThreads) bwd_hot_rows_kernel(const BwdPara
 
 template <bool WEIGHTED>
 __global__ void __launch_bounds__(kBwdThreads, 3) ebag_bwd_kernel(const BwdParams p) {
+    if (p.only_if && *p.only_if == 0) return;
     extern __shared__ __align__(16) unsigned char smem_raw[];
     // per warp: kCacheFloats floats of sums, then kHotSlots ids and kHotSlots flags; after all
     // warps: item_base[T+1]

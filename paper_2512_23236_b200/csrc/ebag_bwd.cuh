@@ -39,6 +39,7 @@ struct BwdParams {
     int32_t idx32;
     int32_t* hot;                // [T, kHotSlots] frequent rows of every table by a sample, at their hash slot (-1: none)
     int32_t use_cache;           // 0: hot rows are not looked for
+    const int32_t* only_if;      // null, or a device word: both kernels return at once while it is 0
 };
 
 size_t bwd_smem_bytes(int T);

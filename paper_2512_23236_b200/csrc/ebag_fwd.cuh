@@ -690,10 +690,9 @@ __device__ __forceinline__ void process_item(const FwdParams& p, const TableMeta
                 if (DT == DT_INT8) {
                     sb = lds64f(my_sb_s + (st * kStageVecs + u) * 64);
                     if (POOL == 0) {
-                        acc_bias = fmaf(wu, sb.y, acc_bias);
-                        wu *= sb.x;
-                        acc_bias = fmaf(wu, -p.code_zero, acc_bias);
-                        wu *= kInt8Up;
+                        // the row's constant, bias - zero * scale, rounded once; then the weight
+                        acc_bias = fmaf(wu, fmaf(-p.code_zero, sb.x, sb.y), acc_bias);
+                        wu *= sb.x * kInt8Up;
                     }
                 }
 #pragma unroll
@@ -714,10 +713,9 @@ __device__ __forceinline__ void process_item(const FwdParams& p, const TableMeta
                 if (DT == DT_INT8) {
                     sb = lds64f(my_sb_s + (st * kStageVecs + u) * 64);
                     if (POOL == 0) {
-                        acc_bias = fmaf(wu, sb.y, acc_bias);
-                        wu *= sb.x;
-                        acc_bias = fmaf(wu, -p.code_zero, acc_bias);
-                        wu *= kInt8Up;
+                        // the row's constant, bias - zero * scale, rounded once; then the weight
+                        acc_bias = fmaf(wu, fmaf(-p.code_zero, sb.x, sb.y), acc_bias);
+                        wu *= sb.x * kInt8Up;
                     }
                 }
 #pragma unroll

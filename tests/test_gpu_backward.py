@@ -38,9 +38,11 @@ def _problem(rng, rows, D, B, max_len, weighted, zipf=False):
     return lengths, off, idx, w, G
 
 
-def _run(dtype, rows, D, B, off, idx, w, G, mode, start=None):
+def _run(dtype, rows, D, B, off, idx, w, G, mode, start=None, params=None):
     tbe = eb.TBE(rows, D, dtype, device=torch.cuda.current_device())
     try:
+        for k, v in (params or {}).items():
+            tbe.set_param(k, v)
         grads = [torch.zeros(r, d, device="cuda") if start is None else torch.from_numpy(start[t]).cuda()
                  for t, (r, d) in enumerate(zip(rows, D))]
         tbe.backward(torch.from_numpy(G).cuda(), torch.from_numpy(idx).cuda(), torch.from_numpy(off).cuda(),
@@ -138,6 +140,52 @@ def test_many_warps_and_tables_against_an_index_add_in_fp64():
         err = np.abs(got[t].astype(np.float64) - ref)
         assert np.all(err <= (8.0 * np.sqrt(n) + 4.0) * U * S), t
         assert not got[t][n[:, 0] == 0].any()
+        col += d
+
+
+@pytest.mark.parametrize("mode,weighted,idx32", [(wl.SUM, False, False), (wl.MEAN, True, False), (wl.SUM, True, True)])
+def test_sorted_path_is_reproducible_and_agrees_with_the_reductions(mode, weighted, idx32):
+    """0.9 M skewed lookups over five tables (several sorting tiles per table, hot rows whose runs
+    span many sub-chunks, row ids that need one, two and three sorting passes, an empty table
+    segment): the default path (lookups sorted by row) gives the same bits on every run, and both
+    it and the reduction kernel meet the bar against an fp64 index_add."""
+    rng = np.random.default_rng(23 + mode)
+    rows, D, B = [40_000, 200, 70_000, 9, 300_000], [64, 256, 32, 128, 8], 5000
+    lengths, off, idx, w, G = _problem(rng, rows, D, B, 70, weighted, zipf=True)
+    # table 3 gets no lookups at all
+    lo3, hi3 = int(off[3 * B]), int(off[4 * B])
+    idx = np.concatenate([idx[:lo3], idx[hi3:]])
+    if w is not None:
+        w = np.concatenate([w[:lo3], w[hi3:]])
+    lengths[3 * B:4 * B] = 0
+    off = np.zeros_like(off)
+    np.cumsum(lengths, out=off[1:])
+    idx[::1013] = -1                                       # skipped ids
+    ids = idx.astype(np.int32) if idx32 else idx
+    a, st_a = _run(wl.F32, rows, D, B, off, ids, w, G, mode)
+    b, st_b = _run(wl.F32, rows, D, B, off, ids, w, G, mode)
+    c, st_c = _run(wl.F32, rows, D, B, off, ids, w, G, mode, params=dict(bwd_sorted=0))
+    n_skipped = int((idx < 0).sum())
+    assert st_a == st_b == st_c == (eb.EBAG_ERR_INDEX_OOB, n_skipped, 0)
+    for x, y in zip(a, b):
+        assert np.array_equal(x.view(np.uint32), y.view(np.uint32)), "two runs differ"
+    col = 0
+    for t, (r, d) in enumerate(zip(rows, D)):
+        lo, hi = int(off[t * B]), int(off[(t + 1) * B])
+        bag = np.repeat(np.arange(B), lengths[t * B:(t + 1) * B])
+        scale = np.ones(hi - lo) if w is None else w[lo:hi].astype(np.float64)
+        if mode == wl.MEAN:
+            scale = scale / np.repeat(lengths[t * B:(t + 1) * B], lengths[t * B:(t + 1) * B])
+        keep = idx[lo:hi] >= 0
+        terms = torch.from_numpy(G[bag, col:col + d].astype(np.float64) * scale[:, None])[keep]
+        tid = torch.from_numpy(idx[lo:hi][keep])
+        ref = torch.zeros(r, d, dtype=torch.float64).index_add_(0, tid, terms).numpy()
+        S = torch.zeros(r, d, dtype=torch.float64).index_add_(0, tid, terms.abs()).numpy()
+        n = np.bincount(idx[lo:hi][keep], minlength=r)[:, None].astype(np.float64)
+        for got in (a[t], c[t]):
+            err = np.abs(got.astype(np.float64) - ref)
+            assert np.all(err <= (8.0 * np.sqrt(n) + 4.0) * U * S), t
+            assert not got[n[:, 0] == 0].any()
         col += d
 
 
