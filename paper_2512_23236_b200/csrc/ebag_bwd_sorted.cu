@@ -381,10 +381,10 @@ __global__ void __launch_bounds__(256, EBAG_RUNSUM_BLOCKS) bwds_run_sums_kernel(
         // the keys, bags and weights of the next 32 lookups are requested before the current 32 are worked on
         auto fetch = [&](uint32_t base, uint32_t& kk, uint32_t& bb, float& ww) {
             const bool have = base + lane < s1;
-            const uint2 x = have ? kb[base + lane] : make_uint2(kNoRow, 0u);
+            const uint2 x = have ? __ldcs(kb + base + lane) : make_uint2(kNoRow, 0u);
             kk = x.x;
             bb = x.y;
-            ww = (WEIGHTS && have) ? wts[base + lane] : 1.0f;
+            ww = (WEIGHTS && have) ? __ldcs(wts + base + lane) : 1.0f;
         };
         uint32_t kk, bb, kk_n, bb_n;
         float ww, ww_n;
