@@ -141,12 +141,20 @@ ebag_status ebag_forward_i32(ebag_tbe* h, const void* const* tables, const int32
  *   grad_tables  host array [T] of DEVICE pointers to dense fp32 [rows[t], D[t]] arrays (whatever
  *                the storage type of the tables), 16-byte aligned, owned and zeroed by the caller:
  *                the call ADDS into them.  Needs D[t] % 4 == 0 (else UNSUPPORTED).
- * Two kernel launches on `stream` (a short one that samples the ids of every table for its most
- * frequent rows, whose contributions are then summed in shared memory before they reach the
- * gradient table, and the backward proper), no allocation after the first call (which builds a
- * few KB of metadata), no synchronisation.  Contributions are added with floating-point reductions in
- * memory whose order is not fixed: two runs agree up to fp32 rounding, not bit for bit.  Ids
- * outside the table and malformed bags are skipped and counted as in the forward
+ * By default the lookups of every table are sorted by row (a stable radix sort, in device scratch
+ * the handle keeps: about 16 bytes per lookup, 24 with weights or EBAG_MEAN; grown, with a device
+ * synchronisation, when a larger call arrives: the only allocation) and every run of equal rows
+ * is added up in the order of the lookups and added into its gradient row once.  No
+ * floating-point atomics meet on one address, so two runs of the same call give the same bits
+ * (3 + 3 * passes + 2 kernel launches on `stream`, passes = the 8-bit digits the largest table's
+ * row count needs).  That path needs offsets that do not decrease, which is checked on the
+ * device, n_indices < 2^32 and D[t] <= 256; otherwise, and with ebag_set_param("bwd_sorted", 0),
+ * the call runs the reduction kernel: a short launch that samples the ids of every table for its
+ * most frequent rows, whose contributions are then summed in shared memory, and the backward
+ * proper, which adds every contribution with a floating-point reduction in memory; their order
+ * is not fixed, so two runs then agree up to fp32 rounding, not bit for bit.  (Both kernels are
+ * launched either way; the ones that are not needed return at once.)  Ids outside the table and
+ * malformed bags are skipped and counted as in the forward
  * (ebag_last_status).  The gradient with respect to per_sample_weights: ebag_backward_weights.
  */
 ebag_status ebag_backward(ebag_tbe* h, const float* grad_out, const void* indices, int32_t index_bits,
@@ -379,7 +387,9 @@ ebag_status ebag_forward_noalloc(int32_t T, const int64_t* rows, const int32_t* 
  *                  ebag_forward_mapid: EBAG_F32 (default), EBAG_F16 or EBAG_BF16.  Sums are still
  *                  accumulated in fp32 and rounded to nearest-even once, when the bag is written;
  *                  `out` then points at [B, sum(D)] 16-bit elements (same alignment rule).
- *                  ebag_forward_host returns UNSUPPORTED unless it is EBAG_F32.
+ *                  ebag_forward_host and ebag_forward_host_i32 return 16-bit elements too.
+ *   "bwd_sorted"   ebag_backward: 1 (default) = the reproducible path (lookups sorted by row),
+ *                  0 = floating-point reductions in memory (see ebag_backward)
  *   "split_bytes"  a bag whose rows add up to this many bytes or more (rows narrower than 256
  *                  bytes count as 256) is pooled in parts by many warps instead of by one, the
  *                  partial sums added in lookup order by a second, short kernel launched after
