@@ -2,7 +2,14 @@
 gradient row widths on both sides of the reproducible path's 256-column limit, row counts that
 need one to three sorting passes, bag lengths from all-empty to thousands, skipped ids, weights,
 mean, both id widths.  ebag_backward against the backward oracle (and bit for bit against a second
-run when the reproducible path applies), ebag_backward_weights against its oracle."""
+run when the reproducible path applies), ebag_backward_weights against its oracle.
+
+The bar per gradient element is the one of tests/test_gpu_backward.py, (8 * sqrt(n) + 4) * u * S,
+plus n / 16 * u * S: the generator can send thousands of lookups of ONE bag to one row of a tiny
+table, i.e. add the same fp32 value n times, and then the roundings all go one way (the error grows
+like n, not like sqrt(n); a longer run of these seeds measured up to 1.05 of the plain bar in four
+of 364 cases, for the reduction kernel and the sorted path alike).  The worst case of a sequential
+sum is (n - 1) * u * S, sixteen times above what is added here."""
 import numpy as np
 import pytest
 import torch
@@ -65,7 +72,7 @@ def test_random_backward(seed):
     for t, g in enumerate(outs[0]):
         err = np.abs(g.astype(np.float64) - ref["grads"][t])
         n = ref["counts"][t][:, None].astype(np.float64)
-        assert np.all(err <= (8.0 * np.sqrt(n) + 4.0) * U * ref["S"][t]), (seed, t)
+        assert np.all(err <= (8.0 * np.sqrt(n) + n / 16.0 + 4.0) * U * ref["S"][t]), (seed, t)
         assert not g[ref["counts"][t] == 0].any()
         if max(Ds) <= 256 and idx.size:                      # the reproducible path ran
             assert np.array_equal(g.view(np.uint32), outs[1][t].view(np.uint32)), (seed, t)
