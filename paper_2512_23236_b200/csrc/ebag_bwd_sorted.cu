@@ -181,8 +181,8 @@ __global__ void __launch_bounds__(256) bwds_scan_kernel(const BwdSortedParams p)
     if (threadIdx.x == 0) p.totals[t * 256 + d] = carry_s;
 }
 
-// ---- 4c. stable scatter of a tile.  Warp w owns lookups [w * 256, (w + 1) * 256) of the tile,
-// 32 consecutive ones per round, so "earlier in the tile" is: a lower warp, an earlier round, a
+// ---- 4c. stable scatter of a tile.  Warp w owns an eighth of the tile's lookups, consecutive ones,
+// 32 per round, so "earlier in the tile" is: a lower warp, an earlier round, a
 // lower lane.  The tile is first put in order in shared memory and then written out, so that
 // every run of equal digits leaves as one contiguous, coalesced piece.
 template <bool WEIGHTS>
@@ -194,8 +194,9 @@ __global__ void __launch_bounds__(256) bwds_scatter_kernel(const BwdSortedParams
     __shared__ uint32_t warp_sum[8];
     __shared__ uint32_t gstart[256];                      // where the tile's lookups with digit d go in the output
     __shared__ uint32_t lstart[256];                      // where they sit in the ordered tile
-    __shared__ uint2 s_kb[kSortTile];
-    __shared__ float s_w[WEIGHTS ? kSortTile : 1];
+    extern __shared__ __align__(16) unsigned char tile_smem[];   // the ordered tile: (row, bag) pairs, then weights
+    uint2* s_kb = reinterpret_cast<uint2*>(tile_smem);
+    float* s_w = reinterpret_cast<float*>(tile_smem + (size_t)kSortTile * sizeof(uint2));
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
     const int t = table_of_tile(p.tile_base, p.T, tile);
     const uint32_t k = tile - p.tile_base[t], nt = p.tile_base[t + 1] - p.tile_base[t];
@@ -220,12 +221,13 @@ __global__ void __launch_bounds__(256) bwds_scatter_kernel(const BwdSortedParams
 
     const uint2* __restrict__ kb = p.kb[side];
     const float* __restrict__ wts = WEIGHTS ? p.wts[side] : nullptr;
-    uint2 e[8];
-    uint32_t where[8];                                    // digit << 16 | rank among the warp's earlier lookups of that digit
-    float wt[8];
+    constexpr int kRounds = kSortTile / 256;              // a warp owns kRounds * 32 consecutive lookups of the tile
+    uint2 e[kRounds];
+    uint32_t where[kRounds];                              // digit << 16 | rank among the warp's earlier lookups of that digit
+    float wt[kRounds];
 #pragma unroll
-    for (int r = 0; r < 8; ++r) {
-        const uint32_t pos = s0 + wid * 256 + r * 32 + lane;
+    for (int r = 0; r < kRounds; ++r) {
+        const uint32_t pos = s0 + (wid * kRounds + r) * 32 + lane;
         const bool have = pos < s1;
         e[r] = have ? kb[pos] : make_uint2(0u, 0u);
         wt[r] = (WEIGHTS && have) ? wts[pos] : 0.0f;
@@ -265,8 +267,8 @@ __global__ void __launch_bounds__(256) bwds_scatter_kernel(const BwdSortedParams
     }
     __syncthreads();
 #pragma unroll
-    for (int r = 0; r < 8; ++r) {
-        const uint32_t pos = s0 + wid * 256 + r * 32 + lane;
+    for (int r = 0; r < kRounds; ++r) {
+        const uint32_t pos = s0 + (wid * kRounds + r) * 32 + lane;
         if (pos < s1) {
             const uint32_t d = where[r] >> 16;
             const uint32_t l = lstart[d] + wcnt[wid][d] + (where[r] & 0xffffu);
@@ -522,7 +524,13 @@ void bwd_sorted_carve(BwdSortedParams& p, void* scratch, int64_t n, int T, int D
 
 cudaError_t launch_bwd_sorted(const BwdSortedParams& p, int num_sms, cudaStream_t s, int* launches) {
     int count = 0;
-    cudaError_t e = cudaMemsetAsync(p.ctl, 0, 256, s);
+    cudaError_t e = cudaFuncSetAttribute(reinterpret_cast<const void*>(bwds_scatter_kernel<true>),
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, kSortTile * 12);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(reinterpret_cast<const void*>(bwds_scatter_kernel<false>),
+                             cudaFuncAttributeMaxDynamicSharedMemorySize, kSortTile * 8);
+    if (e != cudaSuccess) return e;
+    e = cudaMemsetAsync(p.ctl, 0, 256, s);
     if (e != cudaSuccess) return e;
     const int wave = num_sms * 8;
     bwds_check_kernel<<<wave, 256, 0, s>>>(p);
@@ -533,8 +541,8 @@ cudaError_t launch_bwd_sorted(const BwdSortedParams& p, int num_sms, cudaStream_
     for (int pass = 0; pass < p.passes; ++pass) {
         bwds_hist_kernel<<<p.max_tiles, 256, 0, s>>>(p, side, 8 * pass);
         bwds_scan_kernel<<<dim3(256, (unsigned)p.T), 256, 0, s>>>(p);
-        if (p.wts[0]) bwds_scatter_kernel<true><<<p.max_tiles, 256, 0, s>>>(p, side, 8 * pass);
-        else bwds_scatter_kernel<false><<<p.max_tiles, 256, 0, s>>>(p, side, 8 * pass);
+        if (p.wts[0]) bwds_scatter_kernel<true><<<p.max_tiles, 256, kSortTile * 12, s>>>(p, side, 8 * pass);
+        else bwds_scatter_kernel<false><<<p.max_tiles, 256, kSortTile * 8, s>>>(p, side, 8 * pass);
         side ^= 1;
         count += 3;
     }
