@@ -11,7 +11,7 @@ namespace ebag {
 
 constexpr int kSortTile = 2048;          // lookups per sorting tile (one CTA; 1024 and 4096 measured: 8.46 and 9.57 ms against 8.15 ms)
 constexpr int kSubChunk = 1024;          // lookups a warp sums in one go (512 and 2048 measured: 8.79 and 8.18 ms against 8.15 ms)
-constexpr int kSortedMaxD = 256;         // widest gradient row the run sums hold in registers
+constexpr int kSortedMaxD = 8192;        // widest gradient row (the run sums walk it in column tiles of 128; the cut-run scratch grows with it)
 
 struct BwdSortedParams {
     float* const* grad_tables;   // device [T]

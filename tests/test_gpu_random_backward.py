@@ -1,5 +1,5 @@
 """Randomized shapes through both backward entry points: table count (empty tables included),
-gradient row widths on both sides of the reproducible path's 256-column limit, row counts that
+gradient row widths from one vector to three column tiles, row counts that
 need one to three sorting passes, bag lengths from all-empty to thousands, skipped ids, weights,
 mean, both id widths.  ebag_backward against the backward oracle (and bit for bit against a second
 run when the reproducible path applies), ebag_backward_weights against its oracle.
@@ -74,7 +74,7 @@ def test_random_backward(seed):
         n = ref["counts"][t][:, None].astype(np.float64)
         assert np.all(err <= (8.0 * np.sqrt(n) + n / 16.0 + 4.0) * U * ref["S"][t]), (seed, t)
         assert not g[ref["counts"][t] == 0].any()
-        if max(Ds) <= 256 and idx.size:                      # the reproducible path ran
+        if idx.size:                                         # the reproducible path ran
             assert np.array_equal(g.view(np.uint32), outs[1][t].view(np.uint32)), (seed, t)
 
 
