@@ -116,6 +116,18 @@ __global__ void __launch_bounds__(kGwThreads) ebag_bwd_weights_kernel(const BwdW
                 if (on) x = __ldg(reinterpret_cast<const float4*>(go + (size_t)vec * NACC + k));
                 g[k] = x.x; g[k + 1] = x.y; g[k + 2] = x.z; g[k + 3] = x.w;
             }
+            // the ids of the next batch are requested before the current batch's rows
+            int64_t rn[kGwRows];
+            auto fetch_ids = [&](int64_t j0) {
+#pragma unroll
+                for (int k = 0; k < kGwRows; ++k) {
+                    rn[k] = -1;
+                    if (j0 + k < L)
+                        rn[k] = p.idx32 ? (int64_t)__ldg(reinterpret_cast<const int*>(p.indices) + lo + j0 + k)
+                                        : (int64_t)__ldg(reinterpret_cast<const long long*>(p.indices) + lo + j0 + k);
+                }
+            };
+            fetch_ids(0);
             for (int64_t j0 = 0; j0 < Lmax; j0 += kGwRows) {
                 int64_t r[kGwRows];
                 bool valid[kGwRows];
@@ -124,13 +136,11 @@ __global__ void __launch_bounds__(kGwThreads) ebag_bwd_weights_kernel(const BwdW
 #pragma unroll
                 for (int k = 0; k < kGwRows; ++k) {
                     const bool live = j0 + k < L;
-                    r[k] = -1;
-                    if (live)
-                        r[k] = p.idx32 ? (int64_t)__ldg(reinterpret_cast<const int*>(p.indices) + lo + j0 + k)
-                                       : (int64_t)__ldg(reinterpret_cast<const long long*>(p.indices) + lo + j0 + k);
+                    r[k] = rn[k];
                     valid[k] = live && (uint64_t)r[k] < (uint64_t)m.rows;
                     if (live && !valid[k] && lig == 0 && c0 == 0) ++n_oob;
                 }
+                fetch_ids(j0 + kGwRows);
 #pragma unroll
                 for (int k = 0; k < kGwRows; ++k) {
                     d[k] = make_uint4(0u, 0u, 0u, 0u);
