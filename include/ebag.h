@@ -148,7 +148,7 @@ ebag_status ebag_forward_i32(ebag_tbe* h, const void* const* tables, const int32
  * floating-point atomics meet on one address, so two runs of the same call give the same bits
  * (3 + 3 * passes + 2 kernel launches on `stream`, passes = the 8-bit digits the largest table's
  * row count needs).  That path needs offsets that do not decrease, which is checked on the
- * device, n_indices < 2^32 and D[t] <= 8192; otherwise, and with ebag_set_param("bwd_sorted", 0),
+ * device, n_indices < 2^32, D[t] <= 8192 and room for its scratch; otherwise, and with ebag_set_param("bwd_sorted", 0),
  * the call runs the reduction kernel: a short launch that samples the ids of every table for its
  * most frequent rows, whose contributions are then summed in shared memory, and the backward
  * proper, which adds every contribution with a floating-point reduction in memory; their order

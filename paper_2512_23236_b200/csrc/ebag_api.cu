@@ -1050,8 +1050,12 @@ ebag_status ebag_backward(ebag_tbe* h, const float* grad_out, const void* indice
         const bool scaled = w || mode == EBAG_MEAN;
         const size_t need = bwd_sorted_scratch_bytes(n_indices, h->T, max_d, scaled);
         char* scratch = static_cast<char*>(h->s_bwd);
-        if ((st = grow(h, &scratch, &h->cap_bwd, (int64_t)need)) != EBAG_OK) return st;
+        const bool have_scratch = grow(h, &scratch, &h->cap_bwd, (int64_t)need) == EBAG_OK;
         h->s_bwd = scratch;
+        if (!have_scratch) {             // no room for the sorted lists: the reduction kernel needs none
+            h->cuda_error.clear();
+            cudaGetLastError();
+        }
         BwdSortedParams q;
         q.grad_tables = p.grad_tables;
         q.meta = p.meta;
@@ -1066,14 +1070,16 @@ ebag_status ebag_backward(ebag_tbe* h, const float* grad_out, const void* indice
         q.sumD = h->sumD;
         q.mean = p.mean;
         q.idx32 = p.idx32;
-        bwd_sorted_carve(q, h->s_bwd, n_indices, h->T, max_d, scaled);
+        if (have_scratch) bwd_sorted_carve(q, h->s_bwd, n_indices, h->T, max_d, scaled);
         int bits = 1;
         while (bits < 32 && (1ll << bits) <= max_rows) ++bits;       // the key of a skipped id is rows[t] itself
         q.passes = (bits + 7) / 8;
-        int launches = 0;
-        EBAG_CUDA(h, launch_bwd_sorted(q, h->num_sms, s, &launches));
-        h->launches += launches;
-        p.only_if = q.ctl;
+        if (have_scratch) {
+            int launches = 0;
+            EBAG_CUDA(h, launch_bwd_sorted(q, h->num_sms, s, &launches));
+            h->launches += launches;
+            p.only_if = q.ctl;
+        }
     }
     const int grid = h->num_sms * h->bwd_occupancy[w ? 1 : 0];
     EBAG_CUDA(h, launch_bwd(p, w, grid, s));
