@@ -82,8 +82,9 @@ __global__ void __launch_bounds__(256) bwds_plan_kernel(const BwdSortedParams p)
 }
 
 // ---- 3. one key, bag and weight per lookup.  A warp takes 32 consecutive bags; their lookups
-// are one contiguous range, walked 32 at a time, and each lookup finds its bag among the 32 by
+// are one contiguous range, walked 128 at a time (the four loads of a step are issued together), and each lookup finds its bag among the 32 by
 // a five-step search over the lanes' end offsets.
+constexpr int kExpandUnroll = 4;
 __global__ void __launch_bounds__(256) bwds_expand_kernel(const BwdSortedParams p) {
     if (p.ctl[0]) return;
     const int lane = threadIdx.x & 31;
@@ -100,29 +101,40 @@ __global__ void __launch_bounds__(256) bwds_expand_kernel(const BwdSortedParams 
         const int last = n_bags - g0 < 32 ? (int)(n_bags - g0) - 1 : 31;
         const uint32_t p0 = __shfl_sync(kFull, lo, 0);
         const uint32_t p1 = __shfl_sync(kFull, (uint32_t)p.offsets[g + 1], last);
-        for (uint32_t base = p0; base < p1; base += 32) {
-            const uint32_t pos = base + lane;
-            const bool have = pos < p1;
-            const uint32_t q = have ? pos : p1 - 1;
-            int j = 0;                                       // first lane whose bag ends after q
+        for (uint32_t base = p0; base < p1; base += 32 * kExpandUnroll) {
+            int64_t id[kExpandUnroll];
+            float w[kExpandUnroll];
 #pragma unroll
-            for (int step = 16; step > 0; step >>= 1) {
-                const uint32_t hc = __shfl_sync(kFull, hi, j + step - 1);
-                if (hc <= q) j += step;
+            for (int u = 0; u < kExpandUnroll; ++u) {        // every load of the step before any use
+                const uint32_t pos = base + 32 * u + lane;
+                id[u] = 0;
+                w[u] = 1.0f;
+                if (pos < p1) {
+                    id[u] = p.idx32 ? (int64_t)__ldcs(reinterpret_cast<const int*>(p.indices) + pos)
+                                    : (int64_t)__ldcs(reinterpret_cast<const long long*>(p.indices) + pos);
+                    if (p.wts[0] && p.weights) w[u] = __ldcs(p.weights + pos);
+                }
             }
-            const uint32_t rows = __shfl_sync(kFull, rows_l, j);
-            const uint32_t b = __shfl_sync(kFull, b_l, j);
-            const uint32_t len = __shfl_sync(kFull, len_l, j);
-            if (have) {
-                const int64_t id = p.idx32 ? (int64_t)__ldcs(reinterpret_cast<const int*>(p.indices) + pos)
-                                           : (int64_t)__ldcs(reinterpret_cast<const long long*>(p.indices) + pos);
-                const bool ok = (uint64_t)id < (uint64_t)rows;
-                if (!ok) ++n_oob;
-                p.kb[0][pos] = make_uint2(ok ? (uint32_t)id : rows, b);
-                if (p.wts[0]) {
-                    float w = p.weights ? __ldcs(p.weights + pos) : 1.0f;
-                    if (p.mean) w = __fdiv_rn(w, (float)len);
-                    p.wts[0][pos] = w;
+#pragma unroll
+            for (int u = 0; u < kExpandUnroll; ++u) {
+                const uint32_t pos = base + 32 * u + lane;
+                if (base + 32 * u >= p1) break;              // the whole warp
+                const bool have = pos < p1;
+                const uint32_t q = have ? pos : p1 - 1;
+                int j = 0;                                   // first lane whose bag ends after q
+#pragma unroll
+                for (int step = 16; step > 0; step >>= 1) {
+                    const uint32_t hc = __shfl_sync(kFull, hi, j + step - 1);
+                    if (hc <= q) j += step;
+                }
+                const uint32_t rows = __shfl_sync(kFull, rows_l, j);
+                const uint32_t b = __shfl_sync(kFull, b_l, j);
+                const uint32_t len = __shfl_sync(kFull, len_l, j);
+                if (have) {
+                    const bool ok = (uint64_t)id[u] < (uint64_t)rows;
+                    if (!ok) ++n_oob;
+                    p.kb[0][pos] = make_uint2(ok ? (uint32_t)id[u] : rows, b);
+                    if (p.wts[0]) p.wts[0][pos] = p.mean ? __fdiv_rn(w[u], (float)len) : w[u];
                 }
             }
         }
@@ -312,10 +324,10 @@ __device__ __forceinline__ void add_into_row(float* __restrict__ dst, const floa
 }
 
 #ifndef EBAG_RUNSUM_BLOCKS
-#define EBAG_RUNSUM_BLOCKS 4
+#define EBAG_RUNSUM_BLOCKS 3
 #endif
 #ifndef EBAG_RUNSUM_INFLIGHT
-#define EBAG_RUNSUM_INFLIGHT 4
+#define EBAG_RUNSUM_INFLIGHT 8
 #endif
 template <bool WEIGHTS>
 __global__ void __launch_bounds__(256, EBAG_RUNSUM_BLOCKS) bwds_run_sums_kernel(const BwdSortedParams p, int side) {
@@ -451,7 +463,9 @@ __global__ void __launch_bounds__(256, EBAG_RUNSUM_BLOCKS) bwds_run_sums_kernel(
     }
 }
 
-// ---- 6. the runs that sub-chunk borders cut: a warp per run, from the unit where it starts
+// ---- 6. the runs that unit borders cut: a warp per run, from the unit where it starts.  The
+// warp first finds how many pieces follow (32 records at a time), then adds them in order with
+// eight loads in flight: the hottest rows of a table are cut into hundreds of pieces.
 __global__ void __launch_bounds__(256) bwds_join_kernel(const BwdSortedParams p) {
     if (p.ctl[0]) return;
     const int lane = threadIdx.x & 31;
@@ -465,14 +479,38 @@ __global__ void __launch_bounds__(256) bwds_join_kernel(const BwdSortedParams p)
         const uint32_t n_sub = (p.seg[t + 1] - p.seg[t] + kSubChunk - 1) / kSubChunk;
         const uint32_t c = (unit - p.unit_base[t]) / n_sub;
         const int vec = (int)c * 32 + lane;
+        // pieces: units unit + 1 .. unit + count hold a head piece of this run; all but the last say "goes on"
+        uint32_t count = 0;
+        for (uint32_t k0 = unit + 1; k0 < n_units; k0 += 32) {
+            const uint32_t k = k0 + lane;
+            const int32_t flags = k < n_units ? p.rec[2 * k + 1] : 0;
+            // the chain ends at the first unit that has no piece, or after the first piece that does not go on
+            const unsigned none = __ballot_sync(kFull, !(flags & 1));
+            const unsigned last = __ballot_sync(kFull, (flags & 1) && !(flags & 2));
+            const int first_none = none ? __ffs(none) - 1 : 32;
+            const int first_last = last ? __ffs(last) - 1 : 32;
+            if (first_last < first_none) {
+                count += first_last + 1;
+                break;
+            }
+            count += first_none;
+            if (first_none < 32) break;
+        }
         if (vec >= m.nvec) continue;
         float4 acc = *reinterpret_cast<const float4*>(p.partial + ((size_t)p.max_units + unit) * 128 + 4 * lane);
-        for (uint32_t k = unit + 1; k < n_units; ++k) {     // the pieces that follow, in order
-            const int32_t flags = p.rec[2 * k + 1];
-            if (!(flags & 1)) break;
-            const float4 x = *reinterpret_cast<const float4*>(p.partial + (size_t)k * 128 + 4 * lane);
-            acc.x += x.x; acc.y += x.y; acc.z += x.z; acc.w += x.w;
-            if (!(flags & 2)) break;
+        const float* __restrict__ pieces = p.partial + (size_t)(unit + 1) * 128 + 4 * lane;
+        for (uint32_t i0 = 0; i0 < count; i0 += 8) {
+            float4 x[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                x[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (i0 + i < count) x[i] = *reinterpret_cast<const float4*>(pieces + (size_t)(i0 + i) * 128);
+            }
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+                if (i0 + i < count) {                       // in order
+                    acc.x += x[i].x; acc.y += x[i].y; acc.z += x[i].z; acc.w += x[i].w;
+                }
         }
         add_into_row(p.grad_tables[t] + (size_t)row * m.D + 4 * vec, acc);
     }
