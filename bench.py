@@ -1,7 +1,7 @@
 #!/usr/bin/env python
 """Benchmark of the pooled embedding-bag forward on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 1..8] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 1..10] [--impl reference]
 
 One step = one pass of the whole hot path (one ebag_forward launch over all tables of the
 workload).  Default workload: 3, the batched 32-table bf16 TBE (the largest batched-table
@@ -86,6 +86,8 @@ def parse_args():
     ap.add_argument("--ctas-per-sm", type=int, default=0)
     ap.add_argument("--bwd-sorted", type=int, default=-1,
                     help="workload 9: 1/0 = the reproducible (sorted) / the reduction backward; -1: the library's default")
+    ap.add_argument("--gw-base", type=int, default=3, choices=[3, 4, 5],
+                    help="workload 10: whose tables and ids the weights' gradient runs on")
     # shrunk variants of a workload, for profiler captures and quick checks (not bench lines)
     ap.add_argument("--max-tables", type=int, default=0)
     ap.add_argument("--scale-rows", type=float, default=1.0)
@@ -607,6 +609,8 @@ def run_bwd(args, rank, local_rank, world):
     ms = elapsed_ms / args.steps
     achieved = alg / (ms * 1e-3) / 1e9
     n_cpu, dt = cpu_sample()
+    # the kernel that takes most of the call (profiles/ebag_bwd_cfg3.md)
+    bwd_kernel = "ebag_bwd_kernel" if args.bwd_sorted == 0 else "bwds_run_sums_kernel"
     line = {"metric": "pooled_lookups_per_sec", "value": total / (max_ms * 1e-3), "unit": "lookups/s",
             "n_gpus": world, "steps": args.steps, "warmup": warmup, "ms_per_step": max_ms / args.steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
@@ -614,7 +618,7 @@ def run_bwd(args, rank, local_rank, world):
             "e2e": {"value": e2e_total / (e2e_max * 1e-3), "unit": "lookups/s",
                     "h2d_bytes_per_step": int(h_idx.numel() * 8 + h_off.numel() * 8 + h_G.numel() * 4),
                     "d2h_bytes_per_step": 16, "steps": e2e_steps, "ms_per_step": e2e_max / e2e_steps},
-            "roofline": {"bound": "hbm", "kernel": "ebag_bwd_kernel", "achieved": achieved,
+            "roofline": {"bound": "hbm", "kernel": bwd_kernel, "achieved": achieved,
                          "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
                          "peak_source": f"{peaks['source']} HBM copy bandwidth (burst); the reductions are "
                                         "resolved in L2, so this is a reference, not the binding limit",
@@ -624,6 +628,149 @@ def run_bwd(args, rank, local_rank, world):
                              "sample": f"the first {sb} bags of table 0 (Python loops over lookups)",
                              "seconds": dt},
             "steps_accumulated": n_steps}
+    print(json.dumps(line), flush=True)
+
+
+GW_WORKLOAD = 10       # gradient with respect to the per-sample weights
+
+
+def run_gw(args, rank, local_rank, world):
+    """Workload 10: ebag_backward_weights on the tables and jagged ids of workload --gw-base (3, 4
+    or 5): grad_w[i] = <grad_out[b, Doff[t]:+D], value(t, indices[i], :)>.  Algorithmic bytes: per
+    lookup the row + id (8) + the gradient written (4); per bag its grad_out slice (4 D) + offset
+    (8)."""
+    from oracle import ebag_bwd_oracle as bo
+    base = wl.make_workload(args.gw_base, scale_rows=args.scale_rows, scale_B=args.scale_b,
+                            max_tables=args.max_tables or None, seed=bl.rank_seed(0, rank))
+    jag = wl.gen_jagged(base)
+    T, B = base.T, base.B
+    lookups = int(jag.lengths.sum())
+    per_table = np.add.reduceat(jag.lengths, np.arange(0, T * B, B))
+    elem = {wl.F32: 4, wl.F16: 2, wl.BF16: 2, wl.INT8_ROWWISE: 1, wl.UINT8_ROWWISE: 1}[base.dtype]
+    row_bytes = [d * elem + (8 if elem == 1 else 0) for d in base.D]
+    alg = int(sum(int(per_table[t]) * (row_bytes[t] + 12) for t in range(T)) + B * (4 * base.sumD + 8 * T))
+    config = {"workload": "gradw_" + base.name, "tables": T, "bags_per_table": B, "lookups": lookups,
+              "sum_D": base.sumD, "algorithmic_bytes_per_step": alg,
+              "data": f"workload {args.gw_base}'s seeded tables and jagged ids; grad_out N(0,1)",
+              "l2": f"{L2_FLUSH_BYTES >> 20} MiB written between timed steps (L2 flush)"}
+    rng = np.random.default_rng(bl.rank_seed(0, rank) + 1)
+    sb = min(B, 256)                                       # CPU sample: the first bags of table 0
+    rs = min(base.rows[0], 1 << 16)                        # the CPU sample's table: ids folded into its rows
+    cpu_tab = rng.standard_normal((rs, base.D[0])).astype(np.float32)
+
+    def cpu_sample():
+        off = jag.offsets[:sb + 1]
+        idx = jag.indices[:off[-1]] % rs
+        G = rng.standard_normal((sb, base.D[0]))
+        t0 = time.perf_counter()
+        bo.backward_weights([cpu_tab], G, idx, off, sb)
+        return int(off[-1]), time.perf_counter() - t0
+
+    cpu_note = f"the first {sb} bags of table 0 over a {rs}-row table of N(0,1) values (Python loops over lookups)"
+    if args.impl == "reference":
+        if rank != 0:
+            return
+        for _ in range(args.warmup):
+            cpu_sample()
+        n = dt = 0
+        for _ in range(args.steps):
+            a, b = cpu_sample()
+            n += a
+            dt += b
+        v = n / dt
+        print(json.dumps({"impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus,
+                          "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
+                          "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+                          "data": "synthetic", "config": config,
+                          "cpu_baseline": {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": cpu_note},
+                          "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+                          "gpu_launches": 0}), flush=True)
+        return
+    import paper_2512_23236_b200 as eb
+    eb.lib()
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    bl.init_process_group("nccl")
+    warmup = max(3, args.warmup)
+    raw_tables = [wl.gen_table(base, t, dev) for t in range(T)]
+    tables = ([eb.ebag_pack_int8_rowwise(q, s, b) for q, s, b in raw_tables]
+              if base.dtype == wl.INT8_ROWWISE else raw_tables)
+    h_idx = torch.from_numpy(jag.indices).pin_memory()
+    h_off = torch.from_numpy(jag.offsets).pin_memory()
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(bl.rank_seed(0, rank) + 7)
+    d_G = torch.randn((B, base.sumD), device=dev, generator=gen)
+    h_G = d_G.cpu().pin_memory()
+    d_idx, d_off = h_idx.to(dev), h_off.to(dev)
+    s_idx, s_off, s_G = torch.empty_like(d_idx), torch.empty_like(d_off), torch.empty_like(d_G)
+    d_gw = torch.zeros(lookups, device=dev)
+    h_gw = torch.empty(lookups).pin_memory()
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
+    tbe = eb.TBE(base.rows, base.D, base.dtype, device=local_rank)
+    stream = torch.cuda.Stream(device=dev)
+    sampler = bl.ClockSampler(f"GPU-{torch.cuda.get_device_properties(dev).uuid}").start()
+    with torch.cuda.stream(stream):
+        for _ in range(warmup):
+            flush.fill_(1)
+            tbe.backward_weights(tables, d_G, d_idx, d_off, B, base.mode, out=d_gw, stream=stream)
+        stream.synchronize()
+        assert tbe.last_status(stream) == (0, 0, 0)
+        bl.barrier()
+        torch.cuda.synchronize()
+        launches0 = tbe.launch_count()
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+              for _ in range(args.steps)]
+        for a, b in ev:
+            flush.fill_(1)
+            a.record(stream)
+            tbe.backward_weights(tables, d_G, d_idx, d_off, B, base.mode, out=d_gw, stream=stream)
+            b.record(stream)
+        torch.cuda.synchronize()
+        bl.barrier()
+        launches = tbe.launch_count() - launches0
+        step_ms = [a.elapsed_time(b) for a, b in ev]
+        elapsed_ms = float(sum(step_ms))
+        # end to end: host grad_out, ids and offsets in, the weights' gradient back to the host
+        e2e_steps = args.e2e_steps or min(args.steps, 10)
+        ev2 = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+               for _ in range(e2e_steps)]
+        for a, b in ev2:
+            a.record(stream)
+            s_idx.copy_(h_idx, non_blocking=True)
+            s_off.copy_(h_off, non_blocking=True)
+            s_G.copy_(h_G, non_blocking=True)
+            tbe.backward_weights(tables, s_G, s_idx, s_off, B, base.mode, out=d_gw, stream=stream)
+            h_gw.copy_(d_gw, non_blocking=True)
+            b.record(stream)
+        torch.cuda.synchronize()
+        bl.barrier()
+        e2e_ms = float(sum(a.elapsed_time(b) for a, b in ev2))
+    clocks = sampler.stop()
+    total, max_ms = bl.reduce_job(lookups * args.steps, elapsed_ms, dev)
+    e2e_total, e2e_max = bl.reduce_job(lookups * e2e_steps, e2e_ms, dev)
+    tbe.close()
+    if rank != 0:
+        return
+    peaks = bl.measured_peaks(ROOT)
+    ms = elapsed_ms / args.steps
+    achieved = alg / (ms * 1e-3) / 1e9
+    n_cpu, dt = cpu_sample()
+    line = {"metric": METRIC, "value": total / (max_ms * 1e-3), "unit": UNIT,
+            "n_gpus": world, "steps": args.steps, "warmup": warmup, "ms_per_step": max_ms / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+            "data": "synthetic", "config": config, "clocks": clocks, "gpu_launches": launches,
+            "e2e": {"value": e2e_total / (e2e_max * 1e-3), "unit": UNIT,
+                    "h2d_bytes_per_step": int(h_idx.numel() * 8 + h_off.numel() * 8 + h_G.numel() * 4),
+                    "d2h_bytes_per_step": int(h_gw.numel() * 4), "steps": e2e_steps,
+                    "ms_per_step": e2e_max / e2e_steps},
+            "roofline": {"bound": "hbm", "kernel": "ebag_bwd_weights_kernel", "achieved": achieved,
+                         "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
+                         "peak_source": f"{peaks['source']} HBM copy bandwidth (burst); with skewed ids most row "
+                                        "bytes are served by L1 and L2, so this is a reference, not the binding limit",
+                         "algorithmic_bytes_per_launch": alg, "ms_per_launch": ms,
+                         "ms_per_launch_min": min(step_ms), "traffic": None},
+            "cpu_baseline": {"value": n_cpu / dt, "unit": UNIT, "cores": 1, "kind": "oracle",
+                             "sample": cpu_note, "seconds": dt}}
     print(json.dumps(line), flush=True)
 
 
@@ -692,6 +839,9 @@ def main():
         return
     if args.workload == BWD_WORKLOAD:
         run_bwd(args, rank, local_rank, world)
+        return
+    if args.workload == GW_WORKLOAD:
+        run_gw(args, rank, local_rank, world)
         return
     if args.impl == "reference":
         run_reference(args, rank)

@@ -1248,7 +1248,7 @@ ebag_status ebag_backward_weights(ebag_tbe* h, const void* const* tables, const 
     p.idx32 = index_bits == 32 ? 1 : 0;
     p.code_zero = h->dtype == EBAG_UINT8_ROWWISE ? 0.0f : 128.0f;
     EBAG_CUDA(h, launch_bwd_weights(h->dtype == EBAG_UINT8_ROWWISE ? (int)EBAG_INT8_ROWWISE : h->dtype, p,
-                                    h->num_sms * 6, s));
+                                    h->num_sms, s));
     ++h->launches;
     return EBAG_OK;
 }

@@ -25,7 +25,8 @@ struct BwdWeightsParams {
     float code_zero;             // rowwise 8-bit tables: the stored byte that means code 0
 };
 
-size_t bwd_weights_smem_bytes(int T);
-cudaError_t launch_bwd_weights(int dtype, const BwdWeightsParams& p, int grid, cudaStream_t s);
+size_t bwd_weights_smem_bytes(int dtype, int T);
+// one persistent launch: as many CTAs as fit on num_sms multiprocessors
+cudaError_t launch_bwd_weights(int dtype, const BwdWeightsParams& p, int num_sms, cudaStream_t s);
 
 }  // namespace ebag
