@@ -190,6 +190,10 @@ __device__ __forceinline__ void st_stream16(float* p, float a, float b, float c,
 __device__ __forceinline__ void cp_async16(uint32_t smem, const void* gmem) {
     asm volatile("cp.async.ca.shared.global [%0], [%1], 16;" ::"r"(smem), "l"(gmem));
 }
+// a copy of `bytes` (16 or 0) source bytes; what is not copied of the 16 is zeroed
+__device__ __forceinline__ void cp_async16_zfill(uint32_t smem, const void* gmem, uint32_t bytes) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 16, %2;" ::"r"(smem), "l"(gmem), "r"(bytes) : "memory");
+}
 __device__ __forceinline__ void cp_async8(uint32_t smem, const void* gmem) {
     asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(smem), "l"(gmem));
 }
@@ -495,6 +499,9 @@ __device__ __forceinline__ void process_item(const FwdParams& p, const TableMeta
                                                    unsigned& skip, const PartArgs& pa) {
     constexpr int NACC = Elem<DT>::kAcc;
     constexpr int CR = kStageVecs / V;               // rows per stage
+    // stages with gaps: zero-filling copies instead of tests (not for max pooling, where a zero is
+    // not neutral; not for rowwise 8-bit rows, whose instance has no register to spare: measured slower)
+    constexpr bool kZeroFill = POOL == 0 && DT != DT_INT8;
     const int G = 1 << m.g_log2;
     const int NG = 32 >> m.g_log2;
     const int lig = lane & (G - 1);
@@ -566,6 +573,8 @@ __device__ __forceinline__ void process_item(const FwdParams& p, const TableMeta
         const int vec = vec0 + v * G + lig;
         col_on[v] = vec < m.nvec;
         lane_base[v] = tbase + vec * 16;
+        // (a table without rows may come without memory; its copies, all of zero bytes, name the output)
+        if (kZeroFill && m.rows <= 0) lane_base[v] = reinterpret_cast<const char*>(p.out) + vec * 16;
     }
     const uint32_t stride = (uint32_t)m.stride;
     const uint32_t rows = (uint32_t)m.rows;          // tables have fewer than 2^31 rows
@@ -660,17 +669,35 @@ __device__ __forceinline__ void process_item(const FwdParams& p, const TableMeta
             }
             return;
         }
+        if constexpr (kZeroFill) {
+            // A stage with gaps (past a bag's end, a skipped id, a lane past the row's end): every
+            // slot still gets its copy, of zero source bytes where the row is missing, which fills
+            // the slot with zeros and reads nothing; the consuming side then adds zeros and has
+            // nothing to test.  Only the rows past the longest bag's end (warp-uniform) are left out.
 #pragma unroll
-        for (int u = 0; u < CR; ++u) {
-            const uint32_t r = __shfl_sync(0xffffffffu, c.r, j0 + u, G);
-            if (j0 + u < c.nmax && r != kInvalidRow) {
-                const uint64_t roff = (uint64_t)r * stride;
+            for (int u = 0; u < CR; ++u) {
+                if (j0 + u >= c.nmax) break;
+                const uint32_t r = __shfl_sync(0xffffffffu, c.r, j0 + u, G);
+                const bool have = r != kInvalidRow;
+                const uint64_t roff = (uint64_t)(have ? r : 0u) * stride;
 #pragma unroll
                 for (int v = 0; v < V; ++v)
-                    if (col_on[v])
-                        cp_async16(my_rows_s + (st * kStageVecs + u * V + v) * 512, lane_base[v] + roff);
-                if (DT == DT_INT8 && lig == 0)
-                    cp_async8(my_sb_s + (st * kStageVecs + u) * 64, lane_base[0] + roff + sb_delta);
+                    cp_async16_zfill(my_rows_s + (st * kStageVecs + u * V + v) * 512, lane_base[v] + roff,
+                                     (have && col_on[v]) ? 16u : 0u);
+            }
+        } else {
+#pragma unroll
+            for (int u = 0; u < CR; ++u) {
+                const uint32_t r = __shfl_sync(0xffffffffu, c.r, j0 + u, G);
+                if (j0 + u < c.nmax && r != kInvalidRow) {
+                    const uint64_t roff = (uint64_t)r * stride;
+#pragma unroll
+                    for (int v = 0; v < V; ++v)
+                        if (col_on[v])
+                            cp_async16(my_rows_s + (st * kStageVecs + u * V + v) * 512, lane_base[v] + roff);
+                    if (DT == DT_INT8 && lig == 0)
+                        cp_async8(my_sb_s + (st * kStageVecs + u) * 64, lane_base[0] + roff + sb_delta);
+                }
             }
         }
     };
@@ -704,27 +731,41 @@ __device__ __forceinline__ void process_item(const FwdParams& p, const TableMeta
             }
             return;
         }
+        if constexpr (kZeroFill) {
+            // gaps hold zeros (see the request side): the same straight code, up to the longest bag's end
 #pragma unroll
-        for (int u = 0; u < CR; ++u) {
-            const uint32_t r = __shfl_sync(0xffffffffu, c.r, j0 + u, G);
-            float wu = WEIGHTED ? __shfl_sync(0xffffffffu, c.w, j0 + u, G) : 1.0f;
-            if (j0 + u < c.nmax && r != kInvalidRow) {
-                float2 sb = make_float2(1.0f, 0.0f);
-                if (DT == DT_INT8) {
-                    sb = lds64f(my_sb_s + (st * kStageVecs + u) * 64);
-                    if (POOL == 0) {
-                        // the row's constant, bias - zero * scale, rounded once; then the weight
-                        acc_bias = fmaf(wu, fmaf(-p.code_zero, sb.x, sb.y), acc_bias);
-                        wu *= sb.x * kInt8Up;
-                    }
+            for (int u = 0; u < CR; ++u) {
+                if (j0 + u >= c.nmax) break;
+                const float wu = WEIGHTED ? __shfl_sync(0xffffffffu, c.w, j0 + u, G) : 1.0f;
+#pragma unroll
+                for (int v = 0; v < V; ++v) {
+                    const uint4 d = lds128(my_rows_s + (st * kStageVecs + u * V + v) * 512);
+                    accumulate<DT, WEIGHTED>(acc[v], d, wu);
                 }
+            }
+        } else {
 #pragma unroll
-                for (int v = 0; v < V; ++v)
-                    if (col_on[v]) {
-                        const uint4 d = lds128(my_rows_s + (st * kStageVecs + u * V + v) * 512);
-                        if constexpr (POOL == 1) accumulate_max<DT>(acc[v], d, sb.x, sb.y, p.code_zero);
-                        else accumulate<DT, WEIGHTED || DT == DT_INT8>(acc[v], d, wu);
+            for (int u = 0; u < CR; ++u) {
+                const uint32_t r = __shfl_sync(0xffffffffu, c.r, j0 + u, G);
+                float wu = WEIGHTED ? __shfl_sync(0xffffffffu, c.w, j0 + u, G) : 1.0f;
+                if (j0 + u < c.nmax && r != kInvalidRow) {
+                    float2 sb = make_float2(1.0f, 0.0f);
+                    if (DT == DT_INT8) {
+                        sb = lds64f(my_sb_s + (st * kStageVecs + u) * 64);
+                        if (POOL == 0) {
+                            // the row's constant, bias - zero * scale, rounded once; then the weight
+                            acc_bias = fmaf(wu, fmaf(-p.code_zero, sb.x, sb.y), acc_bias);
+                            wu *= sb.x * kInt8Up;
+                        }
                     }
+#pragma unroll
+                    for (int v = 0; v < V; ++v)
+                        if (col_on[v]) {
+                            const uint4 d = lds128(my_rows_s + (st * kStageVecs + u * V + v) * 512);
+                            if constexpr (POOL == 1) accumulate_max<DT>(acc[v], d, sb.x, sb.y, p.code_zero);
+                            else accumulate<DT, WEIGHTED || DT == DT_INT8>(acc[v], d, wu);
+                        }
+                }
             }
         }
     };
