@@ -70,9 +70,11 @@ def _jagged(rng, rows, B, max_len):
 @pytest.mark.parametrize("idx32", [False, True])
 def test_weights_gradient_matches_the_oracle(dtype, mode, idx32):
     rng = np.random.default_rng(11 * dtype + 3 * mode + idx32)
-    # row widths from one vector for four lanes up to two column tiles of 32 lanes
-    D = {wl.F32: [4, 64, 256, 20], wl.F16: [8, 128, 512, 40], wl.BF16: [8, 128, 512, 40]}.get(dtype, [16, 128, 1024, 48])
-    rows = [37, 1000, 211, 64]
+    # row widths of 1, 16 and 64 vectors (two column tiles of 32 lanes), a ragged 5, and 2 and 4 (groups
+    # of fewer lanes than the eight rows of a batch)
+    D = {wl.F32: [4, 64, 256, 20, 8, 16], wl.F16: [8, 128, 512, 40, 16, 32],
+         wl.BF16: [8, 128, 512, 40, 16, 32]}.get(dtype, [16, 128, 1024, 48, 32, 64])
+    rows = [37, 1000, 211, 64, 150, 90]
     B = 97
     lengths, off, idx = _jagged(rng, rows, B, 23)
     idx[::41] = -2                                           # skipped, counted, gradient 0
