@@ -214,6 +214,18 @@ __global__ void __launch_bounds__(256) bwds_scatter_kernel(const BwdSortedParams
     const uint32_t k = tile - p.tile_base[t], nt = p.tile_base[t + 1] - p.tile_base[t];
     const uint32_t s0 = p.seg[t] + k * kSortTile;
     const uint32_t s1 = min(p.seg[t + 1], s0 + (uint32_t)kSortTile);
+    // the tile's lookups are requested first: they travel while the digits' places are worked out
+    const uint2* __restrict__ kb = p.kb[side];
+    const float* __restrict__ wts = WEIGHTS ? p.wts[side] : nullptr;
+    constexpr int kRounds = kSortTile / 256;              // a warp owns kRounds * 32 consecutive lookups of the tile
+    uint2 e[kRounds];
+    float wt[kRounds];
+#pragma unroll
+    for (int r = 0; r < kRounds; ++r) {
+        const uint32_t pos = s0 + (wid * kRounds + r) * 32 + lane;
+        e[r] = pos < s1 ? __ldcs(kb + pos) : make_uint2(0u, 0u);
+        wt[r] = (WEIGHTS && pos < s1) ? __ldcs(wts + pos) : 0.0f;
+    }
 #pragma unroll
     for (int w = 0; w < 8; ++w) wcnt[w][tid] = 0;
     // where digit `tid` of this tile starts in the output: the table's start, the lookups of the
@@ -231,18 +243,11 @@ __global__ void __launch_bounds__(256) bwds_scatter_kernel(const BwdSortedParams
     for (int w = 0; w < wid; ++w) start += warp_sum[w];
     gstart[tid] = start;
 
-    const uint2* __restrict__ kb = p.kb[side];
-    const float* __restrict__ wts = WEIGHTS ? p.wts[side] : nullptr;
-    constexpr int kRounds = kSortTile / 256;              // a warp owns kRounds * 32 consecutive lookups of the tile
-    uint2 e[kRounds];
     uint32_t where[kRounds];                              // digit << 16 | rank among the warp's earlier lookups of that digit
-    float wt[kRounds];
 #pragma unroll
     for (int r = 0; r < kRounds; ++r) {
         const uint32_t pos = s0 + (wid * kRounds + r) * 32 + lane;
         const bool have = pos < s1;
-        e[r] = have ? kb[pos] : make_uint2(0u, 0u);
-        wt[r] = (WEIGHTS && have) ? wts[pos] : 0.0f;
         const uint32_t d = have ? (e[r].x >> shift) & 255u : 256u + lane;     // an absent lookup matches nobody
         const unsigned peers = __match_any_sync(kFull, d);
         const int leader = __ffs(peers) - 1;
