@@ -339,16 +339,26 @@ __global__ void __launch_bounds__(256, EBAG_RUNSUM_BLOCKS) bwds_run_sums_kernel(
     if (p.ctl[0]) return;
     constexpr int kInFlight = EBAG_RUNSUM_INFLIGHT;                          // lookups whose grad_out slices are in flight together
     const int lane = threadIdx.x & 31;
-    const uint32_t n_units = p.unit_base[p.T];
+    // the tables' first units and first lookups, in shared memory: a unit's start-up is then one
+    // round of independent loads instead of a chain of them
+    extern __shared__ uint32_t runsum_smem[];
+    uint32_t* unit_base_s = runsum_smem;                  // [T + 1]
+    uint32_t* seg_s = runsum_smem + p.T + 1;              // [T + 1]
+    for (int i = threadIdx.x; i <= p.T; i += blockDim.x) {
+        unit_base_s[i] = p.unit_base[i];
+        seg_s[i] = p.seg[i];
+    }
+    __syncthreads();
+    const uint32_t n_units = unit_base_s[p.T];
     const uint32_t warps = gridDim.x * (blockDim.x >> 5);
     const uint2* __restrict__ kb = p.kb[side];
     const float* __restrict__ wts = WEIGHTS ? p.wts[side] : nullptr;
     for (uint32_t unit = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); unit < n_units; unit += warps) {
-        const int t = table_of_unit(p.unit_base, p.T, unit);
+        const int t = table_of_unit(unit_base_s, p.T, unit);
         const BwdTableMeta m = p.meta[t];
-        const uint32_t seg0 = p.seg[t], seg1 = p.seg[t + 1];
+        const uint32_t seg0 = seg_s[t], seg1 = seg_s[t + 1];
         const uint32_t n_sub = (seg1 - seg0 + kSubChunk - 1) / kSubChunk;
-        const uint32_t local = unit - p.unit_base[t];
+        const uint32_t local = unit - unit_base_s[t];
         const uint32_t c = local / n_sub, sub = local - c * n_sub;
         const uint32_t s0 = seg0 + sub * kSubChunk;
         const uint32_t s1 = min(seg1, s0 + (uint32_t)kSubChunk);
@@ -589,8 +599,10 @@ cudaError_t launch_bwd_sorted(const BwdSortedParams& p, int num_sms, cudaStream_
         side ^= 1;
         count += 3;
     }
-    if (p.wts[0]) bwds_run_sums_kernel<true><<<wave, 256, 0, s>>>(p, side);
-    else bwds_run_sums_kernel<false><<<wave, 256, 0, s>>>(p, side);
+    const size_t tables_smem = 2 * (size_t)(p.T + 1) * sizeof(uint32_t);
+    const int resident = num_sms * EBAG_RUNSUM_BLOCKS;    // one wave: units are dealt round-robin, all tables in step
+    if (p.wts[0]) bwds_run_sums_kernel<true><<<resident, 256, tables_smem, s>>>(p, side);
+    else bwds_run_sums_kernel<false><<<resident, 256, tables_smem, s>>>(p, side);
     bwds_join_kernel<<<wave, 256, 0, s>>>(p);
     count += 2;
     if (launches) *launches = count;
