@@ -45,12 +45,12 @@ L2_FLUSH_BYTES = 256 << 20
 # by lookups (DRAM traffic here is compulsory misses + ids + output, all proportional to
 # tables x bags); every entry says which capture it came from, and the line carries that along.
 NCU_TRAFFIC = {
-    3: {"small_case_bytes": 993.4e6, "small_case_lookups": 18.83e6, "small_case": "--max-tables 6",
-        "summary": "profiles/ebag_fwd_bf16_cfg3.md", "captured_at_commit": "4ef60c5"},
-    4: {"small_case_bytes": 1.7091e9, "small_case_lookups": 1.637e6, "small_case": "--max-tables 1",
-        "summary": "profiles/ebag_fwd_f32_cfg4.md", "captured_at_commit": "4ef60c5"},
-    5: {"small_case_bytes": 1.3056e9, "small_case_lookups": 20.97e6, "small_case": "--max-tables 8",
-        "summary": "profiles/ebag_fwd_int8_cfg5.md", "captured_at_commit": "4ef60c5"},
+    3: {"small_case_bytes": 991.3e6, "small_case_lookups": 18.83e6, "small_case": "--max-tables 6",
+        "summary": "profiles/ebag_fwd_bf16_cfg3.md", "captured_at_commit": "72112d9"},
+    4: {"small_case_bytes": 1.7087e9, "small_case_lookups": 1.637e6, "small_case": "--max-tables 1",
+        "summary": "profiles/ebag_fwd_f32_cfg4.md", "captured_at_commit": "72112d9"},
+    5: {"small_case_bytes": 1.3074e9, "small_case_lookups": 20.97e6, "small_case": "--max-tables 8",
+        "summary": "profiles/ebag_fwd_int8_cfg5.md", "captured_at_commit": "72112d9"},
 }
 # What the ncu counters of those captures show to be the limit of each workload's launch.
 BOUND = {1: "launch-latency", 2: "latency", 3: "l1+issue", 4: "hbm", 5: "l1+issue"}
