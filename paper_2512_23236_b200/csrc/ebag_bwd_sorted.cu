@@ -7,7 +7,8 @@
 // depends on timing, and the hot rows of a skewed table queue up in L2.  Here the lookups of
 // every table are first SORTED BY ROW, stably, so that the contributions to one row sit next to
 // each other in the order of the lookups, and then every run of equal rows is added up by one
-// warp in that order and written once with a plain read-modify-write.  Two runs of the same call
+// warp in that order and added into its gradient row ONCE (one vector reduction per row and call:
+// a single addend per element, so there is no order to depend on).  Two runs of the same call
 // give the same bits.
 //
 //   1. check     offsets non-decreasing inside [0, n]?  If not, this pipeline steps aside (every
@@ -20,11 +21,13 @@
 //                table's row ids need, tables sorted side by side: per pass a histogram per tile
 //                (2048 lookups), running sums per (table, digit) over the tiles, and a stable
 //                scatter (ranks inside a tile by warp-wide matching, in lookup order)
-//   5. run sums  a warp per sub-chunk of 1024 sorted lookups: walks it in order, adds
-//                w * grad_out[bag] into registers (lanes tile the columns), and at every change of
-//                row adds the sum into the gradient row.  A run cut by the sub-chunk's start or
-//                end leaves its partial sum in scratch instead.
-//   6. join      a warp per cut run: adds the partial sums in order and writes the row.
+//   5. run sums  a warp per unit (table, column tile of 128 columns, 1024 sorted lookups): walks
+//                it in order, eight grad_out slices in flight, adds w * grad_out[bag] into
+//                registers (lanes tile the columns), and at every change of row adds the sum into
+//                the gradient row.  A run cut by the unit's start or end leaves its partial sum
+//                in scratch instead.
+//   6. join      a warp per cut run: counts its pieces, adds them in order and adds the sum into
+//                the row.
 #include <cuda_runtime.h>
 #include <stdint.h>
 
