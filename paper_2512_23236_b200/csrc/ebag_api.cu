@@ -66,6 +66,7 @@ struct ebag_tbe {
     cudaStream_t slot_stream[kTableSlots] = {};    // the stream the slot's copy was enqueued on
     int slot = -1;
     int occupancy[2][2] = {};                      // CTAs per SM, [plain, MapId][unweighted, weighted]
+    unsigned width_classes = 0;                    // bit g: some table's rows are covered by 2^g lanes
     uint32_t item_bytes = 32768;
     int ctas_per_sm = 0;                           // 0: occupancy limit
     // long bags (pooled in parts by a second kernel): one device block carved into the control
@@ -846,6 +847,7 @@ ebag_status ebag_create_tbe(int32_t T, const int64_t* rows, const int32_t* D, eb
     if (T > EBAG_MAX_TABLES) return EBAG_ERR_UNSUPPORTED;
     std::vector<TableMeta> meta(T);
     int64_t d_off = 0;
+    unsigned width_classes = 0;
     for (int t = 0; t < T; ++t) {
         const int64_t stride = ebag_row_stride(dtype, D[t]);
         if (stride < 0 || rows[t] < 0) return EBAG_ERR_INVALID_ARG;
@@ -859,6 +861,7 @@ ebag_status ebag_create_tbe(int32_t T, const int64_t* rows, const int32_t* D, eb
         int g_log2 = 2;
         while ((1 << g_log2) < m.nvec && g_log2 < 5) ++g_log2;
         m.g_log2 = g_log2;
+        width_classes |= 1u << g_log2;
         m.V = m.nvec <= 32 ? 1 : 2;
         d_off += D[t];
         if (d_off >= (1ll << 31)) return EBAG_ERR_UNSUPPORTED;
@@ -876,6 +879,7 @@ ebag_status ebag_create_tbe(int32_t T, const int64_t* rows, const int32_t* D, eb
     h->dtype = dtype;
     h->device = device;
     h->sumD = (int)d_off;
+    h->width_classes = width_classes;
     h->rows.assign(rows, rows + T);
     h->D.assign(D, D + T);
     ebag_status st = EBAG_OK;
@@ -1248,9 +1252,10 @@ ebag_status ebag_backward_weights(ebag_tbe* h, const void* const* tables, const 
     p.mean = mode == EBAG_MEAN ? 1 : 0;
     p.idx32 = index_bits == 32 ? 1 : 0;
     p.code_zero = h->dtype == EBAG_UINT8_ROWWISE ? 0.0f : 128.0f;
+    int launches = 0;
     EBAG_CUDA(h, launch_bwd_weights(h->dtype == EBAG_UINT8_ROWWISE ? (int)EBAG_INT8_ROWWISE : h->dtype, p,
-                                    h->num_sms, s));
-    ++h->launches;
+                                    h->width_classes, h->num_sms, s, &launches));
+    h->launches += launches;
     return EBAG_OK;
 }
 

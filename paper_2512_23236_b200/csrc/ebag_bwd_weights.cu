@@ -74,7 +74,10 @@ __device__ __forceinline__ float dot_vec(const float2* g, const uint4& d, float 
     return s.x + s.y;
 }
 
-template <int DT>
+// One launch per width class: GL = log2 of the lanes that cover a row (or one column tile of
+// it), a compile-time value, so that the butterfly and the batch have no width to branch on; the
+// launch takes the tables of its class and passes the others by.
+template <int DT, int GL>
 __global__ void __launch_bounds__(kGwThreads, DT == DT_INT8 ? 2 : 3) ebag_bwd_weights_kernel(const BwdWeightsParams p) {
     constexpr int NACC = Elem<DT>::kAcc;                // elements per 16-byte row vector
     constexpr int R = kGwRows;
@@ -82,10 +85,9 @@ __global__ void __launch_bounds__(kGwThreads, DT == DT_INT8 ? 2 : 3) ebag_bwd_we
     // [warps][ring], rowwise 8-bit: [warps][scale/bias ring], then [T+1] first item of each table
     int* item_base = reinterpret_cast<int*>(gw_smem + kGwWarps * (kGwRingBytes + (DT == DT_INT8 ? kGwSbBytes : 0)));
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
-    for (int t = tid; t < p.T; t += kGwThreads) {
-        const int ng = 32 >> p.meta[t].g_log2;
-        item_base[t + 1] = (int)((p.B + ng - 1) / ng);
-    }
+    constexpr int G = 1 << GL, ng = 32 >> GL;
+    for (int t = tid; t < p.T; t += kGwThreads)
+        item_base[t + 1] = p.meta[t].g_log2 == GL ? (int)((p.B + ng - 1) / ng) : 0;
     __syncthreads();
     if (tid == 0) {
         item_base[0] = 0;
@@ -108,8 +110,7 @@ __global__ void __launch_bounds__(kGwThreads, DT == DT_INT8 ? 2 : 3) ebag_bwd_we
         }
         const int t = lo_t;
         const TableMeta m = p.meta[t];
-        const int G = 1 << m.g_log2, ng = 32 >> m.g_log2;
-        const int lig = lane & (G - 1), grp = lane >> m.g_log2;
+        const int lig = lane & (G - 1), grp = lane >> GL;
         const int64_t b = (item - item_base[t]) * ng + grp;
         int64_t lo = 0, hi = 0;
         if (b < p.B) {
@@ -134,10 +135,11 @@ __global__ void __launch_bounds__(kGwThreads, DT == DT_INT8 ? 2 : 3) ebag_bwd_we
         const uint32_t rows = (uint32_t)m.rows;             // tables have fewer than 2^31 rows
         const uint32_t stride = (uint32_t)m.stride;
         // after the butterfly this lane holds the sums of n_mine rows of the batch, from row_mine on
-        const int halvings = m.g_log2 < 3 ? m.g_log2 : 3;
-        const int n_mine = R >> halvings;
+        constexpr int halvings = GL < 3 ? GL : 3;
+        constexpr int n_mine = R >> halvings;
         int row_mine = 0;
-        for (int k = 1; k <= halvings; ++k) row_mine += ((lig >> (m.g_log2 - k)) & 1) * (R >> k);
+#pragma unroll
+        for (int k = 1; k <= halvings; ++k) row_mine += ((lig >> (GL - k)) & 1) * (R >> k);
         const bool writer = (lig & ((G >> halvings) - 1)) == 0;
 
         for (int c0 = 0; c0 < m.nvec; c0 += G) {                  // column tiles of G row vectors
@@ -157,7 +159,7 @@ __global__ void __launch_bounds__(kGwThreads, DT == DT_INT8 ? 2 : 3) ebag_bwd_we
             const char* __restrict__ lane_base = tbase + vec * 16;
             // Ids: lane k < C of a group loads the k-th id of a batch (C = min(G, R) rows per batch),
             // two batches before its rows are used; `raw` is looked at one iteration after its load.
-            const int C = G < R ? G : R;
+            constexpr int C = G < R ? G : R;
             int64_t raw = 0;
             bool raw_live = false;
             uint32_t idn = kGwNoRow;                             // lane k: row k of the batch to request next
@@ -191,8 +193,7 @@ __global__ void __launch_bounds__(kGwThreads, DT == DT_INT8 ? 2 : 3) ebag_bwd_we
             };
             auto request = [&](uint32_t slot_s, uint32_t sbslot_s) {
                 const unsigned present = __ballot_sync(0xffffffffu, idn != kGwNoRow);
-                if (G >= R) request_rows(slot_s, sbslot_s, std::true_type());
-                else request_rows(slot_s, sbslot_s, std::false_type());
+                request_rows(slot_s, sbslot_s, std::integral_constant<bool, (G >= R)>());
                 cp_async_commit();
                 return (present >> (lane & ~(G - 1))) & ((1u << C) - 1u);
             };
@@ -220,8 +221,8 @@ __global__ void __launch_bounds__(kGwThreads, DT == DT_INT8 ? 2 : 3) ebag_bwd_we
                 }
                 // the lanes of the group, added along a butterfly (partner distances G/2, G/4, .. 1):
                 // while a lane holds more than one row's value it keeps half and hands over half
-                if (G >= 2) {
-                    const int o = G >> 1;
+                if constexpr (G >= 2) {
+                    constexpr int o = G >> 1;
                     const bool up = (lig & o) != 0;
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
@@ -229,8 +230,8 @@ __global__ void __launch_bounds__(kGwThreads, DT == DT_INT8 ? 2 : 3) ebag_bwd_we
                         s[i] = keep + __shfl_xor_sync(0xffffffffu, send, o);
                     }
                 }
-                if (G >= 4) {
-                    const int o = G >> 2;
+                if constexpr (G >= 4) {
+                    constexpr int o = G >> 2;
                     const bool up = (lig & o) != 0;
 #pragma unroll
                     for (int i = 0; i < 2; ++i) {
@@ -238,12 +239,13 @@ __global__ void __launch_bounds__(kGwThreads, DT == DT_INT8 ? 2 : 3) ebag_bwd_we
                         s[i] = keep + __shfl_xor_sync(0xffffffffu, send, o);
                     }
                 }
-                if (G >= 8) {
-                    const int o = G >> 3;
+                if constexpr (G >= 8) {
+                    constexpr int o = G >> 3;
                     const bool up = (lig & o) != 0;
                     const float keep = up ? s[1] : s[0], send = up ? s[0] : s[1];
                     s[0] = keep + __shfl_xor_sync(0xffffffffu, send, o);
                 }
+#pragma unroll
                 for (int o = G >> 4; o > 0; o >>= 1) s[0] += __shfl_xor_sync(0xffffffffu, s[0], o);
                 {
                     // lookups of this bag in this batch (none if the bag ended before it)
@@ -255,7 +257,7 @@ __global__ void __launch_bounds__(kGwThreads, DT == DT_INT8 ? 2 : 3) ebag_bwd_we
                         if (inv_on && last_tile) x = __fdiv_rn(x, (float)L);
                         *out = x;
                     };
-                    if (G >= R) {                                        // one row per writing lane
+                    if constexpr (G >= R) {                              // one row per writing lane
                         if (writer && row_mine < rem) write(row_mine, s[0]);
                     } else if (writer) {
 #pragma unroll
@@ -285,28 +287,40 @@ size_t bwd_weights_smem_bytes(int dtype, int T) {
     return (size_t)kGwWarps * (kGwRingBytes + (dtype == DT_INT8 ? kGwSbBytes : 0)) + (size_t)(T + 1) * sizeof(int);
 }
 
-template <int DT>
-static cudaError_t launch_one(const BwdWeightsParams& p, int num_sms, cudaStream_t s) {
+template <int DT, int GL>
+static cudaError_t launch_class(const BwdWeightsParams& p, int num_sms, cudaStream_t s) {
     const size_t smem = bwd_weights_smem_bytes(DT, p.T);
     static bool set[64] = {};                            // per device: the shared-memory limit has been raised
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     if (dev < 0 || dev >= 64 || !set[dev]) {
-        e = cudaFuncSetAttribute(ebag_bwd_weights_kernel<DT>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+        e = cudaFuncSetAttribute(ebag_bwd_weights_kernel<DT, GL>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
         if (e != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) set[dev] = true;
     }
-    ebag_bwd_weights_kernel<DT><<<num_sms * (DT == DT_INT8 ? 2 : 3), kGwThreads, smem, s>>>(p);
+    ebag_bwd_weights_kernel<DT, GL><<<num_sms * (DT == DT_INT8 ? 2 : 3), kGwThreads, smem, s>>>(p);
     return cudaGetLastError();
 }
 
-cudaError_t launch_bwd_weights(int dtype, const BwdWeightsParams& p, int num_sms, cudaStream_t s) {
+template <int DT>
+static cudaError_t launch_one(const BwdWeightsParams& p, unsigned classes, int num_sms, cudaStream_t s, int* launches) {
+    cudaError_t e = cudaSuccess;
+    if (e == cudaSuccess && (classes & 4u)) { e = launch_class<DT, 2>(p, num_sms, s); ++*launches; }
+    if (e == cudaSuccess && (classes & 8u)) { e = launch_class<DT, 3>(p, num_sms, s); ++*launches; }
+    if (e == cudaSuccess && (classes & 16u)) { e = launch_class<DT, 4>(p, num_sms, s); ++*launches; }
+    if (e == cudaSuccess && (classes & 32u)) { e = launch_class<DT, 5>(p, num_sms, s); ++*launches; }
+    return e;
+}
+
+cudaError_t launch_bwd_weights(int dtype, const BwdWeightsParams& p, unsigned classes, int num_sms, cudaStream_t s,
+                               int* launches) {
+    *launches = 0;
     switch (dtype) {
-        case DT_F32: return launch_one<DT_F32>(p, num_sms, s);
-        case DT_F16: return launch_one<DT_F16>(p, num_sms, s);
-        case DT_BF16: return launch_one<DT_BF16>(p, num_sms, s);
-        default: return launch_one<DT_INT8>(p, num_sms, s);
+        case DT_F32: return launch_one<DT_F32>(p, classes, num_sms, s, launches);
+        case DT_F16: return launch_one<DT_F16>(p, classes, num_sms, s, launches);
+        case DT_BF16: return launch_one<DT_BF16>(p, classes, num_sms, s, launches);
+        default: return launch_one<DT_INT8>(p, classes, num_sms, s, launches);
     }
 }
 

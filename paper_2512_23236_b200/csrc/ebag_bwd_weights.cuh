@@ -26,7 +26,9 @@ struct BwdWeightsParams {
 };
 
 size_t bwd_weights_smem_bytes(int dtype, int T);
-// one persistent launch: as many CTAs as fit on num_sms multiprocessors
-cudaError_t launch_bwd_weights(int dtype, const BwdWeightsParams& p, int num_sms, cudaStream_t s);
+// one persistent launch (as many CTAs as fit on num_sms multiprocessors) per width class present:
+// bit g of `classes` is set when some table has g_log2 == g (2..5); *launches receives their number
+cudaError_t launch_bwd_weights(int dtype, const BwdWeightsParams& p, unsigned classes, int num_sms, cudaStream_t s,
+                               int* launches);
 
 }  // namespace ebag
