@@ -7,8 +7,9 @@
 // forward's gather with the roles swapped: the bag's slice sits in registers (G lanes x one
 // 16-byte row vector each, wider rows in column tiles of G vectors); the looked-up rows travel
 // eight at a time through a ring of two stages in shared memory (asynchronous 16-byte copies into
-// slots private to each lane, so no barrier is needed; the ids of the batch after the next are
-// requested before that); the eight dot products of a batch are summed over the lanes of the
+// slots private to each lane, so no barrier is needed; the (scale, bias) pair of a rowwise 8-bit
+// row is copied once per group, by its first lane, and read after a __syncwarp; the ids of the
+// batch after the next are requested before that); the eight dot products of a batch are summed over the lanes of the
 // group together (at every step of the butterfly a lane hands half of its values to its partner
 // and keeps the other half: 7 + log2(G/8) shuffles for 8 rows instead of 8 log2(G); the tree of
 // additions is the same for every row, so the result is reproducible bit for bit) and up to eight
@@ -31,7 +32,7 @@ constexpr int kGwWarps = kGwThreads / 32;
 constexpr int kGwRows = 8;            // rows of a bag per batch (one stage of the ring)
 constexpr uint32_t kGwNoRow = 0xffffffffu;
 constexpr int kGwRingBytes = 2 * kGwRows * 512;       // per warp: two stages of kGwRows 16-byte vectors per lane
-constexpr int kGwSbBytes = 2 * kGwRows * 256;         // per warp, rowwise 8-bit: (scale, bias) of every row, a copy per lane
+constexpr int kGwSbBytes = 2 * kGwRows * 8 * 8;       // per warp, rowwise 8-bit: (scale, bias) of every row, one copy per group (at most 8 groups)
 
 // asynchronous copy of `bytes` (16 / 8 or 0) source bytes; the rest of the 16 / 8 are zeroed
 __device__ __forceinline__ void cp_async16_zfill(uint32_t smem, const void* gmem, uint32_t bytes) {
@@ -78,7 +79,7 @@ __device__ __forceinline__ float dot_vec(const float2* g, const uint4& d, float 
 // it), a compile-time value, so that the butterfly and the batch have no width to branch on; the
 // launch takes the tables of its class and passes the others by.
 template <int DT, int GL>
-__global__ void __launch_bounds__(kGwThreads, DT == DT_INT8 ? 2 : 3) ebag_bwd_weights_kernel(const BwdWeightsParams p) {
+__global__ void __launch_bounds__(kGwThreads, 3) ebag_bwd_weights_kernel(const BwdWeightsParams p) {
     constexpr int NACC = Elem<DT>::kAcc;                // elements per 16-byte row vector
     constexpr int R = kGwRows;
     extern __shared__ __align__(16) unsigned char gw_smem[];
@@ -97,9 +98,10 @@ __global__ void __launch_bounds__(kGwThreads, DT == DT_INT8 ? 2 : 3) ebag_bwd_we
     const int64_t total = item_base[p.T];
     const int64_t warps = (int64_t)gridDim.x * kGwWarps;
     unsigned n_oob = 0, n_bad = 0;
-    // this lane's slots: row u of stage st at ring_s + (st * R + u) * 512 (and sb_s + (st * R + u) * 256)
+    // this lane's slots: row u of stage st at ring_s + (st * R + u) * 512; its group's (scale, bias) of
+    // that row at sb_s + (st * R + u) * ng * 8 (copied by the group's first lane, read by all after a __syncwarp)
     uint32_t ring_s = (uint32_t)__cvta_generic_to_shared(gw_smem) + wid * kGwRingBytes + lane * 16;
-    uint32_t sb_s = (uint32_t)__cvta_generic_to_shared(gw_smem) + kGwWarps * kGwRingBytes + wid * kGwSbBytes + lane * 8;
+    uint32_t sb_s = (uint32_t)__cvta_generic_to_shared(gw_smem) + kGwWarps * kGwRingBytes + wid * kGwSbBytes + (lane >> GL) * 8;
     asm volatile("" : "+r"(ring_s), "+r"(sb_s));
 
     for (int64_t item = (int64_t)blockIdx.x * kGwWarps + wid; item < total; item += warps) {
@@ -188,7 +190,7 @@ __global__ void __launch_bounds__(kGwThreads, DT == DT_INT8 ? 2 : 3) ebag_bwd_we
                     const bool have = r != kGwNoRow && on;
                     const uint64_t roff = (uint64_t)(have ? r : 0u) * stride;
                     cp_async16_zfill(slot_s + k * 512, lane_base + roff, have ? 16u : 0u);
-                    if (DT == DT_INT8) cp_async8_zfill(sbslot_s + k * 256, tbase + roff + m.D, have ? 8u : 0u);
+                    if (DT == DT_INT8 && lig == 0) cp_async8_zfill(sbslot_s + k * (ng * 8), tbase + roff + m.D, have ? 8u : 0u);
                 }
             };
             auto request = [&](uint32_t slot_s, uint32_t sbslot_s) {
@@ -202,20 +204,21 @@ __global__ void __launch_bounds__(kGwThreads, DT == DT_INT8 ? 2 : 3) ebag_bwd_we
             fetch_id(C);
             // the stage being used and the one being filled, as addresses in the shared window
             uint32_t slot_c = ring_s, slot_n = ring_s + R * 512;
-            uint32_t sb_c = sb_s, sb_n = sb_s + R * 256;
+            uint32_t sb_c = sb_s, sb_n = sb_s + R * (ng * 8);
             unsigned valid_c = request(slot_c, sb_c);
             for (uint32_t j0 = 0; j0 < Lmax; j0 += C) {
                 check_id();                                      // the batch after this one: loaded an iteration ago
                 fetch_id(j0 + 2 * C);
                 const unsigned valid_n = request(slot_n, sb_n);
                 cp_async_wait<1>();                              // everything but the newest group has landed
+                if (DT == DT_INT8) __syncwarp();                 // (the pairs were copied by the groups' first lanes)
                 float s[R];
 #pragma unroll
                 for (int k = 0; k < R; ++k) {
                     const uint4 d = lds128(slot_c + k * 512);
                     s[k] = dot_vec<DT>(g, d, p.code_zero);
                     if (DT == DT_INT8) {                         // sum g * (scale * q + bias) = scale * sum g q + bias * sum g
-                        const float2 sb = lds64f(sb_c + k * 256);
+                        const float2 sb = lds64f(sb_c + k * (ng * 8));
                         s[k] = fmaf(sb.x, s[k], sb.y * sum_g);
                     }
                 }
@@ -299,7 +302,7 @@ static cudaError_t launch_class(const BwdWeightsParams& p, int num_sms, cudaStre
         if (e != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) set[dev] = true;
     }
-    ebag_bwd_weights_kernel<DT, GL><<<num_sms * (DT == DT_INT8 ? 2 : 3), kGwThreads, smem, s>>>(p);
+    ebag_bwd_weights_kernel<DT, GL><<<num_sms * 3, kGwThreads, smem, s>>>(p);
     return cudaGetLastError();
 }
 
