@@ -394,6 +394,27 @@ def test_out_of_range_ids_skipped_and_counted():
         pu.compare(gpu, ref, wl.F32, lengths, 2, B, D)
 
 
+@pytest.mark.parametrize("dtype", [wl.F32, wl.BF16, wl.INT8_ROWWISE])
+def test_table_without_rows(dtype):
+    """A table of zero rows (it may come without memory): every id that names it is skipped and
+    counted, its output columns read +0, and the other tables are pooled as ever."""
+    rng = np.random.default_rng(21 + dtype)
+    rows, D, B = [50, 0, 20], [32, 64, 16], 37
+    lens = [rng.integers(0, 12, size=B) for _ in rows]
+    lengths = np.concatenate(lens).astype(np.int64)
+    off = np.zeros(3 * B + 1, np.int64)
+    np.cumsum(lengths, out=off[1:])
+    idx = np.concatenate([rng.integers(0, max(r, 5), size=int(l.sum())) for r, l in zip(rows, lens)]).astype(np.int64)
+    tabs = _rand_tables(rng, dtype, rows, D)
+    for mode in (wl.SUM, wl.MEAN):
+        gpu, status, ref = _both(dtype, rows, D, tabs, idx, off, B, mode)
+        n1 = int(lens[1].sum())
+        assert n1 > 0 and ref["n_oob"] == n1
+        assert status == (eb.EBAG_ERR_INDEX_OOB, n1, 0)
+        pu.compare(gpu, ref, dtype, lengths, 3, B, D)
+        assert float(np.abs(gpu[:, 32:96]).max()) == 0.0
+
+
 def test_bad_offsets_treated_as_empty_and_counted():
     rng = np.random.default_rng(10)
     rows, D, B = [100], [16], 40
