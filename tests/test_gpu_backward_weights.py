@@ -108,6 +108,34 @@ def test_weights_gradient_matches_the_oracle(dtype, mode, idx32):
     assert np.all(g[ref["S"] == 0] == 0.0)
 
 
+@pytest.mark.parametrize("dtype", [wl.F32, wl.INT8_ROWWISE])
+def test_weights_gradient_with_a_table_without_rows(dtype):
+    # every id that names the empty table is skipped and counted and gets the gradient 0
+    rng = np.random.default_rng(77 + dtype)
+    rows, D, B = [40, 0, 9], [32, 64, 16], 31
+    lengths = rng.integers(0, 14, size=3 * B)
+    off = np.zeros(3 * B + 1, np.int64)
+    np.cumsum(lengths, out=off[1:])
+    idx = np.concatenate([rng.integers(0, max(rows[t], 3), size=int(lengths[t * B:(t + 1) * B].sum()))
+                          for t in range(3)]).astype(np.int64)
+    tabs, vals = _tables(rng, dtype, rows, D)
+    G = rng.standard_normal((B, sum(D))).astype(np.float32)
+    ref = bo.backward_weights(vals, G, idx, off, B, wl.SUM)
+    tbe = eb.TBE(rows, D, dtype, device=torch.cuda.current_device())
+    try:
+        got = tbe.backward_weights(_device_tables(dtype, tabs), torch.from_numpy(G).cuda(),
+                                   torch.from_numpy(idx).cuda(), torch.from_numpy(off).cuda(), B, wl.SUM)
+        status = tbe.last_status()
+    finally:
+        tbe.close()
+    n1 = int(off[2 * B] - off[B])
+    assert n1 > 0 and ref["n_oob"] == n1 and status[1:] == (n1, 0)
+    g = got.cpu().numpy().astype(np.float64)
+    assert np.all(g[off[B]:off[2 * B]] == 0.0)
+    width = np.concatenate([np.full(int(off[(t + 1) * B] - off[t * B]), D[t]) for t in range(3)])
+    assert np.all(np.abs(g - ref["grad_w"]) <= (width + 4) * U * ref["S"] + 1e-30)
+
+
 def test_weights_gradient_at_a_workload_shape():
     # workload 4's shape scaled down (fp32, 1 KB rows: two column tiles), checked against the oracle
     w = wl.make_workload(4, scale_rows=0.002, scale_B=1 / 256, max_tables=3)
