@@ -175,8 +175,11 @@ ebag_status ebag_backward(ebag_tbe* h, const float* grad_out, const void* indice
  *                 bag (0 for an id outside its table, which is counted); entries that no
  *                 well-formed bag covers are left as they are, and an entry that malformed
  *                 offsets put into several bags receives the value of one of them.
- * One kernel on `stream`, no allocation; the sums over a row are added in a fixed order, so two
- * runs give the same bits.  D[t] must be a multiple of 4.  A bag is walked by one group of lanes,
+ * One to four kernels on `stream` (one per width class of the tables: rows covered by 4, 8, 16
+ * or 32 lanes), no allocation; the sums over a row are added in a fixed order, so two runs give
+ * the same bits.  A rowwise 8-bit row contributes scale * sum_d g_d * code_d + bias * sum_d g_d
+ * (the value() of the forward rounds scale * code + bias per element first; the two differ by a
+ * few roundings of the terms).  D[t] must be a multiple of 4.  A bag is walked by one group of lanes,
  * so a single very long bag is slow (it is not split as in the forward).  Counts of skipped ids
  * and malformed bags go to ebag_last_status.
  */
