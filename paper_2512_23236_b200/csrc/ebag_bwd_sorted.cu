@@ -201,7 +201,7 @@ __global__ void __launch_bounds__(256) bwds_scan_kernel(const BwdSortedParams p)
 // lower lane.  The tile is first put in order in shared memory and then written out, so that
 // every run of equal digits leaves as one contiguous, coalesced piece.
 template <bool WEIGHTS>
-__global__ void __launch_bounds__(256) bwds_scatter_kernel(const BwdSortedParams p, int side, int shift) {
+__global__ void __launch_bounds__(256, 4) bwds_scatter_kernel(const BwdSortedParams p, int side, int shift) {
     if (p.ctl[0]) return;
     const uint32_t tile = blockIdx.x;
     if (tile >= p.tile_base[p.T]) return;
@@ -247,20 +247,25 @@ __global__ void __launch_bounds__(256) bwds_scatter_kernel(const BwdSortedParams
     gstart[tid] = start;
 
     uint32_t where[kRounds];                              // digit << 16 | rank among the warp's earlier lookups of that digit
+    unsigned peers[kRounds];                              // the lanes of the round with the same digit
 #pragma unroll
-    for (int r = 0; r < kRounds; ++r) {
+    for (int r = 0; r < kRounds; ++r) {                   // the matches of all rounds first: they do not depend on one another
         const uint32_t pos = s0 + (wid * kRounds + r) * 32 + lane;
-        const bool have = pos < s1;
-        const uint32_t d = have ? (e[r].x >> shift) & 255u : 256u + lane;     // an absent lookup matches nobody
-        const unsigned peers = __match_any_sync(kFull, d);
-        const int leader = __ffs(peers) - 1;
+        const uint32_t d = pos < s1 ? (e[r].x >> shift) & 255u : 256u + lane;     // an absent lookup matches nobody
+        peers[r] = __match_any_sync(kFull, d);
+        where[r] = d << 16;
+    }
+#pragma unroll
+    for (int r = 0; r < kRounds; ++r) {                   // then the counts, round after round
+        const uint32_t d = where[r] >> 16;
+        const int leader = __ffs(peers[r]) - 1;
         uint32_t old = 0;
-        if (lane == leader && have) {
+        if (lane == leader && d < 256u) {
             old = wcnt[wid][d];
-            wcnt[wid][d] = old + __popc(peers);
+            wcnt[wid][d] = old + __popc(peers[r]);
         }
         old = __shfl_sync(kFull, old, leader);
-        where[r] = (d << 16) | (old + __popc(peers & ((1u << lane) - 1u)));
+        where[r] |= old + __popc(peers[r] & ((1u << lane) - 1u));
         __syncwarp();
     }
     __syncthreads();
