@@ -86,6 +86,8 @@ def parse_args():
     ap.add_argument("--ctas-per-sm", type=int, default=0)
     ap.add_argument("--bwd-sorted", type=int, default=-1,
                     help="workload 9: 1/0 = the reproducible (sorted) / the reduction backward; -1: the library's default")
+    ap.add_argument("--bwd-base", type=int, default=3, choices=[3, 4, 5],
+                    help="workload 9: whose jagged ids (and weights) and table shapes the backward runs on")
     ap.add_argument("--gw-base", type=int, default=3, choices=[3, 4, 5],
                     help="workload 10: whose tables and ids the weights' gradient runs on")
     # shrunk variants of a workload, for profiler captures and quick checks (not bench lines)
@@ -497,16 +499,17 @@ def run_bwd(args, rank, local_rank, world):
     bytes: per lookup the reduction's payload (4 D) + id (8); per bag grad_out (4 D) + offset (8).
     The reductions are resolved in L2, so the HBM copy bandwidth is a reference, not the bound."""
     from oracle import ebag_bwd_oracle as bo
-    base = wl.make_workload(3, scale_rows=args.scale_rows, scale_B=args.scale_b, max_tables=args.max_tables or None,
-                            seed=bl.rank_seed(0, rank))
+    base = wl.make_workload(args.bwd_base, scale_rows=args.scale_rows, scale_B=args.scale_b,
+                            max_tables=args.max_tables or None, seed=bl.rank_seed(0, rank))
     jag = wl.gen_jagged(base)
     T, B = base.T, base.B
     lookups = int(jag.lengths.sum())
     per_table = np.add.reduceat(jag.lengths, np.arange(0, T * B, B))
-    alg = int(sum(int(per_table[t]) * (4 * base.D[t] + 8) for t in range(T)) + B * (4 * base.sumD + 8 * T))
+    wbytes = 4 if jag.weights is not None else 0
+    alg = int(sum(int(per_table[t]) * (4 * base.D[t] + 8 + wbytes) for t in range(T)) + B * (4 * base.sumD + 8 * T))
     config = {"workload": "bwd_" + base.name, "tables": T, "bags_per_table": B, "lookups": lookups,
               "sum_D": base.sumD, "gradient_tables": "dense fp32", "algorithmic_bytes_per_step": alg,
-              "data": "workload 3's seeded jagged ids; grad_out N(0,1)",
+              "data": f"workload {args.bwd_base}'s seeded jagged ids (and weights); grad_out N(0,1)",
               "l2": f"{L2_FLUSH_BYTES >> 20} MiB written between timed steps (L2 flush)"}
     rng = np.random.default_rng(bl.rank_seed(0, rank) + 1)
     sb = min(B, 512)                                       # CPU sample: the first bags of table 0
@@ -553,6 +556,9 @@ def run_bwd(args, rank, local_rank, world):
     d_G = torch.randn((B, base.sumD), device=dev, generator=gen)
     h_G = d_G.cpu().pin_memory()
     d_idx, d_off = h_idx.to(dev), h_off.to(dev)
+    h_w = None if jag.weights is None else torch.from_numpy(jag.weights).pin_memory()
+    d_w = None if h_w is None else h_w.to(dev)
+    s_w = None if h_w is None else torch.empty_like(d_w)
     s_idx, s_off, s_G = torch.empty_like(d_idx), torch.empty_like(d_off), torch.empty_like(d_G)
     h_status = torch.zeros(2, dtype=torch.int64).pin_memory()
     flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
@@ -564,7 +570,7 @@ def run_bwd(args, rank, local_rank, world):
     with torch.cuda.stream(stream):
         for _ in range(warmup):
             flush.fill_(1)
-            tbe.backward(d_G, d_idx, d_off, B, grads, stream=stream)
+            tbe.backward(d_G, d_idx, d_off, B, grads, base.mode, d_w, stream=stream)
         stream.synchronize()
         assert tbe.last_status(stream) == (0, 0, 0)
         bl.barrier()
@@ -575,7 +581,7 @@ def run_bwd(args, rank, local_rank, world):
         for a, b in ev:
             flush.fill_(1)
             a.record(stream)
-            tbe.backward(d_G, d_idx, d_off, B, grads, stream=stream)
+            tbe.backward(d_G, d_idx, d_off, B, grads, base.mode, d_w, stream=stream)
             b.record(stream)
         torch.cuda.synchronize()
         bl.barrier()
@@ -592,7 +598,9 @@ def run_bwd(args, rank, local_rank, world):
             s_idx.copy_(h_idx, non_blocking=True)
             s_off.copy_(h_off, non_blocking=True)
             s_G.copy_(h_G, non_blocking=True)
-            tbe.backward(s_G, s_idx, s_off, B, grads, stream=stream)
+            if s_w is not None:
+                s_w.copy_(h_w, non_blocking=True)
+            tbe.backward(s_G, s_idx, s_off, B, grads, base.mode, s_w, stream=stream)
             h_status.copy_(grads[0][0, :2].to(torch.int64), non_blocking=True)
             b.record(stream)
         torch.cuda.synchronize()
@@ -616,7 +624,8 @@ def run_bwd(args, rank, local_rank, world):
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
             "data": "synthetic", "config": config, "clocks": clocks, "gpu_launches": launches,
             "e2e": {"value": e2e_total / (e2e_max * 1e-3), "unit": "lookups/s",
-                    "h2d_bytes_per_step": int(h_idx.numel() * 8 + h_off.numel() * 8 + h_G.numel() * 4),
+                    "h2d_bytes_per_step": int(h_idx.numel() * 8 + h_off.numel() * 8 + h_G.numel() * 4 +
+                                              (0 if h_w is None else h_w.numel() * 4)),
                     "d2h_bytes_per_step": 16, "steps": e2e_steps, "ms_per_step": e2e_max / e2e_steps},
             "roofline": {"bound": "hbm", "kernel": bwd_kernel, "achieved": achieved,
                          "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
