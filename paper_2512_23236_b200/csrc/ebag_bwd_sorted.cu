@@ -342,10 +342,13 @@ __device__ __forceinline__ void add_into_row(float* __restrict__ dst, const floa
 #ifndef EBAG_RUNSUM_INFLIGHT
 #define EBAG_RUNSUM_INFLIGHT 8
 #endif
+#ifndef EBAG_RUNSUM_INFLIGHT_W
+#define EBAG_RUNSUM_INFLIGHT_W 4
+#endif
 template <bool WEIGHTS>
 __global__ void __launch_bounds__(256, EBAG_RUNSUM_BLOCKS) bwds_run_sums_kernel(const BwdSortedParams p, int side) {
     if (p.ctl[0]) return;
-    constexpr int kInFlight = EBAG_RUNSUM_INFLIGHT;                          // lookups whose grad_out slices are in flight together
+    constexpr int kInFlight = WEIGHTS ? EBAG_RUNSUM_INFLIGHT_W : EBAG_RUNSUM_INFLIGHT;                          // lookups whose grad_out slices are in flight together
     const int lane = threadIdx.x & 31;
     // the tables' first units and first lookups, in shared memory: a unit's start-up is then one
     // round of independent loads instead of a chain of them
