@@ -91,6 +91,7 @@ def parse_args():
     ap.add_argument("--gw-base", type=int, default=3, choices=[3, 4, 5],
                     help="workload 10: whose tables and ids the weights' gradient runs on")
     # shrunk variants of a workload, for profiler captures and quick checks (not bench lines)
+    ap.add_argument("--row-d", type=int, default=0, help="every table with rows of this many elements instead")
     ap.add_argument("--max-tables", type=int, default=0)
     ap.add_argument("--scale-rows", type=float, default=1.0)
     ap.add_argument("--scale-b", type=float, default=1.0)
@@ -106,12 +107,16 @@ def make_workload(args, seed):
                              max_tables=args.max_tables or None, seed=seed)
         w.name = "cfg3_rows_div100_raw_ids_mapid"
         return w
-    return wl.make_workload(args.workload, scale_rows=args.scale_rows, scale_B=args.scale_b,
-                            max_tables=args.max_tables or None, seed=seed)
+    w = wl.make_workload(args.workload, scale_rows=args.scale_rows, scale_B=args.scale_b,
+                         max_tables=args.max_tables or None, seed=seed)
+    if args.row_d:          # the same jagged structure over rows of another width (a probe, not a bench line)
+        w.D = [args.row_d] * w.T
+        w.name += f"_D{args.row_d}"
+    return w
 
 
 def workload_config(w, ab, args=None):
-    shrunk = args is not None and (args.max_tables or args.scale_rows != 1.0 or args.scale_b != 1.0)
+    shrunk = args is not None and (args.max_tables or args.scale_rows != 1.0 or args.scale_b != 1.0 or args.row_d)
     extra = {}
     if args is not None and args.workload == MAPID_WORKLOAD:
         extra = {"mapid": "per table a sorted list of rows-1 known raw ids (1 k - 100 k; the paper's "
