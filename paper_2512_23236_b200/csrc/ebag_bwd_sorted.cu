@@ -164,36 +164,50 @@ __global__ void __launch_bounds__(256) bwds_hist_kernel(const BwdSortedParams p,
     p.hist[(size_t)256 * p.tile_base[t] + (size_t)threadIdx.x * nt + k] = cnt[threadIdx.x];
 }
 
-// ---- 4b. per (digit, table): running sums of the tiles' counts (in place), the total beside them
+// ---- 4b. per (digit, table): running sums of the tiles' counts (in place), the total beside them.
+// A thread takes a run of consecutive tiles (all its loads in flight at once), the runs' totals
+// are scanned across the CTA once; tables of more than 256 * kScanRun tiles go round again.
+constexpr int kScanRun = 8;
 __global__ void __launch_bounds__(256) bwds_scan_kernel(const BwdSortedParams p) {
     if (p.ctl[0]) return;
     const int d = blockIdx.x, t = blockIdx.y;
     const uint32_t nt = p.tile_base[t + 1] - p.tile_base[t];
     uint32_t* __restrict__ a = p.hist + (size_t)256 * p.tile_base[t] + (size_t)d * nt;
     __shared__ uint32_t warp_sum[8];
-    __shared__ uint32_t carry_s;
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
-    if (threadIdx.x == 0) carry_s = 0;
-    __syncthreads();
-    for (uint32_t i0 = 0; i0 < nt; i0 += 256) {
-        const uint32_t i = i0 + threadIdx.x;
-        const uint32_t x = i < nt ? a[i] : 0u;
-        uint32_t inc = x;
+    uint32_t carry = 0;                                   // the same in every thread
+    for (uint32_t i0 = 0; i0 < nt; i0 += 256 * kScanRun) {
+        const uint32_t first = i0 + threadIdx.x * kScanRun;
+        uint32_t x[kScanRun];
+#pragma unroll
+        for (int k = 0; k < kScanRun; ++k) x[k] = first + k < nt ? a[first + k] : 0u;
+        uint32_t mine = 0;
+#pragma unroll
+        for (int k = 0; k < kScanRun; ++k) mine += x[k];
+        uint32_t inc = mine;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
             const uint32_t y = __shfl_up_sync(kFull, inc, o);
             if (lane >= o) inc += y;
         }
+        __syncthreads();                                  // (warp_sum of the round before has been read)
         if (lane == 31) warp_sum[wid] = inc;
         __syncthreads();
-        uint32_t before = carry_s;
-        for (int w = 0; w < wid; ++w) before += warp_sum[w];
-        if (i < nt) a[i] = before + inc - x;
-        __syncthreads();
-        if (threadIdx.x == 255) carry_s = before + inc;
-        __syncthreads();
+        uint32_t before = carry, all = 0;
+#pragma unroll
+        for (int w = 0; w < 8; ++w) {
+            if (w < wid) before += warp_sum[w];
+            all += warp_sum[w];
+        }
+        uint32_t run = before + inc - mine;
+#pragma unroll
+        for (int k = 0; k < kScanRun; ++k) {
+            if (first + k < nt) a[first + k] = run;
+            run += x[k];
+        }
+        carry += all;
     }
-    if (threadIdx.x == 0) p.totals[t * 256 + d] = carry_s;
+    if (threadIdx.x == 0) p.totals[t * 256 + d] = carry;
 }
 
 // ---- 4c. stable scatter of a tile.  Warp w owns an eighth of the tile's lookups, consecutive ones,
